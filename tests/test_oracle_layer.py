@@ -66,7 +66,7 @@ def test_backward_matches_central_finite_differences():
     X, Q, P = g.standard_normal((T, d)), g.standard_normal((r, d)), g.standard_normal((dp, r))
     R = g.standard_normal((T, dp))
     u = O.gate_uniforms(r, 0, 0)
-    alpha = np.array([0.2, -0.4, 1.0, 3.5, -3.5, 0.6])     # two gates end on a clamp
+    alpha = np.array([0.2, -1.5, 1.0, 3.5, -6.0, 0.6])     # gates 2,3 end on the upper clamp, gate 4 on the lower
     z, mask, dzda = O.hard_concrete(alpha, u, BETA, GAMMA, ZETA)
     inner = (z > 0) & (z < 1)
     assert np.any(z == 0) and np.any(z == 1) and inner.sum() >= 3
