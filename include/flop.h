@@ -1,0 +1,160 @@
+/*
+ * flop.h -- C ABI of the B200 (sm_100a) hot path of FLOP, factorized low-rank
+ * pruning ("Structured Pruning of Large Language Models", arXiv 1910.04732).
+ *
+ * The layer is y = P G Q x with G = diag(z) (Section 4.1): W in R^{d_out x d_in}
+ * is replaced by P in R^{d_out x r}, Q in R^{r x d_in} and one hard-concrete
+ * gate z_k per rank-1 component p_k q_k (Section 3).
+ *
+ * Conventions for every entry point
+ *   - Matrices are row-major with an element leading dimension (ld*).  Tokens
+ *     are rows: X[T, d_in], Y[T, d_out], H'[T, r]; P[d_out, r]; Q[r, d_in].
+ *   - Unless a parameter says HOST, every pointer is a DEVICE pointer owned by
+ *     the caller.  The library allocates no device memory; scratch is passed
+ *     in as (ws, ws_bytes) and sized with flop_workspace_bytes().  ws must be
+ *     256-byte aligned.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*); no
+ *     call synchronises unless it says so.
+ *   - dt is the storage type of X, P, Q, Y, H' and of the activation
+ *     gradients.  FLOP_BF16 computes on the tensor cores with fp32
+ *     accumulation and needs every bf16 leading dimension to be a multiple of
+ *     8 elements and every bf16 base pointer to be 16-byte aligned
+ *     (FLOP_ERR_UNSUPPORTED otherwise).  FLOP_F32 computes in fp32 FMA.
+ *   - Errors are return codes.  Arguments are checked on the host before
+ *     anything is launched.  A device-side wait that runs out (a pipeline
+ *     barrier that never completes) makes the kernel stop cleanly and record
+ *     FLOP_ERR_TIMEOUT in a device status word read by flop_device_status().
+ *   - Sizes of zero (T == 0, r == 0, k == 0, n == 0) are legal: outputs that
+ *     exist are zero-filled where the mathematics says so, nothing else runs.
+ */
+#ifndef FLOP_H_
+#define FLOP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FLOP_OK = 0,
+  FLOP_ERR_INVALID_ARG = 1, /* null pointer, negative size, ld too small, bad enum          */
+  FLOP_ERR_UNSUPPORTED = 2, /* alignment / leading-dimension / size limit of the kernels   */
+  FLOP_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than flop_workspace_bytes */
+  FLOP_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed                           */
+  FLOP_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up                          */
+} flop_status_t;
+
+typedef enum { FLOP_F32 = 0, FLOP_BF16 = 1 } flop_dtype_t;
+
+/* Hard-concrete constants: temperature beta > 0 and stretch limits
+ * gamma < 0 < 1 < zeta (the paper's l and r, Section 3; its formulas are the
+ * beta = 1 case). */
+typedef struct {
+  float beta, gamma, zeta;
+} flop_hc_params_t;
+
+typedef enum {
+  FLOP_OP_FWD = 0,         /* flop_gated_lowrank_fwd                   */
+  FLOP_OP_BWD = 1,         /* flop_gated_lowrank_bwd                   */
+  FLOP_OP_L0 = 2,          /* flop_expected_l0_lagrangian (T = gates n, r = n_seg) */
+  FLOP_OP_COMPACT = 3,     /* flop_compact_ranks                       */
+  FLOP_OP_COMPACT_FWD = 4  /* flop_compact_fwd (r = k)                 */
+} flop_op_t;
+
+const char* flop_status_string(int status);
+
+/* Synchronises `stream`, returns the device status word (FLOP_OK or
+ * FLOP_ERR_TIMEOUT) and clears it. */
+int flop_device_status(void* stream);
+
+/* Bytes of scratch the given call needs (HOST out pointer).  For FLOP_OP_L0
+ * pass the total number of gates as T and the number of segments as r. */
+int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt,
+                         size_t* out_bytes);
+
+/* Gate sampling (Section 3, the inverse CDF G(u; alpha) of the hard-concrete
+ * distribution), for gates j = 0..n-1:
+ *     u_j   = ((x_j >> 9) + 1/2) 2^-23, x_j = word (j mod 4) of the Philox4x32-10
+ *             block with counter (offset + j/4) and key `seed`
+ *     s     = sigmoid((log u - log(1-u) + log_alpha) / beta)
+ *     s_bar = s (zeta - gamma) + gamma,   z = min(1, max(0, s_bar))
+ *     mask  = (z > 0),   dz_dla = dz/dlog_alpha (0 on the clamps)
+ * Outputs z[n] f32, mask[n] u8 (nullable), dz_dla[n] f32 (nullable).  The
+ * mask decision is taken in fp64 whenever fp32 could not decide it safely, so
+ * it equals the fp64 evaluation of the formulas above. */
+int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed,
+                     uint64_t offset, float* z, uint8_t* mask, float* dz_dla, void* stream);
+
+/* Forward of the gated factorized layer (Section 4.1):
+ *     H' = (X Q^T) * z   (column k times z_k, applied in the first GEMM's epilogue)
+ *     Y  = H' P^T
+ * H_save[T, r] (ld ldh) receives H' for the backward pass; it may be NULL
+ * (inference), then H' lives in ws.  z is f32[r]. */
+int flop_gated_lowrank_fwd(const void* X, int64_t ldx, const void* Q, int64_t ldq, const void* P,
+                           int64_t ldp, const float* z, void* Y, int64_t ldy, void* H_save,
+                           int64_t ldh, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt,
+                           void* ws, size_t ws_bytes, void* stream);
+
+/* Backward (chain rule through Section 4.1's product; Section 3 notes that
+ * theta and alpha both receive gradients):
+ *     dH' = dY P            dP = dY^T H'          dQ = diag(z) (dH'^T X)
+ *     dz_k = <Q[k,:], (dH'^T X)[k,:]>  (= sum_t H[t,k] dH'[t,k])
+ *     dX  = dH' (diag(z) Q)                dlog_alpha = dz * dz_dla
+ * H_save is the H' written by the forward call.  dX has type dt; dP, dQ have
+ * type wgrad_dt; dlog_alpha is f32[r].  Any of dX, dP, dQ, dlog_alpha may be
+ * NULL (skipped).  accumulate != 0 adds into dP, dQ and dlog_alpha instead of
+ * overwriting them (dX is always overwritten). */
+int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t ldx, const void* Q,
+                           int64_t ldq, const void* P, int64_t ldp, const float* z,
+                           const float* dz_dla, const void* H_save, int64_t ldh, void* dX,
+                           int64_t lddx, void* dP, int64_t lddp, void* dQ, int64_t lddq,
+                           float* dlog_alpha, int accumulate, int64_t T, int64_t d_in,
+                           int64_t d_out, int64_t r, int dt, int wgrad_dt, void* ws,
+                           size_t ws_bytes, void* stream);
+
+/* Expected size and augmented-Lagrangian penalty over all gates of all
+ * matrices at once (Eq. 3 and Section 4.3).  Segment i (one weight matrix)
+ * owns gates seg_off[i]..seg_off[i+1]-1 of log_alpha; each of its gates
+ * stands for seg_size[i] = d_in + d_out parameters.
+ *     pi_j = sigmoid(log_alpha_j - beta log(-gamma/zeta))
+ *     s = sum_j pi_j size_j / sum_j size_j,   g = lambda1 (s - t) + lambda2 (s - t)^2
+ * out4 = {s, g, dg/dlambda1, dg/dlambda2}; seg_expected[n_seg] (nullable) =
+ * sum of pi_j per segment; dlog_alpha[n] (nullable) += dg/dlog_alpha.
+ * n is the total number of gates (= seg_off[n_seg]).  target[1] and
+ * lambda[2] are DEVICE pointers so that an optimiser can update them on the
+ * device.  n_seg <= 4096. */
+int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t* seg_off,
+                                const float* seg_size, int32_t n_seg, flop_hc_params_t hc,
+                                const float* target, const float* lambda, float* out4,
+                                float* seg_expected, float* dlog_alpha, void* ws, size_t ws_bytes,
+                                void* stream);
+
+/* Deterministic gates and compaction of one weight matrix (Sections 4.4, 4.1).
+ * mode 0: log_alpha_or_z holds log_alpha; k = floor(sum_j pi_j + 1/2); the k
+ *         gates with the largest log_alpha are kept (ties: lower index) with
+ *         value pi_j, the rest are 0.
+ * mode 1: log_alpha_or_z holds a gate vector z; component j is kept iff z_j > 0.
+ * Writes idx[r] (first k entries valid, ascending), k_dev[1], z_det[r]
+ * (nullable) and, when P/Q/Pc/Qc are given (all or none),
+ *     Pc[d_out, k] = P[:, idx]          (ld ldpc >= max k the caller allows, e.g. r)
+ *     Qc[k, d_in]  = diag(z[idx]) Q[idx, :]   (the gate is absorbed into Q)
+ * Columns >= k of Pc and rows >= k of Qc are left untouched.  r <= 65536. */
+int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t hc, int64_t r,
+                       const void* P, int64_t ldp, const void* Q, int64_t ldq, int64_t d_in,
+                       int64_t d_out, int dt, int32_t* idx, int32_t* k_dev, float* z_det, void* Pc,
+                       int64_t ldpc, void* Qc, int64_t ldqc, void* ws, size_t ws_bytes,
+                       void* stream);
+
+/* Inference forward on compact factors (Section 4.1: "simple matrix
+ * multiplications"): Y = (X Qc^T) Pc^T with k surviving components, k known
+ * on the host (read k_dev once after flop_compact_ranks). */
+int flop_compact_fwd(const void* X, int64_t ldx, const void* Qc, int64_t ldqc, const void* Pc,
+                     int64_t ldpc, void* Y, int64_t ldy, int64_t T, int64_t d_in, int64_t d_out,
+                     int64_t k, int dt, void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLOP_H_ */

@@ -1,0 +1,181 @@
+"""Thin ctypes binding over the C ABI in include/flop.h.
+
+Argument marshalling only: torch tensors provide device memory and the
+current CUDA stream; every step of the path runs in the library's kernels.
+If the library is missing or a call fails this module raises -- there is no
+CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libflop_b200.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+F32, BF16 = 0, 1
+OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
+
+EXPORTS = ("flop_status_string", "flop_device_status", "flop_workspace_bytes", "flop_gate_sample",
+           "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_expected_l0_lagrangian",
+           "flop_compact_ranks", "flop_compact_fwd")
+
+
+class HcParams(ctypes.Structure):
+    _fields_ = [("beta", ctypes.c_float), ("gamma", ctypes.c_float), ("zeta", ctypes.c_float)]
+
+
+class FlopError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_1910_04732_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i64, vp, sz, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+    lib.flop_status_string.restype = ctypes.c_char_p
+    lib.flop_status_string.argtypes = [ci]
+    lib.flop_device_status.argtypes = [vp]
+    lib.flop_workspace_bytes.argtypes = [ci, i64, i64, i64, i64, ci, ctypes.POINTER(sz)]
+    lib.flop_gate_sample.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
+    lib.flop_gated_lowrank_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
+                                           i64, i64, i64, i64, ci, vp, sz, vp]
+    lib.flop_gated_lowrank_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, i64,
+                                           vp, i64, vp, i64, vp, i64, vp, ci,
+                                           i64, i64, i64, i64, ci, ci, vp, sz, vp]
+    lib.flop_expected_l0_lagrangian.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp,
+                                                vp, sz, vp]
+    lib.flop_compact_ranks.argtypes = [vp, ci, HcParams, i64, vp, i64, vp, i64, i64, i64, ci,
+                                       vp, vp, vp, vp, i64, vp, i64, vp, sz, vp]
+    lib.flop_compact_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, i64, i64, i64, i64, ci, vp, sz, vp]
+    for name in EXPORTS[1:]:
+        getattr(lib, name).restype = ci
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().flop_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise FlopError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ld(t: torch.Tensor) -> int:
+    assert t.dim() == 2 and t.stride(1) == 1, "matrices must be row-major with unit column stride"
+    return t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def _hc(hc) -> HcParams:
+    return HcParams(float(hc[0]), float(hc[1]), float(hc[2]))
+
+
+def workspace_bytes(op: int, T: int, d_in: int, d_out: int, r: int, dt: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().flop_workspace_bytes(op, T, d_in, d_out, r, dt, ctypes.byref(out)), "flop_workspace_bytes")
+    return int(out.value)
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A 256-byte aligned scratch buffer (torch's caching allocator aligns to 512)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def device_status() -> int:
+    return int(load_library().flop_device_status(_stream()))
+
+
+def padded(rows: int, cols: int, dtype, device="cuda", multiple: int = 8) -> torch.Tensor:
+    """A [rows, cols] view whose leading dimension is rounded up to `multiple`
+    elements (bf16 operands need 16-byte aligned rows)."""
+    ld = (cols + multiple - 1) // multiple * multiple
+    return torch.zeros(rows, max(ld, multiple), dtype=dtype, device=device)[:, :cols]
+
+
+def gate_sample(log_alpha: torch.Tensor, hc, seed: int, offset: int, z: torch.Tensor,
+                mask: Optional[torch.Tensor] = None, dz_dla: Optional[torch.Tensor] = None) -> None:
+    n = log_alpha.numel()
+    _check(load_library().flop_gate_sample(_ptr(log_alpha), n, _hc(hc), seed, offset, _ptr(z), _ptr(mask),
+                                           _ptr(dz_dla), _stream()), "flop_gate_sample")
+
+
+def gated_lowrank_fwd(X, Q, P, z, Y, H_save=None, ws=None) -> None:
+    T, d_in = X.shape
+    d_out, r = P.shape
+    _check(load_library().flop_gated_lowrank_fwd(
+        _ptr(X), _ld(X), _ptr(Q), _ld(Q), _ptr(P), _ld(P), _ptr(z), _ptr(Y), _ld(Y),
+        _ptr(H_save), _ld(H_save) if H_save is not None else 0, T, d_in, d_out, r, _dt(X),
+        _ptr(ws), ws.numel() if ws is not None else 0, _stream()), "flop_gated_lowrank_fwd")
+
+
+def gated_lowrank_bwd(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws, accumulate: bool = False) -> None:
+    T, d_in = X.shape
+    d_out, r = P.shape
+    wdt = _dt(dP) if dP is not None else (_dt(dQ) if dQ is not None else _dt(X))
+    _check(load_library().flop_gated_lowrank_bwd(
+        _ptr(dY), _ld(dY), _ptr(X), _ld(X), _ptr(Q), _ld(Q), _ptr(P), _ld(P), _ptr(z), _ptr(dz_dla),
+        _ptr(H_save), _ld(H_save),
+        _ptr(dX), _ld(dX) if dX is not None else 0, _ptr(dP), _ld(dP) if dP is not None else 0,
+        _ptr(dQ), _ld(dQ) if dQ is not None else 0, _ptr(dlog_alpha), int(accumulate),
+        T, d_in, d_out, r, _dt(X), wdt, _ptr(ws), ws.numel() if ws is not None else 0, _stream()),
+        "flop_gated_lowrank_bwd")
+
+
+def expected_l0_lagrangian(log_alpha, seg_off, seg_size, hc, target, lam, out4, seg_expected=None,
+                           dlog_alpha=None, ws=None) -> None:
+    _check(load_library().flop_expected_l0_lagrangian(
+        _ptr(log_alpha), log_alpha.numel(), _ptr(seg_off), _ptr(seg_size), seg_size.numel(), _hc(hc),
+        _ptr(target), _ptr(lam), _ptr(out4), _ptr(seg_expected), _ptr(dlog_alpha),
+        _ptr(ws), ws.numel() if ws is not None else 0, _stream()), "flop_expected_l0_lagrangian")
+
+
+def compact_ranks(log_alpha_or_z, mode: int, hc, idx, k_dev, z_det=None, P=None, Q=None, Pc=None, Qc=None) -> None:
+    r = log_alpha_or_z.numel()
+    d_in = Q.shape[1] if Q is not None else 0
+    d_out = P.shape[0] if P is not None else 0
+    dt = _dt(P) if P is not None else F32
+    _check(load_library().flop_compact_ranks(
+        _ptr(log_alpha_or_z), mode, _hc(hc), r, _ptr(P), _ld(P) if P is not None else 0,
+        _ptr(Q), _ld(Q) if Q is not None else 0, d_in, d_out, dt, _ptr(idx), _ptr(k_dev), _ptr(z_det),
+        _ptr(Pc), _ld(Pc) if Pc is not None else 0, _ptr(Qc), _ld(Qc) if Qc is not None else 0,
+        None, 0, _stream()), "flop_compact_ranks")
+
+
+def compact_fwd(X, Qc, Pc, Y, k: int, ws) -> None:
+    T, d_in = X.shape
+    d_out = Pc.shape[0]
+    _check(load_library().flop_compact_fwd(
+        _ptr(X), _ld(X), _ptr(Qc), _ld(Qc), _ptr(Pc), _ld(Pc), _ptr(Y), _ld(Y), T, d_in, d_out, k, _dt(X),
+        _ptr(ws), ws.numel() if ws is not None else 0, _stream()), "flop_compact_fwd")

@@ -1,0 +1,611 @@
+// C ABI of the FLOP hot path (see include/flop.h): argument checks, workspace
+// planning, tensor-map creation and kernel launches.  Single translation unit;
+// the kernels live in the .cuh files next to it.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
+#include <mutex>
+
+#include "../../include/flop.h"
+#include "common.cuh"
+#include "compact.cuh"
+#include "gate_sample.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "l0_lagrangian.cuh"
+#include "wgrad.cuh"
+
+using namespace flop;
+typedef __nv_bfloat16 bf16;
+
+namespace {
+
+#define FLOP_CUDA(expr)                           \
+  do {                                            \
+    cudaError_t e__ = (expr);                     \
+    if (e__ != cudaSuccess) return FLOP_ERR_CUDA; \
+  } while (0)
+#define FLOP_TRY(expr)              \
+  do {                              \
+    int s__ = (expr);               \
+    if (s__ != FLOP_OK) return s__; \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline bool valid_dt(int dt) { return dt == FLOP_F32 || dt == FLOP_BF16; }
+inline size_t elt(int dt) { return dt == FLOP_BF16 ? 2 : 4; }
+inline bool valid_hc(const flop_hc_params_t& hc) { return hc.beta > 0.f && hc.gamma < 0.f && hc.zeta > 1.f; }
+
+int num_sms() {
+  static int cached = 0;
+  if (cached) return cached;
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return 148;   // B200; used only for planning when no device is visible
+  }
+  cached = n;
+  return n;
+}
+
+// ------------------------------------------------------------------ bump allocator over ws
+struct Arena {
+  unsigned char* base;
+  size_t size, used;
+  void* take(size_t bytes) {
+    const size_t off = align_up(used, 256);
+    used = off + bytes;
+    return base ? base + off : nullptr;
+  }
+};
+
+// ------------------------------------------------------------------ tensor-core GEMM planning
+struct TcPlan {
+  int bn, stages, tiles_m, tiles_n, splits, kb_per_split, num_kb;
+};
+
+constexpr int kSmemBudget = 227 * 1024;
+constexpr int kSmemBarrierBytes = 8 * (2 * tc::kMaxStages + 4);
+
+// Picks the N tile and the split-K factor by a small cost model: waves over the SMs times
+// (k-blocks per work item x the slower of MMA issue and operand fetch, plus the epilogue).
+TcPlan plan_tc(int64_t M, int64_t N, int64_t K, bool allow_split) {
+  const int sms = num_sms();
+  const int num_kb = (int)((K + tc::BK - 1) / tc::BK);
+  TcPlan best{};
+  double best_cost = 1e300;
+  const int bns[4] = {256, 192, 128, 64};
+  for (int bi = 0; bi < 4; ++bi) {
+    const int bn = bns[bi];
+    if (bn > 64 && bn - 64 >= N) continue;   // a smaller tile already covers N
+    const int tiles_m = (int)((M + tc::BM - 1) / tc::BM), tiles_n = (int)((N + bn - 1) / bn);
+    const int max_split = allow_split ? std::min(num_kb, 32) : 1;
+    for (int s = 1; s <= max_split; ++s) {
+      const int kbps = (num_kb + s - 1) / s;
+      const int splits = (num_kb + kbps - 1) / kbps;
+      if (splits != s) continue;
+      const double items = (double)tiles_m * tiles_n * splits;
+      const double waves = ceil(items / sms);
+      const double mma = 2.0 * bn;                                  // cycles per k-block at full rate
+      const double fetch = (double)tc::stage_bytes(bn) / 80.0;      // cycles per k-block at ~80 B/clk/SM
+      const double epi = 600.0 + 10.0 * bn;
+      double cost = waves * (kbps * std::max(mma, fetch) + epi);
+      if (splits > 1) cost += 0.002 * (double)splits * (double)M * (double)N / sms + 3000.0;   // ordered reduction pass
+      if (cost < best_cost) {
+        best_cost = cost;
+        best.bn = bn; best.tiles_m = tiles_m; best.tiles_n = tiles_n;
+        best.splits = splits; best.kb_per_split = kbps; best.num_kb = num_kb;
+      }
+    }
+  }
+  const int sb = (int)tc::stage_bytes(best.bn);
+  best.stages = std::min(tc::kMaxStages, (kSmemBudget - 1024 - kSmemBarrierBytes) / sb);
+  return best;
+}
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  });
+  return fn;
+}
+
+// Row-major bf16 matrix [rows, cols] with leading dimension ld; box = box_cols x box_rows, 128-byte swizzle.
+int make_tmap(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return FLOP_ERR_CUDA;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FLOP_OK : FLOP_ERR_CUDA;
+}
+
+// Operand of D = sum_k A(m,k) B(n,k) taken from a row-major matrix.
+struct Operand {
+  const void* ptr;
+  int64_t ld;
+  bool mn_major;   // false: memory is [MN rows, K cols]; true: memory is [K rows, MN cols]
+};
+
+struct TcEpilogue {
+  int kind;   // tc::EPI_STORE or tc::EPI_SLICE
+  bf16* out; int64_t ldo; const float* col_scale;
+  float* slices; int64_t slice_elems, ld_slice;
+  const bf16* qdot; int64_t ldq; float* dz_part; int64_t dz_stride;
+};
+
+template <bool A_MN, bool B_MN, int EPI>
+int launch_tc_inst(const CUtensorMap& ta, const CUtensorMap& tb, const tc::Params& p, cudaStream_t st) {
+  static bool configured = false;
+  auto kern = tc::gemm_kernel<A_MN, B_MN, EPI>;
+  if (!configured) {
+    FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    configured = true;
+  }
+  const int smem = 1024 + p.stages * (int)tc::stage_bytes(p.bn) + kSmemBarrierBytes;
+  const int total = p.tiles_m * p.tiles_n * p.splits;
+  const int grid = std::min(total, num_sms());
+  kern<<<grid, tc::kThreads, smem, st>>>(ta, tb, p);
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+int launch_tc(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, const TcPlan& pl,
+              const TcEpilogue& ep, cudaStream_t st) {
+  if (M <= 0 || N <= 0 || K <= 0) return FLOP_OK;
+  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  CUtensorMap ta, tb;
+  if (!A.mn_major) FLOP_TRY(make_tmap(&ta, A.ptr, M, K, A.ld, tc::BK, tc::BM));
+  else             FLOP_TRY(make_tmap(&ta, A.ptr, K, M, A.ld, tc::kBoxMN, tc::BK));
+  if (!B.mn_major) FLOP_TRY(make_tmap(&tb, B.ptr, N, K, B.ld, tc::BK, (uint32_t)pl.bn));
+  else             FLOP_TRY(make_tmap(&tb, B.ptr, K, N, B.ld, tc::kBoxMN, tc::BK));
+  tc::Params p{};
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.bn = pl.bn; p.stages = pl.stages; p.tiles_m = pl.tiles_m; p.tiles_n = pl.tiles_n;
+  p.splits = pl.splits; p.kb_per_split = pl.kb_per_split; p.num_kb = pl.num_kb;
+  p.out = ep.out; p.ldo = ep.ldo; p.col_scale = ep.col_scale;
+  p.slices = ep.slices; p.slice_elems = ep.slice_elems; p.ld_slice = ep.ld_slice;
+  p.qdot = ep.qdot; p.ldq = ep.ldq; p.dz_part = ep.dz_part; p.dz_stride = ep.dz_stride;
+  if (!A.mn_major && !B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, false, tc::EPI_STORE>(ta, tb, p, st);
+  if (!A.mn_major && B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, true, tc::EPI_STORE>(ta, tb, p, st);
+  if (A.mn_major && B.mn_major && ep.kind == tc::EPI_SLICE) return launch_tc_inst<true, true, tc::EPI_SLICE>(ta, tb, p, st);
+  return FLOP_ERR_UNSUPPORTED;
+}
+
+TcEpilogue store_epilogue(void* out, int64_t ldo, const float* col_scale) {
+  TcEpilogue e{};
+  e.kind = tc::EPI_STORE; e.out = (bf16*)out; e.ldo = ldo; e.col_scale = col_scale;
+  return e;
+}
+
+int launch_simt(const float* A, int64_t a_sm, int64_t a_sk, const float* B, int64_t b_sn, int64_t b_sk, float* C,
+                int64_t ldc, int64_t M, int64_t N, int64_t K, const float* col_scale, const float* row_scale,
+                int accumulate, cudaStream_t st) {
+  if (M <= 0 || N <= 0) return FLOP_OK;
+  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  SimtGemmArgs a{A, a_sm, a_sk, B, b_sn, b_sk, C, ldc, (int)M, (int)N, (int)K, col_scale, row_scale, accumulate};
+  const dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64));
+  if (grid.y > 65535) return FLOP_ERR_UNSUPPORTED;
+  simt_gemm_kernel<<<grid, 256, 0, st>>>(a);
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+template <typename T>
+int zero_2d(void* out, int64_t ld, int64_t rows, int64_t cols, cudaStream_t st) {
+  if (!out || rows <= 0 || cols <= 0) return FLOP_OK;
+  const int64_t n = rows * cols;
+  fill_zero_2d_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((T*)out, ld, (int)rows, (int)cols);
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+bool check_mat(const void* p, int64_t ld, int64_t cols) { return p != nullptr && ld >= cols; }
+bool bf16_ok(const void* p, int64_t ld) { return aligned16(p) && (ld % 8) == 0; }
+
+// Workspace layouts (shared by the size query and the calls).
+struct FwdWs { void* H; int64_t ldh; size_t bytes; };
+FwdWs plan_fwd_ws(Arena& ar, int64_t T, int64_t r, int dt) {
+  FwdWs w{};
+  w.ldh = round_up(std::max<int64_t>(r, 1), 8);
+  w.H = ar.take((size_t)T * w.ldh * elt(dt));
+  w.bytes = ar.used;
+  return w;
+}
+
+struct BwdWs {
+  void* dH; int64_t lddh;        // dH'[T, r]
+  void* Qz; int64_t ldqz;        // diag(z) Q [r, d_in]
+  float* slices; int64_t ld_slice_p, ld_slice_q, slice_elems_p, slice_elems_q;
+  float* dz_part; int n_part;
+  TcPlan plan_p, plan_q;
+  size_t bytes;
+};
+BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt) {
+  BwdWs w{};
+  w.lddh = round_up(std::max<int64_t>(r, 1), 8);
+  w.dH = ar.take((size_t)T * w.lddh * elt(dt));
+  w.ldqz = round_up(std::max<int64_t>(d_in, 1), 8);
+  w.Qz = ar.take((size_t)r * w.ldqz * elt(dt));
+  w.ld_slice_p = round_up(std::max<int64_t>(r, 1), 4);
+  w.ld_slice_q = round_up(std::max<int64_t>(d_in, 1), 4);
+  int sp = 1, sq = 1;
+  w.n_part = 1;
+  if (dt == FLOP_BF16) {
+    w.plan_p = plan_tc(d_out, r, T, true);
+    w.plan_q = plan_tc(r, d_in, T, true);
+    sp = std::max(1, w.plan_p.splits);
+    sq = std::max(1, w.plan_q.splits);
+    w.n_part = sq * std::max(1, w.plan_q.tiles_n);
+  }
+  w.slice_elems_p = d_out * w.ld_slice_p;
+  w.slice_elems_q = r * w.ld_slice_q;
+  const size_t slice_bytes = std::max((size_t)sp * w.slice_elems_p, (size_t)sq * w.slice_elems_q) * 4;
+  w.slices = (float*)ar.take(slice_bytes);
+  w.dz_part = (float*)ar.take((size_t)w.n_part * std::max<int64_t>(r, 1) * 4);
+  w.bytes = ar.used;
+  return w;
+}
+
+size_t l0_ws_bytes(int64_t n, int64_t n_seg) {
+  const int64_t chunks = (n + kL0Chunk - 1) / kL0Chunk + n_seg;
+  return sizeof(L0Scratch) + (size_t)std::max<int64_t>(chunks, 1) * sizeof(double);
+}
+
+int check_ws(const void* ws, size_t ws_bytes, size_t need) {
+  if (need == 0) return FLOP_OK;
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || ws_bytes < need) return FLOP_ERR_WORKSPACE;
+  return FLOP_OK;
+}
+
+}  // namespace
+
+template <typename TW, typename TQ>
+static int finalize_wgrad(const float* slices, int n_slices, int64_t slice_elems, int64_t ld_slice, int64_t M, int64_t N,
+                          const float* row_scale, void* out, int64_t ldo, int accumulate, const void* qdot, int64_t ldq,
+                          float* dz_out, cudaStream_t st) {
+  if (M <= 0) return FLOP_OK;
+  wgrad_finalize_kernel<TW, TQ><<<(unsigned)M, 256, 0, st>>>(slices, n_slices, slice_elems, ld_slice, (int)M, (int)N, row_scale,
+                                                            (TW*)out, ldo, accumulate, (const TQ*)qdot, ldq, dz_out);
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+// ====================================================================== C ABI
+extern "C" {
+
+const char* flop_status_string(int status) {
+  switch (status) {
+    case FLOP_OK: return "ok";
+    case FLOP_ERR_INVALID_ARG: return "invalid argument";
+    case FLOP_ERR_UNSUPPORTED: return "unsupported shape, alignment or size";
+    case FLOP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case FLOP_ERR_CUDA: return "CUDA call failed";
+    case FLOP_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int flop_device_status(void* stream) {
+  FLOP_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  int v = 0;
+  FLOP_CUDA(cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)));
+  if (v != 0) {
+    const int zero = 0;
+    FLOP_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)));
+  }
+  return v;
+}
+
+int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt, size_t* out_bytes) {
+  if (!out_bytes || T < 0 || d_in < 0 || d_out < 0 || r < 0 || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  Arena ar{nullptr, 0, 0};
+  switch (op) {
+    case FLOP_OP_FWD:
+    case FLOP_OP_COMPACT_FWD: plan_fwd_ws(ar, T, r, dt); break;
+    case FLOP_OP_BWD: plan_bwd_ws(ar, T, d_in, d_out, r, dt); break;
+    case FLOP_OP_L0: ar.used = l0_ws_bytes(T, r); break;
+    case FLOP_OP_COMPACT: ar.used = 0; break;
+    default: return FLOP_ERR_INVALID_ARG;
+  }
+  *out_bytes = align_up(ar.used, 256);
+  return FLOP_OK;
+}
+
+int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed, uint64_t offset, float* z,
+                     uint8_t* mask, float* dz_dla, void* stream) {
+  if (n < 0 || !valid_hc(hc)) return FLOP_ERR_INVALID_ARG;
+  if (n == 0) return FLOP_OK;
+  if (!log_alpha || !z) return FLOP_ERR_INVALID_ARG;
+  GateConsts g;
+  g.beta_d = (double)hc.beta; g.gamma_d = (double)hc.gamma; g.zeta_d = (double)hc.zeta;
+  g.inv_beta = (float)(1.0 / g.beta_d); g.gamma = hc.gamma; g.zeta = hc.zeta;
+  g.c0 = (float)(g.beta_d * log(-g.gamma_d / g.zeta_d));
+  g.c1 = (float)(g.beta_d * log((1.0 - g.gamma_d) / (g.zeta_d - 1.0)));
+  const int vec_ok = aligned16(log_alpha) && aligned16(z) && (!dz_dla || aligned16(dz_dla)) &&
+                     (!mask || (reinterpret_cast<uintptr_t>(mask) & 3) == 0);
+  const int64_t nblk = (n + 3) / 4;
+  const int64_t want = (nblk + 255) / 256;
+  const int grid = (int)std::min<int64_t>(want, (int64_t)num_sms() * 16);
+  gate_sample_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(log_alpha, n, g, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)),
+                                                             offset, z, mask, dz_dla, vec_ok);
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+static int fwd_impl(const void* X, int64_t ldx, const void* Q, int64_t ldq, const void* P, int64_t ldp, const float* z,
+                    void* Y, int64_t ldy, void* H, int64_t ldh, int64_t T, int64_t d_in, int64_t d_out, int64_t r,
+                    int dt, cudaStream_t st) {
+  if (dt == FLOP_BF16) {
+    if (r == 0 || d_in == 0) {
+      FLOP_TRY(zero_2d<bf16>(Y, ldy, T, d_out, st));
+      if (r > 0) FLOP_TRY(zero_2d<bf16>(H, ldh, T, r, st));
+      return FLOP_OK;
+    }
+    // GEMM1: H' = (X Q^T) * z, gate applied to column k in the epilogue
+    const TcPlan p1 = plan_tc(T, r, d_in, false);
+    FLOP_TRY(launch_tc({X, ldx, false}, {Q, ldq, false}, T, r, d_in, p1, store_epilogue(H, ldh, z), st));
+    // GEMM2: Y = H' P^T
+    const TcPlan p2 = plan_tc(T, d_out, r, false);
+    FLOP_TRY(launch_tc({H, ldh, false}, {P, ldp, false}, T, d_out, r, p2, store_epilogue(Y, ldy, nullptr), st));
+  } else {
+    FLOP_TRY(launch_simt((const float*)X, ldx, 1, (const float*)Q, ldq, 1, (float*)H, ldh, T, r, d_in, z, nullptr, 0, st));
+    FLOP_TRY(launch_simt((const float*)H, ldh, 1, (const float*)P, ldp, 1, (float*)Y, ldy, T, d_out, r, nullptr, nullptr, 0, st));
+  }
+  return FLOP_OK;
+}
+
+int flop_gated_lowrank_fwd(const void* X, int64_t ldx, const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                           const float* z, void* Y, int64_t ldy, void* H_save, int64_t ldh, int64_t T, int64_t d_in,
+                           int64_t d_out, int64_t r, int dt, void* ws, size_t ws_bytes, void* stream) {
+  if (T < 0 || d_in < 0 || d_out < 0 || r < 0 || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  if (T == 0 || d_out == 0) return FLOP_OK;
+  if (!check_mat(Y, ldy, d_out)) return FLOP_ERR_INVALID_ARG;
+  if (r > 0 && (!z || !check_mat(P, ldp, r))) return FLOP_ERR_INVALID_ARG;
+  if (r > 0 && d_in > 0 && (!check_mat(X, ldx, d_in) || !check_mat(Q, ldq, d_in))) return FLOP_ERR_INVALID_ARG;
+  if (H_save && ldh < r) return FLOP_ERR_INVALID_ARG;
+  void* H = H_save;
+  if (!H && r > 0) {
+    Arena ar{(unsigned char*)ws, ws_bytes, 0};
+    Arena probe{nullptr, 0, 0};
+    const size_t need = plan_fwd_ws(probe, T, r, dt).bytes;
+    FLOP_TRY(check_ws(ws, ws_bytes, need));
+    const FwdWs w = plan_fwd_ws(ar, T, r, dt);
+    H = w.H; ldh = w.ldh;
+  }
+  if (dt == FLOP_BF16) {
+    if (!bf16_ok(Y, ldy) || (r > 0 && (!bf16_ok(P, ldp) || !bf16_ok(H, ldh))) ||
+        (r > 0 && d_in > 0 && (!bf16_ok(X, ldx) || !bf16_ok(Q, ldq))))
+      return FLOP_ERR_UNSUPPORTED;
+  }
+  return fwd_impl(X, ldx, Q, ldq, P, ldp, z, Y, ldy, H, ldh, T, d_in, d_out, r, dt, (cudaStream_t)stream);
+}
+
+int flop_compact_fwd(const void* X, int64_t ldx, const void* Qc, int64_t ldqc, const void* Pc, int64_t ldpc, void* Y,
+                     int64_t ldy, int64_t T, int64_t d_in, int64_t d_out, int64_t k, int dt, void* ws, size_t ws_bytes,
+                     void* stream) {
+  if (T < 0 || d_in < 0 || d_out < 0 || k < 0 || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  if (T == 0 || d_out == 0) return FLOP_OK;
+  if (!check_mat(Y, ldy, d_out)) return FLOP_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (k == 0 || d_in == 0) {
+    if (dt == FLOP_BF16) { if (!bf16_ok(Y, ldy)) return FLOP_ERR_UNSUPPORTED; return zero_2d<bf16>(Y, ldy, T, d_out, st); }
+    return zero_2d<float>(Y, ldy, T, d_out, st);
+  }
+  if (!check_mat(X, ldx, d_in) || !check_mat(Qc, ldqc, d_in) || !check_mat(Pc, ldpc, k)) return FLOP_ERR_INVALID_ARG;
+  Arena probe{nullptr, 0, 0};
+  FLOP_TRY(check_ws(ws, ws_bytes, plan_fwd_ws(probe, T, k, dt).bytes));
+  Arena ar{(unsigned char*)ws, ws_bytes, 0};
+  const FwdWs w = plan_fwd_ws(ar, T, k, dt);
+  if (dt == FLOP_BF16) {
+    if (!bf16_ok(Y, ldy) || !bf16_ok(X, ldx) || !bf16_ok(Qc, ldqc) || !bf16_ok(Pc, ldpc)) return FLOP_ERR_UNSUPPORTED;
+    const TcPlan p1 = plan_tc(T, k, d_in, false);
+    FLOP_TRY(launch_tc({X, ldx, false}, {Qc, ldqc, false}, T, k, d_in, p1, store_epilogue(w.H, w.ldh, nullptr), st));
+    const TcPlan p2 = plan_tc(T, d_out, k, false);
+    FLOP_TRY(launch_tc({w.H, w.ldh, false}, {Pc, ldpc, false}, T, d_out, k, p2, store_epilogue(Y, ldy, nullptr), st));
+  } else {
+    FLOP_TRY(launch_simt((const float*)X, ldx, 1, (const float*)Qc, ldqc, 1, (float*)w.H, w.ldh, T, k, d_in, nullptr, nullptr, 0, st));
+    FLOP_TRY(launch_simt((const float*)w.H, w.ldh, 1, (const float*)Pc, ldpc, 1, (float*)Y, ldy, T, d_out, k, nullptr, nullptr, 0, st));
+  }
+  return FLOP_OK;
+}
+
+int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t ldx, const void* Q, int64_t ldq,
+                           const void* P, int64_t ldp, const float* z, const float* dz_dla, const void* H_save,
+                           int64_t ldh, void* dX, int64_t lddx, void* dP, int64_t lddp, void* dQ, int64_t lddq,
+                           float* dlog_alpha, int accumulate, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt,
+                           int wgrad_dt, void* ws, size_t ws_bytes, void* stream) {
+  if (T < 0 || d_in < 0 || d_out < 0 || r < 0 || !valid_dt(dt) || !valid_dt(wgrad_dt)) return FLOP_ERR_INVALID_ARG;
+  if (dt == FLOP_F32 && wgrad_dt != FLOP_F32) return FLOP_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dX && lddx < d_in) return FLOP_ERR_INVALID_ARG;
+  if (dP && lddp < r) return FLOP_ERR_INVALID_ARG;
+  if (dQ && lddq < d_in) return FLOP_ERR_INVALID_ARG;
+  if (dlog_alpha && r > 0 && !dz_dla) return FLOP_ERR_INVALID_ARG;
+  const bool degenerate = T == 0 || r == 0 || d_in == 0 || d_out == 0;
+  if (!degenerate) {
+    if (!check_mat(dY, lddy, d_out) || !check_mat(X, ldx, d_in) || !check_mat(Q, ldq, d_in) || !check_mat(P, ldp, r) ||
+        !z || !check_mat(H_save, ldh, r))
+      return FLOP_ERR_INVALID_ARG;
+  }
+  if (dt == FLOP_BF16) {
+    if ((dX && !bf16_ok(dX, lddx)) || (!degenerate && (!bf16_ok(dY, lddy) || !bf16_ok(X, ldx) || !bf16_ok(Q, ldq) ||
+                                                       !bf16_ok(P, ldp) || !bf16_ok(H_save, ldh))))
+      return FLOP_ERR_UNSUPPORTED;
+  }
+  if (degenerate) {
+    // every product is empty: gradients are zero (or unchanged when accumulating)
+    if (dX && T > 0 && d_in > 0) FLOP_TRY(dt == FLOP_BF16 ? zero_2d<bf16>(dX, lddx, T, d_in, st) : zero_2d<float>(dX, lddx, T, d_in, st));
+    if (!accumulate) {
+      if (dP) FLOP_TRY(wgrad_dt == FLOP_BF16 ? zero_2d<bf16>(dP, lddp, d_out, r, st) : zero_2d<float>(dP, lddp, d_out, r, st));
+      if (dQ) FLOP_TRY(wgrad_dt == FLOP_BF16 ? zero_2d<bf16>(dQ, lddq, r, d_in, st) : zero_2d<float>(dQ, lddq, r, d_in, st));
+      if (dlog_alpha) FLOP_TRY(zero_2d<float>(dlog_alpha, r, 1, r, st));
+    }
+    return FLOP_OK;
+  }
+  Arena probe{nullptr, 0, 0};
+  FLOP_TRY(check_ws(ws, ws_bytes, plan_bwd_ws(probe, T, d_in, d_out, r, dt).bytes));
+  Arena ar{(unsigned char*)ws, ws_bytes, 0};
+  const BwdWs w = plan_bwd_ws(ar, T, d_in, d_out, r, dt);
+  const bool need_m = dQ || dlog_alpha;   // M = dH'^T X feeds both dQ and dz
+
+  if (dt == FLOP_BF16) {
+    // dH' = dY P            (A = dY K-major over d_out; B(n=k_rank, k=i) = P[i, k_rank]: MN-major)
+    const TcPlan ph = plan_tc(T, r, d_out, false);
+    FLOP_TRY(launch_tc({dY, lddy, false}, {P, ldp, true}, T, r, d_out, ph, store_epilogue(w.dH, w.lddh, nullptr), st));
+    if (dP) {
+      // dP = dY^T H'        (contract over tokens: both operands MN-major), fp32 split-K slices
+      TcEpilogue e{};
+      e.kind = tc::EPI_SLICE; e.slices = w.slices; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
+      FLOP_TRY(launch_tc({dY, lddy, true}, {H_save, ldh, true}, d_out, r, T, w.plan_p, e, st));
+      if (wgrad_dt == FLOP_BF16)
+        FLOP_TRY((finalize_wgrad<bf16, bf16>(w.slices, w.plan_p.splits, w.slice_elems_p, w.ld_slice_p, d_out, r, nullptr, dP, lddp, accumulate, nullptr, 0, nullptr, st)));
+      else
+        FLOP_TRY((finalize_wgrad<float, bf16>(w.slices, w.plan_p.splits, w.slice_elems_p, w.ld_slice_p, d_out, r, nullptr, dP, lddp, accumulate, nullptr, 0, nullptr, st)));
+    }
+    if (need_m) {
+      // M = dH'^T X; dQ = diag(z) M; dz_k = <Q[k,:], M[k,:]> fused into the GEMM epilogue per tile
+      TcEpilogue e{};
+      e.kind = tc::EPI_SLICE; e.slices = w.slices; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
+      if (dlog_alpha) { e.qdot = (const bf16*)Q; e.ldq = ldq; e.dz_part = w.dz_part; e.dz_stride = r; }
+      FLOP_TRY(launch_tc({w.dH, w.lddh, true}, {X, ldx, true}, r, d_in, T, w.plan_q, e, st));
+      if (dQ) {
+        if (wgrad_dt == FLOP_BF16)
+          FLOP_TRY((finalize_wgrad<bf16, bf16>(w.slices, w.plan_q.splits, w.slice_elems_q, w.ld_slice_q, r, d_in, z, dQ, lddq, accumulate, nullptr, 0, nullptr, st)));
+        else
+          FLOP_TRY((finalize_wgrad<float, bf16>(w.slices, w.plan_q.splits, w.slice_elems_q, w.ld_slice_q, r, d_in, z, dQ, lddq, accumulate, nullptr, 0, nullptr, st)));
+      }
+      if (dlog_alpha) {
+        dalpha_kernel<<<(unsigned)((r + 255) / 256), 256, 0, st>>>(w.dz_part, w.n_part, r, dz_dla, (int)r, dlog_alpha, accumulate);
+        FLOP_CUDA(cudaGetLastError());
+      }
+    }
+    if (dX) {
+      // dX = dH' (diag(z) Q)   (B(n=j, k=k_rank) = Qz[k_rank, j]: MN-major)
+      scale_rows_kernel<bf16><<<(unsigned)r, 256, 0, st>>>((const bf16*)Q, ldq, z, (int)r, (int)d_in, (bf16*)w.Qz, w.ldqz);
+      FLOP_CUDA(cudaGetLastError());
+      const TcPlan px = plan_tc(T, d_in, r, false);
+      FLOP_TRY(launch_tc({w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, T, d_in, r, px, store_epilogue(dX, lddx, nullptr), st));
+    }
+  } else {
+    const float* dYf = (const float*)dY; const float* Xf = (const float*)X; const float* Qf = (const float*)Q;
+    const float* Pf = (const float*)P; const float* Hf = (const float*)H_save;
+    float* dHf = (float*)w.dH;
+    // dH'[t,k] = sum_i dY[t,i] P[i,k]
+    FLOP_TRY(launch_simt(dYf, lddy, 1, Pf, 1, ldp, dHf, w.lddh, T, r, d_out, nullptr, nullptr, 0, st));
+    // dP[i,k] = sum_t dY[t,i] H'[t,k]
+    if (dP) FLOP_TRY(launch_simt(dYf, 1, lddy, Hf, 1, ldh, (float*)dP, lddp, d_out, r, T, nullptr, nullptr, accumulate, st));
+    if (need_m) {
+      // M[k,j] = sum_t dH'[t,k] X[t,j] into the slice buffer, then the same finalisation as the tensor-core path
+      FLOP_TRY(launch_simt(dHf, 1, w.lddh, Xf, 1, ldx, w.slices, w.ld_slice_q, r, d_in, T, nullptr, nullptr, 0, st));
+      FLOP_TRY((finalize_wgrad<float, float>(w.slices, 1, w.slice_elems_q, w.ld_slice_q, r, d_in, z, dQ, lddq, accumulate,
+                                             dlog_alpha ? Q : nullptr, ldq, w.dz_part, st)));
+      if (dlog_alpha) {
+        dalpha_kernel<<<(unsigned)((r + 255) / 256), 256, 0, st>>>(w.dz_part, 1, r, dz_dla, (int)r, dlog_alpha, accumulate);
+        FLOP_CUDA(cudaGetLastError());
+      }
+    }
+    if (dX) {
+      scale_rows_kernel<float><<<(unsigned)r, 256, 0, st>>>(Qf, ldq, z, (int)r, (int)d_in, (float*)w.Qz, w.ldqz);
+      FLOP_CUDA(cudaGetLastError());
+      // dX[t,j] = sum_k dH'[t,k] Qz[k,j]
+      FLOP_TRY(launch_simt(dHf, w.lddh, 1, (const float*)w.Qz, 1, w.ldqz, (float*)dX, lddx, T, d_in, r, nullptr, nullptr, 0, st));
+    }
+  }
+  return FLOP_OK;
+}
+
+int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t* seg_off, const float* seg_size,
+                                int32_t n_seg, flop_hc_params_t hc, const float* target, const float* lambda,
+                                float* out4, float* seg_expected, float* dlog_alpha, void* ws, size_t ws_bytes,
+                                void* stream) {
+  if (n < 0 || n_seg < 0 || !valid_hc(hc) || !out4 || !target || !lambda) return FLOP_ERR_INVALID_ARG;
+  if (n_seg > kL0MaxSeg) return FLOP_ERR_UNSUPPORTED;
+  if (n_seg > 0 && (!seg_off || !seg_size)) return FLOP_ERR_INVALID_ARG;
+  if (n > 0 && !log_alpha) return FLOP_ERR_INVALID_ARG;
+  const size_t need = l0_ws_bytes(n, n_seg);
+  FLOP_TRY(check_ws(ws, ws_bytes, need));
+  cudaStream_t st = (cudaStream_t)stream;
+  L0Scratch* sc = (L0Scratch*)ws;
+  const float thr = (float)((double)hc.beta * log(-(double)hc.gamma / (double)hc.zeta));
+  const int64_t chunks = (n + kL0Chunk - 1) / kL0Chunk + n_seg;
+  if (chunks > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  if (chunks > 0 && n_seg > 0)
+    l0_chunk_kernel<false><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
+  l0_finalize_kernel<<<1, kL0Threads, 0, st>>>(seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
+  if (dlog_alpha && chunks > 0 && n_seg > 0)
+    l0_chunk_kernel<true><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t hc, int64_t r, const void* P, int64_t ldp,
+                       const void* Q, int64_t ldq, int64_t d_in, int64_t d_out, int dt, int32_t* idx, int32_t* k_dev,
+                       float* z_det, void* Pc, int64_t ldpc, void* Qc, int64_t ldqc, void* ws, size_t ws_bytes,
+                       void* stream) {
+  (void)ws; (void)ws_bytes;
+  if (r < 0 || d_in < 0 || d_out < 0 || (mode != 0 && mode != 1) || !valid_dt(dt) || !k_dev) return FLOP_ERR_INVALID_ARG;
+  if (mode == 0 && !valid_hc(hc)) return FLOP_ERR_INVALID_ARG;
+  if (r > 65536) return FLOP_ERR_UNSUPPORTED;
+  if (r > 0 && (!log_alpha_or_z || !idx)) return FLOP_ERR_INVALID_ARG;
+  const bool gather = P || Q || Pc || Qc;
+  if (gather) {
+    if (!P || !Q || !Pc || !Qc || ldp < r || ldq < d_in || ldqc < d_in) return FLOP_ERR_INVALID_ARG;
+    if (!z_det && mode == 0) return FLOP_ERR_INVALID_ARG;   // the gather scales Q rows by the deterministic gate
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  const double thr = (double)hc.beta * log(-(double)hc.gamma / (double)hc.zeta);
+  compact_select_kernel<<<1, kSelThreads, 0, st>>>(log_alpha_or_z, mode, thr, (int)r, idx, k_dev, z_det);
+  FLOP_CUDA(cudaGetLastError());
+  if (gather && r > 0) {
+    const float* zsrc = z_det ? z_det : log_alpha_or_z;
+    const size_t es = elt(dt);
+    const int vq = aligned16(Q) && aligned16(Qc) && (ldq * es) % 16 == 0 && (ldqc * es) % 16 == 0;
+    const int vp = aligned16(P) && (ldp * es) % 16 == 0;
+    const int rows_per_block = 4;
+    const size_t smem = (size_t)r * es;
+    if (smem > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
+    if (dt == FLOP_BF16) {
+      if (d_in > 0) gather_q_kernel<bf16><<<(unsigned)r, 256, 0, st>>>((const bf16*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (bf16*)Qc, ldqc, vq);
+      if (d_out > 0) {
+        if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(gather_p_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        gather_p_kernel<bf16><<<(unsigned)((d_out + rows_per_block - 1) / rows_per_block), 256, smem, st>>>(
+            (const bf16*)P, ldp, idx, k_dev, (int)r, (int)d_out, (bf16*)Pc, ldpc, rows_per_block, vp);
+      }
+    } else {
+      if (d_in > 0) gather_q_kernel<float><<<(unsigned)r, 256, 0, st>>>((const float*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (float*)Qc, ldqc, vq);
+      if (d_out > 0) {
+        if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(gather_p_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        gather_p_kernel<float><<<(unsigned)((d_out + rows_per_block - 1) / rows_per_block), 256, smem, st>>>(
+            (const float*)P, ldp, idx, k_dev, (int)r, (int)d_out, (float*)Pc, ldpc, rows_per_block, vp);
+      }
+    }
+    FLOP_CUDA(cudaGetLastError());
+  }
+  return FLOP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,383 @@
+// bf16 tensor-core GEMM for sm_100a: D[M,N] = sum_k A(m,k) B(n,k), fp32 accumulate.
+//
+// One persistent, warp-specialised kernel serves all six GEMMs of the gated
+// factorized layer W = P diag(z) Q (Section 4.1 of the paper):
+//   warp 0      TMA producer: cp.async.bulk.tensor (no multicast) into a ring of
+//               128-byte-swizzled shared-memory stages, completion on mbarriers
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (128 x BN x 16, bf16 in,
+//               fp32 accumulators in tensor memory), tcgen05.commit frees stages
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (one output row per thread),
+//               apply the gate / write bf16, or write fp32 split-K slices and the
+//               fused per-row dot product that becomes dz (hence dlog_alpha)
+// Two accumulator buffers in tensor memory let the epilogue of one tile overlap
+// the main loop of the next.  Operands may be K-major (rows of the row-major
+// matrix run along K) or MN-major (the backward GEMMs that contract over tokens
+// or over d_out read the same row-major tensors "transposed"), selected in the
+// shared-memory and instruction descriptors; nothing is transposed in memory.
+// Ragged sizes rely on TMA zero fill for loads and on guarded stores.
+//
+// Every wait on an mbarrier is bounded: if it gives up, the kernel records
+// FLOP_ERR_TIMEOUT, all roles leave their loops, outstanding copies are waited
+// for (bounded), tensor memory is freed and the CTA returns.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace flop {
+namespace tc {
+
+constexpr int BM = 128;          // rows of D per tile = TMEM lanes
+constexpr int BK = 64;           // K per stage = one 128-byte swizzle row of bf16
+constexpr int UMMA_K = 16;
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr uint32_t kATileBytes = BM * BK * 2;     // 16 KB
+constexpr uint32_t kBoxMN = 64;                   // MN-major operands arrive in 64(mn) x 64(k) boxes
+constexpr uint32_t kBoxBytes = kBoxMN * BK * 2;   // 8 KB
+constexpr uint32_t kTmemCols = 512;
+constexpr long long kWaitCycles = 2000000000LL;   // ~1 s
+
+struct Params {
+  int M, N, K;
+  int bn;                 // N per tile: 64, 128, 192 or 256
+  int stages;
+  int tiles_m, tiles_n, splits, kb_per_split, num_kb;
+  // EPI_STORE: out[m*ldo + n] = acc * col_scale[n]  (bf16)
+  __nv_bfloat16* out; int64_t ldo;
+  const float* col_scale;               // nullable
+  // EPI_SLICE: slices[split][m*ld_slice + n] = acc (fp32); optional fused row dot
+  float* slices; int64_t slice_elems; int64_t ld_slice;
+  const __nv_bfloat16* qdot; int64_t ldq;      // nullable: dz_part[(split*tiles_n+tn)*dz_stride + m] = sum_n acc*qdot[m,n]
+  float* dz_part; int64_t dz_stride;
+};
+
+enum { EPI_STORE = 0, EPI_SLICE = 1 };
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (and records the timeout) if the phase never completes
+// or another role has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        report_timeout();
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier receives one arrival once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (tcgen05): start address, leading/stride byte
+// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
+//   K-major tile  (rows of 128 B = 64 bf16 along K): 8-row groups 1024 B apart (SBO); LBO unused.
+//   MN-major tile (rows of 128 B = 64 bf16 along M/N, one row per k): 8-k groups 1024 B apart (SBO),
+//                 successive 64-wide M/N chunks one box (8 KB) apart (LBO).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
+  const uint64_t lbo = mn_major ? (kBoxBytes >> 4) : 1;
+  const uint64_t sbo = 1024 >> 4;
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, majors, N>>3, M>>4.
+__device__ __forceinline__ uint32_t instr_desc(bool a_mn, bool b_mn, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__host__ __device__ inline uint32_t stage_bytes(int bn) { return kATileBytes + (uint32_t)bn * BK * 2; }
+
+struct WorkItem { int tm, tn, split, kb0, kb1; };
+__device__ __forceinline__ WorkItem decode(const Params& p, int w) {
+  WorkItem it;
+  const int tiles = p.tiles_m * p.tiles_n;
+  it.split = w / tiles;
+  const int t = w - it.split * tiles;
+  it.tm = t / p.tiles_n;
+  it.tn = t - it.tm * p.tiles_n;
+  it.kb0 = it.split * p.kb_per_split;
+  it.kb1 = min(it.kb0 + p.kb_per_split, p.num_kb);
+  return it;
+}
+
+template <bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
+  const uint32_t sbytes = stage_bytes(p.bn);
+  const uint32_t bar_base = smem_base + (uint32_t)p.stages * sbytes;  // 8-byte aligned
+  // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2]
+  auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (uint32_t)(kMaxStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + 2 + a); };
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total = p.tiles_m * p.tiles_n * p.splits;
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    prefetch_tmap(&tmap_a);
+    prefetch_tmap(&tmap_b);
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = s_tmem_base;
+  volatile int* abort_flag = &s_abort;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int armed = 0;   // stages armed so far (capped at p.stages): all of them hold a copy until consumed
+      bool ok = true;
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+        const WorkItem it = decode(p, w);
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t sa = smem_base + (uint32_t)stage * sbytes, sb = sa + kATileBytes;
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, sbytes);
+          if (!A_MN) {
+            tma_load_2d(sa, &tmap_a, kb * BK, it.tm * BM, fb);
+          } else {
+#pragma unroll
+            for (int i = 0; i < BM / (int)kBoxMN; ++i)
+              tma_load_2d(sa + i * kBoxBytes, &tmap_a, it.tm * BM + i * (int)kBoxMN, kb * BK, fb);
+          }
+          if (!B_MN) {
+            tma_load_2d(sb, &tmap_b, kb * BK, it.tn * p.bn, fb);
+          } else {
+            for (int i = 0; i < p.bn / (int)kBoxMN; ++i)
+              tma_load_2d(sb + i * kBoxBytes, &tmap_b, it.tn * p.bn + i * (int)kBoxMN, kb * BK, fb);
+          }
+          if (armed < p.stages) ++armed;
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok || *abort_flag) {
+        // Leaving early: wait (bounded) until the copies already issued have landed, so that
+        // nothing writes this CTA's shared memory after it has exited.
+        int s = stage;
+        uint32_t ph = phase;
+        for (int i = 0; i < armed; ++i) {
+          if (--s < 0) { s = p.stages - 1; ph ^= 1u; }
+          const long long t0 = clock64();
+          while (!mbar_try_wait(full_bar(s), ph) && clock64() - t0 < kWaitCycles) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc(A_MN, B_MN, p.bn);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+        const WorkItem it = decode(p, w);
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.bn);
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tcgen05_fence_after();
+          const uint32_t sa = smem_base + (uint32_t)stage * sbytes, sb = sa + kATileBytes;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t ad = smem_desc(sa + (A_MN ? k * (UMMA_K * 128) : k * (UMMA_K * 2)), A_MN);
+            const uint64_t bd = smem_desc(sb + (B_MN ? k * (UMMA_K * 128) : k * (UMMA_K * 2)), B_MN);
+            umma_bf16(d_tmem, ad, bd, idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));       // stage reusable once these MMAs have read it
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));           // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;                    // TMEM lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+      const WorkItem it = decode(p, w);
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tcgen05_fence_after();
+      const int row = it.tm * BM + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      const int n_base = it.tn * p.bn;
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.bn);
+      float dot = 0.f;
+      for (int c = 0; c < p.bn / 32; ++c) {
+        const int n0 = n_base + c * 32;
+        if (n0 >= p.N) break;                  // uniform across the warp
+        uint32_t v[32];
+        tmem_ld32(t_row + (uint32_t)(c * 32), v);
+        tmem_ld_wait();
+        const bool full_chunk = n0 + 32 <= p.N;
+        if (EPI == EPI_STORE) {
+          if (row_ok) {
+            __nv_bfloat16* o = p.out + (int64_t)row * p.ldo + n0;
+            if (full_chunk) {
+              uint32_t packed[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                float a = __uint_as_float(v[2 * i]), b = __uint_as_float(v[2 * i + 1]);
+                if (p.col_scale) { a *= __ldg(p.col_scale + n0 + 2 * i); b *= __ldg(p.col_scale + n0 + 2 * i + 1); }
+                __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                packed[i] = *reinterpret_cast<uint32_t*>(&h);
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                *reinterpret_cast<uint4*>(o + 8 * i) = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                if (n0 + i < p.N) {
+                  float a = __uint_as_float(v[i]);
+                  if (p.col_scale) a *= __ldg(p.col_scale + n0 + i);
+                  o[i] = __float2bfloat16_rn(a);
+                }
+              }
+            }
+          }
+        } else {
+          if (row_ok) {
+            float* o = p.slices + (int64_t)it.split * p.slice_elems + (int64_t)row * p.ld_slice + n0;
+            if (full_chunk) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<uint4*>(o + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n0 + i < p.N) o[i] = __uint_as_float(v[i]);
+            }
+            if (p.qdot) {
+              const __nv_bfloat16* qr = p.qdot + (int64_t)row * p.ldq + n0;
+              if (full_chunk) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(qr + 8 * i));
+                  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    const float2 f = __bfloat1622float2(h[j]);
+                    dot = fmaf(__uint_as_float(v[8 * i + 2 * j]), f.x, dot);
+                    dot = fmaf(__uint_as_float(v[8 * i + 2 * j + 1]), f.y, dot);
+                  }
+                }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+              }
+            }
+          }
+        }
+      }
+      if (EPI == EPI_SLICE && p.qdot && row_ok)
+        p.dz_part[(int64_t)(it.split * p.tiles_n + it.tn) * p.dz_stride + row] = dot;
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tcgen05_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace tc
+}  // namespace flop

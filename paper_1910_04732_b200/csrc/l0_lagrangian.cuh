@@ -1,0 +1,154 @@
+// Expected L0 size and augmented-Lagrangian penalty (Eq. 3 and Section 4.3).
+//
+// Three launches, no atomics, fixed summation order (bit-reproducible):
+//   1. l0_partial_kernel : every block owns one chunk of kChunk gates of ONE
+//      segment and writes sum(pi_j) of the chunk (fp64) to scratch.
+//   2. l0_finalize_kernel: one block adds the chunk sums per segment in chunk
+//      order, forms s, g, dg/dlambda and the gradient coefficient.
+//   3. l0_grad_kernel    : dlog_alpha_j += coef * size_seg * pi_j (1 - pi_j).
+// Blocks find their (segment, chunk) from the segment table alone: chunk
+// counts per segment are prefix-summed in shared memory by every block.
+#pragma once
+#include "common.cuh"
+
+namespace flop {
+
+constexpr int kL0Threads = 256;
+constexpr int kL0PerThread = 4;
+constexpr int kL0Chunk = kL0Threads * kL0PerThread;  // gates per block
+constexpr int kL0MaxSeg = 4096;
+
+struct L0Scratch {         // layout of the caller's workspace
+  double coef;             // (lambda1 + 2 lambda2 (s - t)) / S
+  double pad[31];
+  double partial[1];       // [n_chunks_max]
+};
+
+// Fills seg_first_chunk[0..n_seg] (exclusive prefix of chunks per segment) in
+// shared memory.  Serial per 16 segments per thread, then a block scan.
+__device__ __forceinline__ void l0_chunk_table(const int64_t* __restrict__ seg_off, int n_seg, int* first_chunk,
+                                               int* scan_scratch) {
+  constexpr int per = kL0MaxSeg / kL0Threads;  // 16
+  const int s0 = threadIdx.x * per;
+  int cnt[per];
+  int sum = 0;
+#pragma unroll
+  for (int i = 0; i < per; ++i) {
+    const int s = s0 + i;
+    int c = 0;
+    if (s < n_seg) {
+      const int64_t len = seg_off[s + 1] - seg_off[s];
+      c = len > 0 ? (int)((len + kL0Chunk - 1) / kL0Chunk) : 0;
+    }
+    cnt[i] = c;
+    sum += c;
+  }
+  int total;
+  int base = block_exclusive_scan(sum, scan_scratch, &total);
+#pragma unroll
+  for (int i = 0; i < per; ++i) {
+    const int s = s0 + i;
+    if (s < n_seg) first_chunk[s] = base;
+    base += cnt[i];
+  }
+  if (threadIdx.x == 0) first_chunk[n_seg] = total;
+  __syncthreads();
+}
+
+// Largest s with first_chunk[s] <= b and a non-empty chunk range containing b.
+__device__ __forceinline__ int l0_find_segment(const int* first_chunk, int n_seg, int b) {
+  int lo = 0, hi = n_seg;  // invariant: first_chunk[lo] <= b < first_chunk[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (first_chunk[mid] <= b) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ float l0_pi(float a, float thr) { return 1.0f / (1.0f + expf(-(a - thr))); }
+
+template <bool kGrad>
+__global__ void __launch_bounds__(kL0Threads)
+l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__ seg_off,
+                const float* __restrict__ seg_size, int n_seg, float thr, L0Scratch* __restrict__ sc,
+                float* __restrict__ dlog_alpha) {
+  __shared__ int first_chunk[kL0MaxSeg + 1];
+  __shared__ int scan_scratch[33];
+  __shared__ double red[32];
+  l0_chunk_table(seg_off, n_seg, first_chunk, scan_scratch);
+  const int b = blockIdx.x;
+  if (b >= first_chunk[n_seg]) {            // surplus block of the upper-bound grid
+    return;
+  }
+  const int seg = l0_find_segment(first_chunk, n_seg, b);
+  const int64_t lo = seg_off[seg] + (int64_t)(b - first_chunk[seg]) * kL0Chunk;
+  const int64_t hi = min(seg_off[seg + 1], lo + (int64_t)kL0Chunk);
+  const int64_t j0 = lo + (int64_t)threadIdx.x * kL0PerThread;
+  float a[kL0PerThread];
+  const bool vec = (j0 + kL0PerThread <= hi) && ((reinterpret_cast<uintptr_t>(log_alpha + j0) & 15) == 0);
+  if (vec) {
+    const float4 v = *reinterpret_cast<const float4*>(log_alpha + j0);
+    a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w;
+  } else {
+#pragma unroll
+    for (int i = 0; i < kL0PerThread; ++i) a[i] = (j0 + i < hi) ? log_alpha[j0 + i] : 0.f;
+  }
+  if (!kGrad) {
+    double sum = 0.0;
+#pragma unroll
+    for (int i = 0; i < kL0PerThread; ++i)
+      if (j0 + i < hi) sum += (double)l0_pi(a[i], thr);
+    sum = block_sum_f64(sum, red);
+    if (threadIdx.x == 0) sc->partial[b] = sum;
+  } else {
+    const float w = (float)(sc->coef * (double)seg_size[seg]);
+    float gsum[kL0PerThread];
+#pragma unroll
+    for (int i = 0; i < kL0PerThread; ++i) {
+      const float p = l0_pi(a[i], thr);
+      gsum[i] = w * p * (1.0f - p);
+    }
+    const bool vecg = vec && ((reinterpret_cast<uintptr_t>(dlog_alpha + j0) & 15) == 0);
+    if (vecg) {
+      float4 g = *reinterpret_cast<float4*>(dlog_alpha + j0);
+      g.x += gsum[0]; g.y += gsum[1]; g.z += gsum[2]; g.w += gsum[3];
+      *reinterpret_cast<float4*>(dlog_alpha + j0) = g;
+    } else {
+#pragma unroll
+      for (int i = 0; i < kL0PerThread; ++i)
+        if (j0 + i < hi) dlog_alpha[j0 + i] += gsum[i];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kL0Threads)
+l0_finalize_kernel(const int64_t* __restrict__ seg_off, const float* __restrict__ seg_size, int n_seg,
+                   const float* __restrict__ target, const float* __restrict__ lambda, L0Scratch* __restrict__ sc,
+                   float* __restrict__ out4, float* __restrict__ seg_expected) {
+  __shared__ int first_chunk[kL0MaxSeg + 1];
+  __shared__ int scan_scratch[33];
+  __shared__ double red[32];
+  l0_chunk_table(seg_off, n_seg, first_chunk, scan_scratch);
+  double weighted = 0.0, total_size = 0.0;   // identical in every thread
+  for (int s = 0; s < n_seg; ++s) {
+    double v = 0.0;
+    for (int c = first_chunk[s] + threadIdx.x; c < first_chunk[s + 1]; c += kL0Threads) v += sc->partial[c];
+    v = block_sum_f64(v, red);
+    if (threadIdx.x == 0 && seg_expected) seg_expected[s] = (float)v;
+    const double size = (double)seg_size[s];
+    weighted += size * v;
+    total_size += size * (double)(seg_off[s + 1] - seg_off[s]);
+  }
+  if (threadIdx.x == 0) {
+    const double s = total_size > 0.0 ? weighted / total_size : 0.0;
+    const double diff = s - (double)target[0];
+    const double l1 = (double)lambda[0], l2 = (double)lambda[1];
+    out4[0] = (float)s;
+    out4[1] = (float)(l1 * diff + l2 * diff * diff);
+    out4[2] = (float)diff;
+    out4[3] = (float)(diff * diff);
+    sc->coef = total_size > 0.0 ? (l1 + 2.0 * l2 * diff) / total_size : 0.0;
+  }
+}
+
+}  // namespace flop
