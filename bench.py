@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the FLOP gated low-rank hot path on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+sample every gate of every layer (one launch), then for every factorized matrix
+of every layer the gated forward (2 GEMMs) and backward (4 GEMMs + the fused
+dlog_alpha reduction), then the expected-L0 / Lagrangian term over all gates.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload bert|sru|txl] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e`
+is the same step fed from pinned host memory (H2D of every X and dY inside the
+timed region, D2H of dlog_alpha and the Lagrangian scalars); `roofline` times
+the tensor-core GEMM launches with CUDA events; `cpu_baseline` is the fp64
+oracle timed on the host cores on a bounded sample.  `--impl reference` times
+the oracle alone.  Under torchrun every rank processes its own token batch
+with the same gate sample and the weight gradients are all-reduced (NCCL).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1910_04732_b200 import inputs as I  # noqa: E402
+
+METRIC = "gated low-rank fwd+bwd tokens/s and TFLOP/s, % of B200 bf16 tensor peak"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+HC = tuple(float(np.float32(v)) for v in (I.BETA, I.GAMMA, I.ZETA))
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower() == "active":
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- our arm
+class Job:
+    """Device state of one workload: inputs, outputs and scratch of every matrix."""
+
+    def __init__(self, w: I.Workload, device, seed: int):
+        import torch
+        from paper_1910_04732_b200 import binding as b
+        self.w, self.b, self.torch = w, b, torch
+        bf = torch.bfloat16
+        g = torch.Generator(device=device)
+        g.manual_seed(seed)
+        mats = w.all_matrices()
+        self.n_gates = w.n_gates()
+        # gate state, concatenated over all matrices
+        alphas, offs, sizes = [], [0], []
+        for l, i, m in mats:
+            alphas.append(I.log_alpha(w.alpha, m.r, 0, l, i))
+            offs.append(offs[-1] + m.r)
+            sizes.append(float(m.d_in + m.d_out))
+        self.log_alpha = torch.from_numpy(np.concatenate(alphas)).to(device)
+        self.seg_off = torch.tensor(offs, dtype=torch.int64, device=device)
+        self.seg_size = torch.tensor(sizes, dtype=torch.float32, device=device)
+        self.z = torch.empty(self.n_gates, device=device)
+        self.dz_dla = torch.empty(self.n_gates, device=device)
+        self.mask = torch.empty(self.n_gates, dtype=torch.uint8, device=device)
+        self.dlog_alpha = torch.zeros(self.n_gates, device=device)
+        self.target = torch.tensor([w.target], device=device)
+        self.lam = torch.tensor([0.3, 1.7], device=device)
+        self.out4 = torch.zeros(4, device=device)
+        # weight gradients of all matrices in one flat buffer (one all-reduce under data parallelism)
+        r8 = lambda v: (v + 7) // 8 * 8
+        n_w = sum(m.d_out * r8(m.r) + m.r * r8(m.d_in) for _, _, m in mats)
+        self.wgrad = torch.zeros(n_w, dtype=bf, device=device)
+        self.mats, pos, ws_bytes = [], 0, 0
+        randn = lambda rows, cols, scale=1.0: (torch.randn(rows, r8(cols), generator=g, device=device) * scale).to(bf)[:, :cols]
+        for (l, i, m), lo in zip(mats, offs):
+            e = dict(m=m, lo=lo, hi=lo + m.r)
+            e["X"], e["dY"] = randn(w.T, m.d_in), randn(w.T, m.d_out)
+            e["Q"], e["P"] = randn(m.r, m.d_in, m.d_in ** -0.5), randn(m.d_out, m.r, m.r ** -0.5)
+            e["H"], e["Y"], e["dX"] = (b.padded(w.T, c, bf, device) for c in (m.r, m.d_out, m.d_in))
+            e["dP"] = self.wgrad[pos:pos + m.d_out * r8(m.r)].view(m.d_out, r8(m.r))[:, :m.r]; pos += m.d_out * r8(m.r)
+            e["dQ"] = self.wgrad[pos:pos + m.r * r8(m.d_in)].view(m.r, r8(m.d_in))[:, :m.d_in]; pos += m.r * r8(m.d_in)
+            ws_bytes = max(ws_bytes, b.workspace_bytes(b.OP_BWD, w.T, m.d_in, m.d_out, m.r, b.BF16))
+            self.mats.append(e)
+        self.ws = b.alloc_workspace(ws_bytes, device)
+        self.ws_l0 = b.alloc_workspace(b.workspace_bytes(b.OP_L0, self.n_gates, 0, 0, len(sizes), b.F32), device)
+        self.step_no = 0
+        self.world = 1
+
+    def input_bytes(self) -> int:
+        return sum(e["X"].numel() * 2 + e["dY"].numel() * 2 for e in self.mats)
+
+    def run_matrix(self, e):
+        b = self.b
+        z, dzd = self.z[e["lo"]:e["hi"]], self.dz_dla[e["lo"]:e["hi"]]
+        b.gated_lowrank_fwd(e["X"], e["Q"], e["P"], z, e["Y"], e["H"], None)
+        b.gated_lowrank_bwd(e["dY"], e["X"], e["Q"], e["P"], z, dzd, e["H"], e["dX"], e["dP"], e["dQ"],
+                            self.dlog_alpha[e["lo"]:e["hi"]], self.ws)
+
+    def sample_gates(self):
+        # one launch for all gates of all layers; every rank uses the same (seed, offset): one mask per global batch
+        self.b.gate_sample(self.log_alpha, HC, 0, self.step_no << 24, self.z, self.mask, self.dz_dla)
+        self.step_no += 1
+
+    def finish(self):
+        self.b.expected_l0_lagrangian(self.log_alpha, self.seg_off, self.seg_size, HC, self.target, self.lam,
+                                      self.out4, None, self.dlog_alpha, self.ws_l0)
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.all_reduce(self.wgrad)
+            dist.all_reduce(self.dlog_alpha)
+
+    def step(self):
+        self.sample_gates()
+        for e in self.mats:
+            self.run_matrix(e)
+        self.finish()
+
+
+def time_steps(job: Job, steps: int, world: int):
+    """K steps between two synchronisation points, timed with CUDA events on the launching stream."""
+    import torch
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        job.step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    return ms
+
+
+def time_e2e(job: Job, steps: int, world: int):
+    """The same step fed from pinned host memory: every X and dY crosses PCIe inside the timed
+    region (copy stream, overlapped with compute), dlog_alpha and the Lagrangian scalars come back."""
+    import torch
+    host_in = [(e["X"].cpu().pin_memory(), e["dY"].cpu().pin_memory()) for e in job.mats]
+    host_dla = torch.empty(job.n_gates, dtype=torch.float32).pin_memory()
+    host_out4 = torch.empty(4, dtype=torch.float32).pin_memory()
+    copy_stream = torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+    events = [torch.cuda.Event() for _ in job.mats]
+
+    def one_step():
+        copy_stream.wait_stream(main)          # the previous step has consumed the device buffers
+        with torch.cuda.stream(copy_stream):
+            for (hx, hdy), e, ev in zip(host_in, job.mats, events):
+                e["X"].copy_(hx, non_blocking=True)
+                e["dY"].copy_(hdy, non_blocking=True)
+                ev.record(copy_stream)
+        job.sample_gates()
+        for e, ev in zip(job.mats, events):
+            main.wait_event(ev)
+            job.run_matrix(e)
+        job.finish()
+        host_dla.copy_(job.dlog_alpha, non_blocking=True)
+        host_out4.copy_(job.out4, non_blocking=True)
+
+    one_step()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one_step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    h2d = sum(hx.numel() * 2 + hdy.numel() * 2 for hx, hdy in host_in)
+    d2h = host_dla.numel() * 4 + 16
+    assert np.isfinite(host_out4.numpy()).all()
+    return ms, h2d, d2h
+
+
+# ----------------------------------------------------------------------------- oracle arm
+def oracle_sample(w: I.Workload):
+    """The fp64 oracle on a bounded sample: the matrices of layer 0 at the full token count
+    (gate sample, forward, backward) plus the Lagrangian term over all gates of the model.
+    Returns (seconds for the sample, description, threads used)."""
+    from oracle import flop_oracle as O
+    probs = [I.layer_problem(w, 0, i) for i in range(len(w.matrices))]
+    offs, sizes, alphas = [0], [], []
+    for l, i, m in w.all_matrices():
+        alphas.append(I.log_alpha(w.alpha, m.r, 0, l, i)); offs.append(offs[-1] + m.r); sizes.append(m.d_in + m.d_out)
+    alpha_all = np.concatenate(alphas)
+    t0 = time.perf_counter()
+    for i, p in enumerate(probs):
+        z, mask, dzd = O.gate_sample(p["log_alpha"], *HC, seed=0, offset=I.gate_offset(0, i))
+        O.gated_lowrank_fwd(p["X"], p["Q"], p["P"], z)
+        O.gated_lowrank_bwd(p["dY"], p["X"], p["Q"], p["P"], z, dzd)
+    O.expected_l0_lagrangian(alpha_all, offs, sizes, *HC, w.target, 0.3, 1.7)
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return dt, f"layer 0 of {w.layers} ({len(probs)} matrices) at the full T={w.T}; step time = sample x {w.layers}", threads
+
+
+def run_reference(args, w: I.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt, sample, threads = oracle_sample(w)
+        if i >= args.warmup:
+            times.append(dt)
+    step_s = float(np.mean(times)) * w.layers
+    value = w.T / step_s
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "tflops": w.flops_per_step() / step_s / 1e12,
+            "config": {"workload": w.name, "T": w.T, "layers": w.layers,
+                       "matrices": [[m.name, m.d_in, m.d_out, m.r] for m in w.matrices]},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="bert", choices=["bert", "sru", "txl"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    w = I.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args, w)
+        return
+    args.steps = 100 if args.steps is None else args.steps
+    args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
+
+    import torch
+    from paper_1910_04732_b200 import build as _build
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        _build.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    from paper_1910_04732_b200 import binding as b
+    b.load_library()
+
+    job = Job(w, torch.device("cuda", local), seed=1234 + rank)
+    job.world = world
+    for _ in range(args.warmup):
+        job.step()
+    torch.cuda.synchronize()
+    assert b.device_status() == b.OK
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    n0 = b.launch_count()
+    ms = time_steps(job, args.steps, world)
+    launches = (b.launch_count() - n0) // args.steps
+    # second pass of the same steps with CUDA events around every tensor-core GEMM launch
+    b.gemm_timing_begin()
+    ms_timed_pass = time_steps(job, args.steps, world)
+    gemm_ms, gemm_flops, gemm_launches = b.gemm_timing_end()
+    clocks = sampler.stop() if rank == 0 else None
+    assert b.device_status() == b.OK
+
+    e2e = None
+    if not args.no_e2e:
+        e2e_ms, h2d, d2h = time_e2e(job, max(3, min(args.steps, 20)), world)
+        e2e_steps = max(3, min(args.steps, 20))
+        e2e = {"value": w.T * world / (e2e_ms / e2e_steps / 1e3), "unit": "tokens/s", "ms_per_step": e2e_ms / e2e_steps,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = measured_peaks()
+    step_ms = ms / args.steps
+    tokens_s = w.T * world / (step_ms / 1e3)
+    tflops = w.flops_per_step() * world / (step_ms / 1e3) / 1e12
+    gemm_tflops = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
+    line = {
+        "metric": METRIC, "value": tokens_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "tflops": tflops, "pct_of_bf16_peak_nominal": 100.0 * tflops / world / NOMINAL_BF16_TFLOPS,
+        "pct_of_bf16_peak_measured_sustained": 100.0 * tflops / world / peaks["bf16_tflops_sustained"],
+        "config": {"workload": w.name, "T": w.T, "layers": w.layers,
+                   "matrices": [[m.name, m.d_in, m.d_out, m.r] for m in w.matrices],
+                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}",
+                   "l2": f"inputs larger than L2: {job.input_bytes() / 1e6:.0f} MB of X and dY per step, each matrix its own buffers"},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": peaks["bf16_tflops_sustained"],
+                     "unit": "TFLOP/s", "frac": gemm_tflops / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "peak_kind": f"{peak_kind} (sustained; burst {peaks['bf16_tflops']})",
+                     "kernel": "tc::gemm_kernel (all six GEMMs of every matrix)", "launches_per_step": gemm_launches // args.steps,
+                     "kernel_ms_per_step": gemm_ms / args.steps, "step_ms_in_timed_pass": ms_timed_pass / args.steps,
+                     "frac_of_nominal": gemm_tflops / NOMINAL_BF16_TFLOPS},
+        "clocks": clocks,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        dt, sample, threads = oracle_sample(w)
+        line["cpu_baseline"] = {"value": w.T / (dt * w.layers), "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                                "sample": sample, "tflops": w.flops_per_step() / (dt * w.layers) / 1e12}
+    print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -69,6 +69,16 @@ const char* flop_status_string(int status);
  * FLOP_ERR_TIMEOUT) and clears it. */
 int flop_device_status(void* stream);
 
+/* Instrumentation (no counterpart in the paper).  flop_launch_count: kernels this
+ * library has launched so far in this process.  flop_gemm_timing_begin/end: while
+ * timing is on, every tensor-core GEMM launch is bracketed by CUDA events on its
+ * stream; _end waits for them and returns the summed kernel time (ms), the summed
+ * algorithmic flops 2 M N K of those launches and their number (HOST out pointers,
+ * nullable).  Not thread-safe with respect to concurrent launches. */
+unsigned long long flop_launch_count(void);
+int flop_gemm_timing_begin(void);
+int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launches);
+
 /* Bytes of scratch the given call needs (HOST out pointer).  For FLOP_OP_L0
  * pass the total number of gates as T and the number of segments as r. */
 int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt,

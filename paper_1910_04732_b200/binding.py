@@ -20,7 +20,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 
-EXPORTS = ("flop_status_string", "flop_device_status", "flop_workspace_bytes", "flop_gate_sample",
+EXPORTS = ("flop_status_string", "flop_device_status", "flop_launch_count", "flop_gemm_timing_begin",
+           "flop_gemm_timing_end", "flop_workspace_bytes", "flop_gate_sample",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_expected_l0_lagrangian",
            "flop_compact_ranks", "flop_compact_fwd")
 
@@ -51,6 +52,10 @@ def load_library() -> ctypes.CDLL:
     lib.flop_status_string.argtypes = [ci]
     lib.flop_device_status.argtypes = [vp]
     lib.flop_workspace_bytes.argtypes = [ci, i64, i64, i64, i64, ci, ctypes.POINTER(sz)]
+    lib.flop_launch_count.argtypes = []
+    lib.flop_gemm_timing_begin.argtypes = []
+    lib.flop_gemm_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                         ctypes.POINTER(ctypes.c_int64)]
     lib.flop_gate_sample.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
     lib.flop_gated_lowrank_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
                                            i64, i64, i64, i64, ci, vp, sz, vp]
@@ -64,6 +69,7 @@ def load_library() -> ctypes.CDLL:
     lib.flop_compact_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, i64, i64, i64, i64, ci, vp, sz, vp]
     for name in EXPORTS[1:]:
         getattr(lib, name).restype = ci
+    lib.flop_launch_count.restype = ctypes.c_ulonglong
     _lib = lib
     return lib
 
@@ -111,6 +117,22 @@ def workspace_bytes(op: int, T: int, d_in: int, d_out: int, r: int, dt: int) -> 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
     """A 256-byte aligned scratch buffer (torch's caching allocator aligns to 512)."""
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def launch_count() -> int:
+    return int(load_library().flop_launch_count())
+
+
+def gemm_timing_begin() -> None:
+    _check(load_library().flop_gemm_timing_begin(), "flop_gemm_timing_begin")
+
+
+def gemm_timing_end():
+    """(total kernel ms, total algorithmic flops, launches) of the GEMMs since gemm_timing_begin()."""
+    ms, fl, n = ctypes.c_double(0), ctypes.c_double(0), ctypes.c_int64(0)
+    _check(load_library().flop_gemm_timing_end(ctypes.byref(ms), ctypes.byref(fl), ctypes.byref(n)),
+           "flop_gemm_timing_end")
+    return ms.value, fl.value, int(n.value)
 
 
 def device_status() -> int:

@@ -5,10 +5,13 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
 #include <mutex>
+#include <vector>
 
 #include "../../include/flop.h"
 #include "common.cuh"
@@ -24,10 +27,20 @@ typedef __nv_bfloat16 bf16;
 
 namespace {
 
-#define FLOP_CUDA(expr)                           \
-  do {                                            \
-    cudaError_t e__ = (expr);                     \
-    if (e__ != cudaSuccess) return FLOP_ERR_CUDA; \
+// FLOP_DEBUG=1 in the environment prints the failing CUDA call to stderr.
+inline bool debug_on() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("FLOP_DEBUG"); v = (e && e[0] && e[0] != '0') ? 1 : 0; }
+  return v == 1;
+}
+#define FLOP_CUDA(expr)                                                                           \
+  do {                                                                                            \
+    cudaError_t e__ = (expr);                                                                     \
+    if (e__ != cudaSuccess) {                                                                     \
+      if (debug_on()) fprintf(stderr, "[flop] %s:%d: %s -> %s\n", __FILE__, __LINE__, #expr, cudaGetErrorString(e__)); \
+      cudaGetLastError();                                                                         \
+      return FLOP_ERR_CUDA;                                                                       \
+    }                                                                                             \
   } while (0)
 #define FLOP_TRY(expr)              \
   do {                              \
@@ -54,6 +67,45 @@ int num_sms() {
   return n;
 }
 
+
+// ------------------------------------------------------------------ instrumentation
+// Host-side count of kernels launched by this library, and optional CUDA-event timing of
+// the tensor-core GEMM launches (flop_gemm_timing_begin/end): events are recorded on the
+// launching stream around every gemm_kernel launch and summed when timing ends.
+unsigned long long g_launches = 0;
+struct GemmTiming {
+  bool on = false;
+  std::vector<cudaEvent_t> ev;   // pairs (start, stop)
+  size_t used = 0;
+  double flops = 0.0;
+} g_timing;
+std::mutex g_timing_mu;
+
+inline void count_launch(int n = 1) { g_launches += (unsigned long long)n; }
+
+struct GemmTimer {
+  cudaStream_t st;
+  bool active;
+  cudaEvent_t stop = nullptr;
+  GemmTimer(cudaStream_t s, double flops) : st(s), active(false) {
+    if (!g_timing.on) return;
+    std::lock_guard<std::mutex> lk(g_timing_mu);
+    if (g_timing.used + 2 > g_timing.ev.size()) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        g_timing.ev.push_back(e);
+      }
+    }
+    cudaEventRecord(g_timing.ev[g_timing.used], st);
+    stop = g_timing.ev[g_timing.used + 1];
+    g_timing.used += 2;
+    g_timing.flops += flops;
+    active = true;
+  }
+  ~GemmTimer() { if (active) cudaEventRecord(stop, st); }
+};
+
 // ------------------------------------------------------------------ bump allocator over ws
 struct Arena {
   unsigned char* base;
@@ -70,7 +122,7 @@ struct TcPlan {
   int bn, stages, tiles_m, tiles_n, splits, kb_per_split, num_kb;
 };
 
-constexpr int kSmemBudget = 227 * 1024;
+constexpr int kSmemBudget = 227 * 1024 - 1024;   // opt-in maximum minus room for the static __shared__ variables
 constexpr int kSmemBarrierBytes = 8 * (2 * tc::kMaxStages + 4);
 
 // Picks the N tile and the split-K factor by a small cost model: waves over the SMs times
@@ -132,7 +184,10 @@ EncodeTiledFn encode_fn() {
 // Row-major bf16 matrix [rows, cols] with leading dimension ld; box = box_cols x box_rows, 128-byte swizzle.
 int make_tmap(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, uint32_t box_cols, uint32_t box_rows) {
   EncodeTiledFn fn = encode_fn();
-  if (!fn) return FLOP_ERR_CUDA;
+  if (!fn) {
+    if (debug_on()) fprintf(stderr, "[flop] cuTensorMapEncodeTiled entry point not found\n");
+    return FLOP_ERR_CUDA;
+  }
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
   const cuuint32_t box[2] = {box_cols, box_rows};
@@ -140,6 +195,9 @@ int make_tmap(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS && debug_on())
+    fprintf(stderr, "[flop] cuTensorMapEncodeTiled failed (%d): ptr=%p rows=%lld cols=%lld ld=%lld box=%ux%u\n", (int)r, ptr,
+            (long long)rows, (long long)cols, (long long)ld, box_cols, box_rows);
   return r == CUDA_SUCCESS ? FLOP_OK : FLOP_ERR_CUDA;
 }
 
@@ -168,7 +226,11 @@ int launch_tc_inst(const CUtensorMap& ta, const CUtensorMap& tb, const tc::Param
   const int smem = 1024 + p.stages * (int)tc::stage_bytes(p.bn) + kSmemBarrierBytes;
   const int total = p.tiles_m * p.tiles_n * p.splits;
   const int grid = std::min(total, num_sms());
-  kern<<<grid, tc::kThreads, smem, st>>>(ta, tb, p);
+  {
+    GemmTimer timer(st, 2.0 * p.M * (double)p.N * p.K);
+    kern<<<grid, tc::kThreads, smem, st>>>(ta, tb, p);
+  }
+  count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
 }
@@ -210,6 +272,7 @@ int launch_simt(const float* A, int64_t a_sm, int64_t a_sk, const float* B, int6
   const dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64));
   if (grid.y > 65535) return FLOP_ERR_UNSUPPORTED;
   simt_gemm_kernel<<<grid, 256, 0, st>>>(a);
+  count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
 }
@@ -219,6 +282,7 @@ int zero_2d(void* out, int64_t ld, int64_t rows, int64_t cols, cudaStream_t st) 
   if (!out || rows <= 0 || cols <= 0) return FLOP_OK;
   const int64_t n = rows * cols;
   fill_zero_2d_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((T*)out, ld, (int)rows, (int)cols);
+  count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
 }
@@ -290,6 +354,7 @@ static int finalize_wgrad(const float* slices, int n_slices, int64_t slice_elems
   if (M <= 0) return FLOP_OK;
   wgrad_finalize_kernel<TW, TQ><<<(unsigned)M, 256, 0, st>>>(slices, n_slices, slice_elems, ld_slice, (int)M, (int)N, row_scale,
                                                             (TW*)out, ldo, accumulate, (const TQ*)qdot, ldq, dz_out);
+  count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
 }
@@ -318,6 +383,32 @@ int flop_device_status(void* stream) {
     FLOP_CUDA(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)));
   }
   return v;
+}
+
+unsigned long long flop_launch_count(void) { return g_launches; }
+
+int flop_gemm_timing_begin(void) {
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  g_timing.used = 0;
+  g_timing.flops = 0.0;
+  g_timing.on = true;
+  return FLOP_OK;
+}
+
+int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launches) {
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  g_timing.on = false;
+  double ms = 0.0;
+  for (size_t i = 0; i + 1 < g_timing.used; i += 2) {
+    FLOP_CUDA(cudaEventSynchronize(g_timing.ev[i + 1]));
+    float t = 0.f;
+    FLOP_CUDA(cudaEventElapsedTime(&t, g_timing.ev[i], g_timing.ev[i + 1]));
+    ms += (double)t;
+  }
+  if (total_ms) *total_ms = ms;
+  if (total_flops) *total_flops = g_timing.flops;
+  if (launches) *launches = (int64_t)(g_timing.used / 2);
+  return FLOP_OK;
 }
 
 int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt, size_t* out_bytes) {
@@ -352,6 +443,7 @@ int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uin
   const int grid = (int)std::min<int64_t>(want, (int64_t)num_sms() * 16);
   gate_sample_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(log_alpha, n, g, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)),
                                                              offset, z, mask, dz_dla, vec_ok);
+  count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
 }
@@ -500,12 +592,14 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
       }
       if (dlog_alpha) {
         dalpha_kernel<<<(unsigned)((r + 255) / 256), 256, 0, st>>>(w.dz_part, w.n_part, r, dz_dla, (int)r, dlog_alpha, accumulate);
+        count_launch();
         FLOP_CUDA(cudaGetLastError());
       }
     }
     if (dX) {
       // dX = dH' (diag(z) Q)   (B(n=j, k=k_rank) = Qz[k_rank, j]: MN-major)
       scale_rows_kernel<bf16><<<(unsigned)r, 256, 0, st>>>((const bf16*)Q, ldq, z, (int)r, (int)d_in, (bf16*)w.Qz, w.ldqz);
+      count_launch();
       FLOP_CUDA(cudaGetLastError());
       const TcPlan px = plan_tc(T, d_in, r, false);
       FLOP_TRY(launch_tc({w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, T, d_in, r, px, store_epilogue(dX, lddx, nullptr), st));
@@ -525,11 +619,13 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
                                              dlog_alpha ? Q : nullptr, ldq, w.dz_part, st)));
       if (dlog_alpha) {
         dalpha_kernel<<<(unsigned)((r + 255) / 256), 256, 0, st>>>(w.dz_part, 1, r, dz_dla, (int)r, dlog_alpha, accumulate);
+        count_launch();
         FLOP_CUDA(cudaGetLastError());
       }
     }
     if (dX) {
       scale_rows_kernel<float><<<(unsigned)r, 256, 0, st>>>(Qf, ldq, z, (int)r, (int)d_in, (float*)w.Qz, w.ldqz);
+      count_launch();
       FLOP_CUDA(cudaGetLastError());
       // dX[t,j] = sum_k dH'[t,k] Qz[k,j]
       FLOP_TRY(launch_simt(dHf, w.lddh, 1, (const float*)w.Qz, 1, w.ldqz, (float*)dX, lddx, T, d_in, r, nullptr, nullptr, 0, st));
@@ -553,11 +649,16 @@ int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t
   const float thr = (float)((double)hc.beta * log(-(double)hc.gamma / (double)hc.zeta));
   const int64_t chunks = (n + kL0Chunk - 1) / kL0Chunk + n_seg;
   if (chunks > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
-  if (chunks > 0 && n_seg > 0)
+  if (chunks > 0 && n_seg > 0) {
     l0_chunk_kernel<false><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
+    count_launch();
+  }
   l0_finalize_kernel<<<1, kL0Threads, 0, st>>>(seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
-  if (dlog_alpha && chunks > 0 && n_seg > 0)
+  count_launch();
+  if (dlog_alpha && chunks > 0 && n_seg > 0) {
     l0_chunk_kernel<true><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
+    count_launch();
+  }
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
 }
@@ -579,6 +680,7 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
   cudaStream_t st = (cudaStream_t)stream;
   const double thr = (double)hc.beta * log(-(double)hc.gamma / (double)hc.zeta);
   compact_select_kernel<<<1, kSelThreads, 0, st>>>(log_alpha_or_z, mode, thr, (int)r, idx, k_dev, z_det);
+  count_launch();
   FLOP_CUDA(cudaGetLastError());
   if (gather && r > 0) {
     const float* zsrc = z_det ? z_det : log_alpha_or_z;
@@ -603,6 +705,7 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
             (const float*)P, ldp, idx, k_dev, (int)r, (int)d_out, (float*)Pc, ldpc, rows_per_block, vp);
       }
     }
+    count_launch((d_in > 0) + (d_out > 0));
     FLOP_CUDA(cudaGetLastError());
   }
   return FLOP_OK;

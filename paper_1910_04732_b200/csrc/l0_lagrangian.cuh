@@ -105,8 +105,10 @@ l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__
     float gsum[kL0PerThread];
 #pragma unroll
     for (int i = 0; i < kL0PerThread; ++i) {
-      const float p = l0_pi(a[i], thr);
-      gsum[i] = w * p * (1.0f - p);
+      // pi (1 - pi) = e / (1 + e)^2 with e = exp(-|alpha - thr|): no cancellation near pi = 1
+      const float e = expf(-fabsf(a[i] - thr));
+      const float q = 1.0f / (1.0f + e);
+      gsum[i] = w * e * q * q;
     }
     const bool vecg = vec && ((reinterpret_cast<uintptr_t>(dlog_alpha + j0) & 15) == 0);
     if (vecg) {
