@@ -141,6 +141,32 @@ int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t
                                 float* seg_expected, float* dlog_alpha, void* ws, size_t ws_bytes,
                                 void* stream);
 
+/* The same computation as flop_expected_l0_lagrangian for callers that cannot
+ * allocate device memory at all (the paper has no counterpart; this is a
+ * deployment convenience).  Such callers exist: code running inside someone
+ * else's memory plan -- an inference server or training loop whose pool was
+ * sized up front and is now frozen, a plug-in that is handed tensors but no
+ * allocator, a region where cudaMalloc would synchronise the device or is
+ * simply forbidden.  The caller passes only inputs and outputs; the kernels'
+ * scratch is a fixed array that is part of the loaded library (about 41 KB,
+ * held on every GPU that loads the library until the process exits), so the
+ * call performs no cudaMalloc/cudaFree and uses no allocating library routine.
+ *   - Limits: n <= 1,048,576 gates and n_seg <= 4096 segments; larger sizes
+ *     return FLOP_ERR_UNSUPPORTED (FLOP_DEBUG=1 prints the limits) and must use
+ *     flop_expected_l0_lagrangian with a caller-provided workspace.
+ *   - The first call on each device looks up the device address of the
+ *     built-in array (with that device current); make that first call outside
+ *     any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the
+ *     previous call left in it.  Nothing in it has to start at zero (every
+ *     value read is rewritten by the same call first), but two calls whose
+ *     kernels overlap on the GPU -- different streams, no ordering between
+ *     them -- race on it: order them. */
+int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const int64_t* seg_off,
+                                        const float* seg_size, int32_t n_seg, flop_hc_params_t hc,
+                                        const float* target, const float* lambda, float* out4,
+                                        float* seg_expected, float* dlog_alpha, void* stream);
+
 /* Deterministic gates and compaction of one weight matrix (Sections 4.4, 4.1).
  * mode 0: log_alpha_or_z holds log_alpha; k = floor(sum_j pi_j + 1/2); the k
  *         gates with the largest log_alpha are kept (ties: lower index) with

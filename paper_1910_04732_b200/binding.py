@@ -23,6 +23,7 @@ OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 EXPORTS = ("flop_status_string", "flop_device_status", "flop_launch_count", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_workspace_bytes", "flop_gate_sample",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_expected_l0_lagrangian",
+           "flop_expected_l0_lagrangian_noalloc",
            "flop_compact_ranks", "flop_compact_fwd")
 
 
@@ -64,6 +65,7 @@ def load_library() -> ctypes.CDLL:
                                            i64, i64, i64, i64, ci, ci, vp, sz, vp]
     lib.flop_expected_l0_lagrangian.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp,
                                                 vp, sz, vp]
+    lib.flop_expected_l0_lagrangian_noalloc.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp, vp]
     lib.flop_compact_ranks.argtypes = [vp, ci, HcParams, i64, vp, i64, vp, i64, i64, i64, ci,
                                        vp, vp, vp, vp, i64, vp, i64, vp, sz, vp]
     lib.flop_compact_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, i64, i64, i64, i64, ci, vp, sz, vp]
@@ -181,6 +183,18 @@ def expected_l0_lagrangian(log_alpha, seg_off, seg_size, hc, target, lam, out4, 
         _ptr(log_alpha), log_alpha.numel(), _ptr(seg_off), _ptr(seg_size), seg_size.numel(), _hc(hc),
         _ptr(target), _ptr(lam), _ptr(out4), _ptr(seg_expected), _ptr(dlog_alpha),
         _ptr(ws), ws.numel() if ws is not None else 0, _stream()), "flop_expected_l0_lagrangian")
+
+
+def expected_l0_lagrangian_noalloc(log_alpha, seg_off, seg_size, hc, target, lam, out4, seg_expected=None,
+                                   dlog_alpha=None) -> None:
+    """flop_expected_l0_lagrangian_noalloc: same outputs, no workspace argument.  For callers that
+    may not allocate device memory (a frozen memory pool, a plug-in without an allocator): the
+    scratch is a fixed array inside the library, limited to 1,048,576 gates in 4096 segments and
+    shared by all calls on a device, so calls must not overlap on the GPU."""
+    _check(load_library().flop_expected_l0_lagrangian_noalloc(
+        _ptr(log_alpha), log_alpha.numel(), _ptr(seg_off), _ptr(seg_size), seg_size.numel(), _hc(hc),
+        _ptr(target), _ptr(lam), _ptr(out4), _ptr(seg_expected), _ptr(dlog_alpha), _stream()),
+        "flop_expected_l0_lagrangian_noalloc")
 
 
 def compact_ranks(log_alpha_or_z, mode: int, hc, idx, k_dev, z_det=None, P=None, Q=None, Pc=None, Qc=None) -> None:

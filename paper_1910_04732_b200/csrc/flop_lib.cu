@@ -345,6 +345,38 @@ int check_ws(const void* ws, size_t ws_bytes, size_t need) {
   return FLOP_OK;
 }
 
+
+// ------------------------------------------------------------------ built-in scratch (no-allocation entry point)
+// Scratch of flop_expected_l0_lagrangian_noalloc: a fixed device array that is part of the
+// loaded library image (every GPU that loads the library holds it until the process exits).
+// Sized for kNoAllocMaxGates gates in kNoAllocMaxSeg segments.
+constexpr int64_t kNoAllocMaxGates = 1 << 20;
+constexpr int kNoAllocMaxSeg = kL0MaxSeg;
+constexpr size_t kNoAllocScratchBytes =
+    sizeof(L0Scratch) + (size_t)(kNoAllocMaxGates / kL0Chunk + kNoAllocMaxSeg) * sizeof(double);
+static __device__ __align__(256) unsigned char g_l0_builtin_scratch[kNoAllocScratchBytes];
+
+// In host code the array's name is only a handle; the device address comes from the runtime,
+// asked once per device with that device current.
+constexpr int kMaxDevices = 64;
+void* g_l0_builtin_ptr[kMaxDevices] = {};
+std::mutex g_l0_builtin_mu;
+
+int builtin_scratch(L0Scratch** out) {
+  int dev = -1;
+  FLOP_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return FLOP_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lk(g_l0_builtin_mu);
+  if (!g_l0_builtin_ptr[dev]) {
+    void* p = nullptr;
+    FLOP_CUDA(cudaGetSymbolAddress(&p, g_l0_builtin_scratch));
+    if (!p) return FLOP_ERR_CUDA;
+    g_l0_builtin_ptr[dev] = p;
+  }
+  *out = reinterpret_cast<L0Scratch*>(g_l0_builtin_ptr[dev]);
+  return FLOP_OK;
+}
+
 }  // namespace
 
 template <typename TW, typename TQ>
@@ -649,6 +681,41 @@ int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t
   const float thr = (float)((double)hc.beta * log(-(double)hc.gamma / (double)hc.zeta));
   const int64_t chunks = (n + kL0Chunk - 1) / kL0Chunk + n_seg;
   if (chunks > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  if (chunks > 0 && n_seg > 0) {
+    l0_chunk_kernel<false><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
+    count_launch();
+  }
+  l0_finalize_kernel<<<1, kL0Threads, 0, st>>>(seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
+  count_launch();
+  if (dlog_alpha && chunks > 0 && n_seg > 0) {
+    l0_chunk_kernel<true><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
+    count_launch();
+  }
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const int64_t* seg_off,
+                                        const float* seg_size, int32_t n_seg, flop_hc_params_t hc,
+                                        const float* target, const float* lambda, float* out4,
+                                        float* seg_expected, float* dlog_alpha, void* stream) {
+  if (n < 0 || n_seg < 0 || !valid_hc(hc) || !out4 || !target || !lambda) return FLOP_ERR_INVALID_ARG;
+  if (n > kNoAllocMaxGates || n_seg > kNoAllocMaxSeg) {
+    if (debug_on())
+      fprintf(stderr, "[flop] flop_expected_l0_lagrangian_noalloc: n=%lld gates / n_seg=%d segments exceed the built-in "
+                      "scratch (at most %lld gates, %d segments); use flop_expected_l0_lagrangian with a workspace\n",
+              (long long)n, (int)n_seg, (long long)kNoAllocMaxGates, kNoAllocMaxSeg);
+    return FLOP_ERR_UNSUPPORTED;
+  }
+  if (n_seg > 0 && (!seg_off || !seg_size)) return FLOP_ERR_INVALID_ARG;
+  if (n > 0 && !log_alpha) return FLOP_ERR_INVALID_ARG;
+  L0Scratch* sc = nullptr;
+  FLOP_TRY(builtin_scratch(&sc));
+  cudaStream_t st = (cudaStream_t)stream;
+  const float thr = (float)((double)hc.beta * log(-(double)hc.gamma / (double)hc.zeta));
+  const int64_t chunks = (n + kL0Chunk - 1) / kL0Chunk + n_seg;
+  // Nothing in the scratch has to start at zero: every chunk sum that the finalisation reads and
+  // the gradient coefficient are rewritten by this call before they are read.
   if (chunks > 0 && n_seg > 0) {
     l0_chunk_kernel<false><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
     count_launch();
