@@ -12,6 +12,13 @@ namespace flop {
 // whose bounded wait gave up.  Read and cleared by flop_device_status().
 __device__ int g_device_status = 0;
 
+// Programmatic dependent launch: every kernel of the library is launched so that its prologue may
+// overlap the tail of the kernel before it on the stream.  pdl_wait() blocks until all earlier
+// kernels have completed and their writes are visible; it comes before the first access to
+// global memory.  pdl_launch_dependents() lets the next kernel start its own prologue.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void report_timeout() { atomicExch(&g_device_status, (int)FLOP_ERR_TIMEOUT); }
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);

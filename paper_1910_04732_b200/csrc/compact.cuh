@@ -23,6 +23,8 @@ __device__ __forceinline__ uint32_t order_key(float a) {
 __global__ void __launch_bounds__(kSelThreads)
 compact_select_kernel(const float* __restrict__ in, int mode, double thr, int r, int32_t* __restrict__ idx,
                       int32_t* __restrict__ k_dev, float* __restrict__ z_det) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ double red[32];
   __shared__ int hist[256];
   __shared__ int scan_scratch[33];
@@ -111,6 +113,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 gather_q_kernel(const T* __restrict__ Q, int64_t ldq, const int32_t* __restrict__ idx, const int32_t* __restrict__ k_dev,
                 const float* __restrict__ z, int d_in, T* __restrict__ Qc, int64_t ldqc, int vec_ok) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int c = blockIdx.x;
   if (c >= *k_dev) return;
   const int src = idx[c];
@@ -140,6 +144,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 gather_p_kernel(const T* __restrict__ P, int64_t ldp, const int32_t* __restrict__ idx, const int32_t* __restrict__ k_dev,
                 int r, int d_out, T* __restrict__ Pc, int64_t ldpc, int rows_per_block, int vec_ok) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* row = reinterpret_cast<T*>(smem_raw);
   const int k = *k_dev;

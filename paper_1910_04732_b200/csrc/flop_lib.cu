@@ -11,6 +11,7 @@
 
 #include <algorithm>
 #include <mutex>
+#include <utility>
 #include <vector>
 
 #include "../../include/flop.h"
@@ -47,6 +48,27 @@ inline bool debug_on() {
     int s__ = (expr);               \
     if (s__ != FLOP_OK) return s__; \
   } while (0)
+
+
+// Every kernel goes through here: programmatic dependent launch lets a kernel's prologue overlap
+// the tail of its predecessor on the stream (the kernels call griddepcontrol.wait before they
+// touch global memory).  FLOP_NO_PDL=1 in the environment turns the attribute off.
+inline bool pdl_on() {
+  static int v = -1;
+  if (v < 0) { const char* e = getenv("FLOP_NO_PDL"); v = (e && e[0] && e[0] != '0') ? 0 : 1; }
+  return v == 1;
+}
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_on() ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);   // errors are picked up by cudaGetLastError()
+}
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
@@ -228,7 +250,7 @@ int launch_tc_inst(const CUtensorMap& ta, const CUtensorMap& tb, const tc::Param
   const int grid = std::min(total, num_sms());
   {
     GemmTimer timer(st, 2.0 * p.M * (double)p.N * p.K);
-    kern<<<grid, tc::kThreads, smem, st>>>(ta, tb, p);
+    launch_k(kern, dim3(grid), dim3(tc::kThreads), (size_t)(smem), st, ta, tb, p);
   }
   count_launch();
   FLOP_CUDA(cudaGetLastError());
@@ -271,7 +293,7 @@ int launch_simt(const float* A, int64_t a_sm, int64_t a_sk, const float* B, int6
   SimtGemmArgs a{A, a_sm, a_sk, B, b_sn, b_sk, C, ldc, (int)M, (int)N, (int)K, col_scale, row_scale, accumulate};
   const dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64));
   if (grid.y > 65535) return FLOP_ERR_UNSUPPORTED;
-  simt_gemm_kernel<<<grid, 256, 0, st>>>(a);
+  launch_k(simt_gemm_kernel, dim3(grid), dim3(256), (size_t)(0), st, a);
   count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
@@ -281,7 +303,7 @@ template <typename T>
 int zero_2d(void* out, int64_t ld, int64_t rows, int64_t cols, cudaStream_t st) {
   if (!out || rows <= 0 || cols <= 0) return FLOP_OK;
   const int64_t n = rows * cols;
-  fill_zero_2d_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((T*)out, ld, (int)rows, (int)cols);
+  launch_k(fill_zero_2d_kernel<T>, dim3((unsigned)((n + 255) / 256)), dim3(256), (size_t)(0), st, (T*)out, ld, (int)rows, (int)cols);
   count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
@@ -303,7 +325,8 @@ FwdWs plan_fwd_ws(Arena& ar, int64_t T, int64_t r, int dt) {
 struct BwdWs {
   void* dH; int64_t lddh;        // dH'[T, r]
   void* Qz; int64_t ldqz;        // diag(z) Q [r, d_in]
-  float* slices; int64_t ld_slice_p, ld_slice_q, slice_elems_p, slice_elems_q;
+  float* slices_p; float* slices_q;   // fp32 split-K slices of dY^T H' and dH'^T X
+  int64_t ld_slice_p, ld_slice_q, slice_elems_p, slice_elems_q;
   float* dz_part; int n_part;
   TcPlan plan_p, plan_q;
   size_t bytes;
@@ -327,8 +350,8 @@ BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, 
   }
   w.slice_elems_p = d_out * w.ld_slice_p;
   w.slice_elems_q = r * w.ld_slice_q;
-  const size_t slice_bytes = std::max((size_t)sp * w.slice_elems_p, (size_t)sq * w.slice_elems_q) * 4;
-  w.slices = (float*)ar.take(slice_bytes);
+  w.slices_p = dt == FLOP_BF16 ? (float*)ar.take((size_t)sp * w.slice_elems_p * 4) : nullptr;
+  w.slices_q = (float*)ar.take((size_t)sq * w.slice_elems_q * 4);
   w.dz_part = (float*)ar.take((size_t)w.n_part * std::max<int64_t>(r, 1) * 4);
   w.bytes = ar.used;
   return w;
@@ -384,7 +407,7 @@ static int finalize_wgrad(const float* slices, int n_slices, int64_t slice_elems
                           const float* row_scale, void* out, int64_t ldo, int accumulate, const void* qdot, int64_t ldq,
                           float* dz_out, cudaStream_t st) {
   if (M <= 0) return FLOP_OK;
-  wgrad_finalize_kernel<TW, TQ><<<(unsigned)M, 256, 0, st>>>(slices, n_slices, slice_elems, ld_slice, (int)M, (int)N, row_scale,
+  launch_k(wgrad_finalize_kernel<TW, TQ>, dim3((unsigned)M), dim3(256), (size_t)(0), st, slices, n_slices, slice_elems, ld_slice, (int)M, (int)N, row_scale,
                                                             (TW*)out, ldo, accumulate, (const TQ*)qdot, ldq, dz_out);
   count_launch();
   FLOP_CUDA(cudaGetLastError());
@@ -473,7 +496,7 @@ int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uin
   const int64_t nblk = (n + 3) / 4;
   const int64_t want = (nblk + 255) / 256;
   const int grid = (int)std::min<int64_t>(want, (int64_t)num_sms() * 16);
-  gate_sample_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(log_alpha, n, g, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)),
+  launch_k(gate_sample_kernel, dim3(grid), dim3(256), (size_t)(0), (cudaStream_t)stream, log_alpha, n, g, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)),
                                                              offset, z, mask, dz_dla, vec_ok);
   count_launch();
   FLOP_CUDA(cudaGetLastError());
@@ -603,36 +626,36 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
     if (dP) {
       // dP = dY^T H'        (contract over tokens: both operands MN-major), fp32 split-K slices
       TcEpilogue e{};
-      e.kind = tc::EPI_SLICE; e.slices = w.slices; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
+      e.kind = tc::EPI_SLICE; e.slices = w.slices_p; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
       FLOP_TRY(launch_tc({dY, lddy, true}, {H_save, ldh, true}, d_out, r, T, w.plan_p, e, st));
-      if (wgrad_dt == FLOP_BF16)
-        FLOP_TRY((finalize_wgrad<bf16, bf16>(w.slices, w.plan_p.splits, w.slice_elems_p, w.ld_slice_p, d_out, r, nullptr, dP, lddp, accumulate, nullptr, 0, nullptr, st)));
-      else
-        FLOP_TRY((finalize_wgrad<float, bf16>(w.slices, w.plan_p.splits, w.slice_elems_p, w.ld_slice_p, d_out, r, nullptr, dP, lddp, accumulate, nullptr, 0, nullptr, st)));
     }
     if (need_m) {
       // M = dH'^T X; dQ = diag(z) M; dz_k = <Q[k,:], M[k,:]> fused into the GEMM epilogue per tile
       TcEpilogue e{};
-      e.kind = tc::EPI_SLICE; e.slices = w.slices; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
+      e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
       if (dlog_alpha) { e.qdot = (const bf16*)Q; e.ldq = ldq; e.dz_part = w.dz_part; e.dz_stride = r; }
       FLOP_TRY(launch_tc({w.dH, w.lddh, true}, {X, ldx, true}, r, d_in, T, w.plan_q, e, st));
-      if (dQ) {
-        if (wgrad_dt == FLOP_BF16)
-          FLOP_TRY((finalize_wgrad<bf16, bf16>(w.slices, w.plan_q.splits, w.slice_elems_q, w.ld_slice_q, r, d_in, z, dQ, lddq, accumulate, nullptr, 0, nullptr, st)));
-        else
-          FLOP_TRY((finalize_wgrad<float, bf16>(w.slices, w.plan_q.splits, w.slice_elems_q, w.ld_slice_q, r, d_in, z, dQ, lddq, accumulate, nullptr, 0, nullptr, st)));
-      }
-      if (dlog_alpha) {
-        dalpha_kernel<<<(unsigned)((r + 255) / 256), 256, 0, st>>>(w.dz_part, w.n_part, r, dz_dla, (int)r, dlog_alpha, accumulate);
+    }
+    {
+      // one launch: ordered split-K sums -> dP, diag(z)-scaled dQ; diag(z) Q for the dX GEMM; dlog_alpha
+      BwdFinishArgs a{};
+      a.slices_p = w.slices_p; a.n_slices_p = w.plan_p.splits; a.slice_elems_p = w.slice_elems_p; a.ld_slice_p = w.ld_slice_p;
+      a.d_out = (int)d_out; a.r = (int)r; a.dP = dP; a.lddp = lddp;
+      a.slices_q = w.slices_q; a.n_slices_q = w.plan_q.splits; a.slice_elems_q = w.slice_elems_q; a.ld_slice_q = w.ld_slice_q;
+      a.d_in = (int)d_in; a.dQ = dQ; a.lddq = lddq; a.z = z;
+      a.Q = (const bf16*)Q; a.ldq = ldq; a.Qz = dX ? (bf16*)w.Qz : nullptr; a.ldqz = w.ldqz;
+      a.dz_part = w.dz_part; a.n_part = w.n_part; a.dz_dla = dz_dla; a.dlog_alpha = dlog_alpha; a.accumulate = accumulate;
+      const int64_t units = (dP ? d_out * ((r + 3) / 4) : 0) + ((dQ ? 1 : 0) + (dX ? 1 : 0)) * r * ((d_in + 3) / 4) + (dlog_alpha ? r : 0);
+      if (units > 0) {
+        const int grid = (int)std::min<int64_t>((units + 255) / 256, (int64_t)num_sms() * 8);
+        if (wgrad_dt == FLOP_BF16) launch_k(bwd_finish_kernel<bf16>, dim3(grid), dim3(256), (size_t)(0), st, a);
+        else                       launch_k(bwd_finish_kernel<float>, dim3(grid), dim3(256), (size_t)(0), st, a);
         count_launch();
         FLOP_CUDA(cudaGetLastError());
       }
     }
     if (dX) {
       // dX = dH' (diag(z) Q)   (B(n=j, k=k_rank) = Qz[k_rank, j]: MN-major)
-      scale_rows_kernel<bf16><<<(unsigned)r, 256, 0, st>>>((const bf16*)Q, ldq, z, (int)r, (int)d_in, (bf16*)w.Qz, w.ldqz);
-      count_launch();
-      FLOP_CUDA(cudaGetLastError());
       const TcPlan px = plan_tc(T, d_in, r, false);
       FLOP_TRY(launch_tc({w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, T, d_in, r, px, store_epilogue(dX, lddx, nullptr), st));
     }
@@ -646,17 +669,17 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
     if (dP) FLOP_TRY(launch_simt(dYf, 1, lddy, Hf, 1, ldh, (float*)dP, lddp, d_out, r, T, nullptr, nullptr, accumulate, st));
     if (need_m) {
       // M[k,j] = sum_t dH'[t,k] X[t,j] into the slice buffer, then the same finalisation as the tensor-core path
-      FLOP_TRY(launch_simt(dHf, 1, w.lddh, Xf, 1, ldx, w.slices, w.ld_slice_q, r, d_in, T, nullptr, nullptr, 0, st));
-      FLOP_TRY((finalize_wgrad<float, float>(w.slices, 1, w.slice_elems_q, w.ld_slice_q, r, d_in, z, dQ, lddq, accumulate,
+      FLOP_TRY(launch_simt(dHf, 1, w.lddh, Xf, 1, ldx, w.slices_q, w.ld_slice_q, r, d_in, T, nullptr, nullptr, 0, st));
+      FLOP_TRY((finalize_wgrad<float, float>(w.slices_q, 1, w.slice_elems_q, w.ld_slice_q, r, d_in, z, dQ, lddq, accumulate,
                                              dlog_alpha ? Q : nullptr, ldq, w.dz_part, st)));
       if (dlog_alpha) {
-        dalpha_kernel<<<(unsigned)((r + 255) / 256), 256, 0, st>>>(w.dz_part, 1, r, dz_dla, (int)r, dlog_alpha, accumulate);
+        launch_k(dalpha_kernel, dim3((unsigned)((r + 255) / 256)), dim3(256), (size_t)(0), st, w.dz_part, 1, r, dz_dla, (int)r, dlog_alpha, accumulate);
         count_launch();
         FLOP_CUDA(cudaGetLastError());
       }
     }
     if (dX) {
-      scale_rows_kernel<float><<<(unsigned)r, 256, 0, st>>>(Qf, ldq, z, (int)r, (int)d_in, (float*)w.Qz, w.ldqz);
+      launch_k(scale_rows_kernel<float>, dim3((unsigned)r), dim3(256), (size_t)(0), st, Qf, ldq, z, (int)r, (int)d_in, (float*)w.Qz, w.ldqz);
       count_launch();
       FLOP_CUDA(cudaGetLastError());
       // dX[t,j] = sum_k dH'[t,k] Qz[k,j]
@@ -682,13 +705,13 @@ int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t
   const int64_t chunks = (n + kL0Chunk - 1) / kL0Chunk + n_seg;
   if (chunks > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
   if (chunks > 0 && n_seg > 0) {
-    l0_chunk_kernel<false><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
+    launch_k(l0_chunk_kernel<false>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
     count_launch();
   }
-  l0_finalize_kernel<<<1, kL0Threads, 0, st>>>(seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
+  launch_k(l0_finalize_kernel, dim3(1), dim3(kL0Threads), (size_t)(0), st, seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
   count_launch();
   if (dlog_alpha && chunks > 0 && n_seg > 0) {
-    l0_chunk_kernel<true><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
+    launch_k(l0_chunk_kernel<true>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
     count_launch();
   }
   FLOP_CUDA(cudaGetLastError());
@@ -717,13 +740,13 @@ int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const
   // Nothing in the scratch has to start at zero: every chunk sum that the finalisation reads and
   // the gradient coefficient are rewritten by this call before they are read.
   if (chunks > 0 && n_seg > 0) {
-    l0_chunk_kernel<false><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
+    launch_k(l0_chunk_kernel<false>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
     count_launch();
   }
-  l0_finalize_kernel<<<1, kL0Threads, 0, st>>>(seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
+  launch_k(l0_finalize_kernel, dim3(1), dim3(kL0Threads), (size_t)(0), st, seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
   count_launch();
   if (dlog_alpha && chunks > 0 && n_seg > 0) {
-    l0_chunk_kernel<true><<<(unsigned)chunks, kL0Threads, 0, st>>>(log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
+    launch_k(l0_chunk_kernel<true>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
     count_launch();
   }
   FLOP_CUDA(cudaGetLastError());
@@ -746,7 +769,7 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
   }
   cudaStream_t st = (cudaStream_t)stream;
   const double thr = (double)hc.beta * log(-(double)hc.gamma / (double)hc.zeta);
-  compact_select_kernel<<<1, kSelThreads, 0, st>>>(log_alpha_or_z, mode, thr, (int)r, idx, k_dev, z_det);
+  launch_k(compact_select_kernel, dim3(1), dim3(kSelThreads), (size_t)(0), st, log_alpha_or_z, mode, thr, (int)r, idx, k_dev, z_det);
   count_launch();
   FLOP_CUDA(cudaGetLastError());
   if (gather && r > 0) {
@@ -758,17 +781,17 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
     const size_t smem = (size_t)r * es;
     if (smem > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
     if (dt == FLOP_BF16) {
-      if (d_in > 0) gather_q_kernel<bf16><<<(unsigned)r, 256, 0, st>>>((const bf16*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (bf16*)Qc, ldqc, vq);
+      if (d_in > 0) launch_k(gather_q_kernel<bf16>, dim3((unsigned)r), dim3(256), (size_t)(0), st, (const bf16*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (bf16*)Qc, ldqc, vq);
       if (d_out > 0) {
         if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(gather_p_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        gather_p_kernel<bf16><<<(unsigned)((d_out + rows_per_block - 1) / rows_per_block), 256, smem, st>>>(
+        launch_k(gather_p_kernel<bf16>, dim3((unsigned)((d_out + rows_per_block - 1) / rows_per_block)), dim3(256), (size_t)(smem), st, 
             (const bf16*)P, ldp, idx, k_dev, (int)r, (int)d_out, (bf16*)Pc, ldpc, rows_per_block, vp);
       }
     } else {
-      if (d_in > 0) gather_q_kernel<float><<<(unsigned)r, 256, 0, st>>>((const float*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (float*)Qc, ldqc, vq);
+      if (d_in > 0) launch_k(gather_q_kernel<float>, dim3((unsigned)r), dim3(256), (size_t)(0), st, (const float*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (float*)Qc, ldqc, vq);
       if (d_out > 0) {
         if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(gather_p_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        gather_p_kernel<float><<<(unsigned)((d_out + rows_per_block - 1) / rows_per_block), 256, smem, st>>>(
+        launch_k(gather_p_kernel<float>, dim3((unsigned)((d_out + rows_per_block - 1) / rows_per_block)), dim3(256), (size_t)(smem), st, 
             (const float*)P, ldp, idx, k_dev, (int)r, (int)d_out, (float*)Pc, ldpc, rows_per_block, vp);
       }
     }

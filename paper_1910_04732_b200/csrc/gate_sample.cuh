@@ -67,6 +67,8 @@ __device__ __forceinline__ void gate_one(float alpha, uint32_t bits, const GateC
 __global__ void __launch_bounds__(256)
 gate_sample_kernel(const float* __restrict__ log_alpha, int64_t n, GateConsts g, uint2 key, uint64_t offset,
                    float* __restrict__ z, uint8_t* __restrict__ mask, float* __restrict__ dz_dla, int vec_ok) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int64_t nblk = (n + 3) >> 2;
   for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
     const uint64_t ctr = offset + (uint64_t)b;

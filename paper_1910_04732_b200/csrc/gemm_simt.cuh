@@ -22,6 +22,8 @@ struct SimtGemmArgs {
 
 __global__ void __launch_bounds__(256)
 simt_gemm_kernel(SimtGemmArgs p) {
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs[BK][BN + 4];

@@ -202,6 +202,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   tcgen05_fence_after();
   const uint32_t tmem_base = s_tmem_base;
   volatile int* abort_flag = &s_abort;
+  // Everything above touched only shared and tensor memory; from here on global memory written by
+  // earlier kernels is read (and their inputs may be overwritten), so wait for them.
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer

@@ -72,6 +72,8 @@ __global__ void __launch_bounds__(kL0Threads)
 l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__ seg_off,
                 const float* __restrict__ seg_size, int n_seg, float thr, L0Scratch* __restrict__ sc,
                 float* __restrict__ dlog_alpha) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ int first_chunk[kL0MaxSeg + 1];
   __shared__ int scan_scratch[33];
   __shared__ double red[32];
@@ -127,21 +129,31 @@ __global__ void __launch_bounds__(kL0Threads)
 l0_finalize_kernel(const int64_t* __restrict__ seg_off, const float* __restrict__ seg_size, int n_seg,
                    const float* __restrict__ target, const float* __restrict__ lambda, L0Scratch* __restrict__ sc,
                    float* __restrict__ out4, float* __restrict__ seg_expected) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ int first_chunk[kL0MaxSeg + 1];
   __shared__ int scan_scratch[33];
-  __shared__ double red[32];
+  __shared__ double red_w[32], red_s[32];
   l0_chunk_table(seg_off, n_seg, first_chunk, scan_scratch);
-  double weighted = 0.0, total_size = 0.0;   // identical in every thread
-  for (int s = 0; s < n_seg; ++s) {
+  // One warp per segment (segments w, w + nwarp, ...): lanes stride over the segment's chunk sums,
+  // a butterfly adds them, and every warp keeps running totals over its own segments.  The
+  // assignment is fixed, so the result is bit-reproducible.
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = kL0Threads / 32;
+  double weighted = 0.0, total_size = 0.0;
+  for (int s = warp; s < n_seg; s += nwarp) {
     double v = 0.0;
-    for (int c = first_chunk[s] + threadIdx.x; c < first_chunk[s + 1]; c += kL0Threads) v += sc->partial[c];
-    v = block_sum_f64(v, red);
-    if (threadIdx.x == 0 && seg_expected) seg_expected[s] = (float)v;
+    for (int c = first_chunk[s] + lane; c < first_chunk[s + 1]; c += 32) v += sc->partial[c];
+    v = warp_sum_f64(v);
+    if (lane == 0 && seg_expected) seg_expected[s] = (float)v;
     const double size = (double)seg_size[s];
     weighted += size * v;
     total_size += size * (double)(seg_off[s + 1] - seg_off[s]);
   }
+  if (lane == 0) { red_w[warp] = weighted; red_s[warp] = total_size; }
+  __syncthreads();
   if (threadIdx.x == 0) {
+    weighted = 0.0; total_size = 0.0;
+    for (int w = 0; w < nwarp; ++w) { weighted += red_w[w]; total_size += red_s[w]; }
     const double s = total_size > 0.0 ? weighted / total_size : 0.0;
     const double diff = s - (double)target[0];
     const double l1 = (double)lambda[0], l2 = (double)lambda[1];

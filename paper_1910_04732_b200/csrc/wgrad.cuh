@@ -11,6 +11,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 scale_rows_kernel(const T* __restrict__ Q, int64_t ldq, const float* __restrict__ z, int rows, int cols,
                   T* __restrict__ out, int64_t ldo) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int k = blockIdx.x;
   if (k >= rows) return;
   const float g = z[k];
@@ -45,6 +47,8 @@ __global__ void __launch_bounds__(256)
 wgrad_finalize_kernel(const float* __restrict__ slices, int n_slices, int64_t slice_elems, int64_t ld_slice,
                       int M, int N, const float* __restrict__ row_scale, TOut* __restrict__ out, int64_t ldo,
                       int accumulate, const TQ* __restrict__ qdot, int64_t ldq, float* __restrict__ dz_out) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ double red[32];
   const int m = blockIdx.x;
   if (m >= M) return;
@@ -70,6 +74,8 @@ wgrad_finalize_kernel(const float* __restrict__ slices, int n_slices, int64_t sl
 __global__ void __launch_bounds__(256)
 dalpha_kernel(const float* __restrict__ dz_part, int n_part, int64_t part_stride, const float* __restrict__ dz_dla,
               int r, float* __restrict__ dlog_alpha, int accumulate) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= r) return;
   float s = 0.f;
@@ -78,9 +84,130 @@ dalpha_kernel(const float* __restrict__ dz_part, int n_part, int64_t part_stride
   dlog_alpha[k] = accumulate ? dlog_alpha[k] + v : v;
 }
 
+
+// One launch that finishes the backward pass of the tensor-core path:
+//   dP[i,k]      (=|+=) sum_s slices_p[s][i,k]                      (d_out x r)
+//   dQ[k,j]      (=|+=) z[k] * sum_s slices_q[s][k,j]               (r x d_in)
+//   Qz[k,j]      =      z[k] * Q[k,j]                                (r x d_in, feeds the dX GEMM)
+//   dlog_alpha[k](=|+=) dz_dla[k] * sum_p dz_part[p][k]
+// Split-K slices and dz partials are added in index order (bit-reproducible).  Work is cut into
+// units of 4 consecutive columns of one row; a grid-stride loop walks the four regions in turn.
+struct BwdFinishArgs {
+  const float* slices_p; int n_slices_p; int64_t slice_elems_p, ld_slice_p; int d_out, r;
+  void* dP; int64_t lddp;
+  const float* slices_q; int n_slices_q; int64_t slice_elems_q, ld_slice_q; int d_in;
+  void* dQ; int64_t lddq;
+  const float* z;
+  const __nv_bfloat16* Q; int64_t ldq; __nv_bfloat16* Qz; int64_t ldqz;
+  const float* dz_part; int n_part; const float* dz_dla; float* dlog_alpha;
+  int accumulate;
+};
+
+template <typename TW>
+__device__ __forceinline__ void store4(TW* o, const float (&v)[4], int valid, int accumulate, bool vec) {
+  if (vec && valid == 4) {
+    if constexpr (sizeof(TW) == 4) {
+      float4 w = make_float4(v[0], v[1], v[2], v[3]);
+      if (accumulate) { const float4 c = *reinterpret_cast<const float4*>(o); w.x += c.x; w.y += c.y; w.z += c.z; w.w += c.w; }
+      *reinterpret_cast<float4*>(o) = w;
+    } else {
+      float w[4] = {v[0], v[1], v[2], v[3]};
+      if (accumulate) {
+        const uint2 c = *reinterpret_cast<const uint2*>(o);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&c);
+        const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+        w[0] += a.x; w[1] += a.y; w[2] += b.x; w[3] += b.y;
+      }
+      __nv_bfloat162 lo = __floats2bfloat162_rn(w[0], w[1]), hi = __floats2bfloat162_rn(w[2], w[3]);
+      uint2 out;
+      out.x = *reinterpret_cast<uint32_t*>(&lo);
+      out.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(o) = out;
+    }
+  } else {
+    for (int i = 0; i < valid; ++i) o[i] = from_f32<TW>(accumulate ? to_f32<TW>(o[i]) + v[i] : v[i]);
+  }
+}
+
+template <typename TW>
+__device__ __forceinline__ void reduce_unit(const float* __restrict__ slices, int n_slices, int64_t slice_elems, int64_t ld_slice,
+                                            int row, int c0, int ncols, float scale, TW* __restrict__ out, int64_t ldo,
+                                            int accumulate, bool vec_out) {
+  const int valid = min(4, ncols - c0);
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  const float* src = slices + (int64_t)row * ld_slice + c0;
+  if (valid == 4) {
+    for (int s = 0; s < n_slices; ++s) {
+      const float4 v = *reinterpret_cast<const float4*>(src + (int64_t)s * slice_elems);
+      acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+    }
+  } else {
+    for (int s = 0; s < n_slices; ++s)
+      for (int i = 0; i < valid; ++i) acc[i] += src[(int64_t)s * slice_elems + i];
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) acc[i] *= scale;
+  store4<TW>(out + (int64_t)row * ldo + c0, acc, valid, accumulate, vec_out);
+}
+
+template <typename TW>
+__global__ void __launch_bounds__(256)
+bwd_finish_kernel(const BwdFinishArgs a) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int c4r = (a.r + 3) >> 2, c4d = (a.d_in + 3) >> 2;
+  const int64_t n_p = a.dP ? (int64_t)a.d_out * c4r : 0;
+  const int64_t n_q = a.dQ ? (int64_t)a.r * c4d : 0;
+  const int64_t n_qz = a.Qz ? (int64_t)a.r * c4d : 0;
+  const int64_t n_a = a.dlog_alpha ? (int64_t)a.r : 0;
+  const int64_t total = n_p + n_q + n_qz + n_a;
+  constexpr int al = sizeof(TW) == 4 ? 15 : 7;   // 4 outputs: 16 B (fp32) or 8 B (bf16)
+  const bool vec_p = a.dP && ((reinterpret_cast<uintptr_t>(a.dP) & al) == 0) && (a.lddp % 4 == 0);
+  const bool vec_q = a.dQ && ((reinterpret_cast<uintptr_t>(a.dQ) & al) == 0) && (a.lddq % 4 == 0);
+  for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x) {
+    if (u < n_p) {
+      const int row = (int)(u / c4r), c0 = (int)(u % c4r) * 4;
+      reduce_unit<TW>(a.slices_p, a.n_slices_p, a.slice_elems_p, a.ld_slice_p, row, c0, a.r, 1.f, (TW*)a.dP, a.lddp,
+                      a.accumulate, vec_p);
+    } else if (u < n_p + n_q) {
+      const int64_t v = u - n_p;
+      const int row = (int)(v / c4d), c0 = (int)(v % c4d) * 4;
+      reduce_unit<TW>(a.slices_q, a.n_slices_q, a.slice_elems_q, a.ld_slice_q, row, c0, a.d_in, a.z[row], (TW*)a.dQ, a.lddq,
+                      a.accumulate, vec_q);
+    } else if (u < n_p + n_q + n_qz) {
+      const int64_t v = u - n_p - n_q;
+      const int row = (int)(v / c4d), c0 = (int)(v % c4d) * 4;
+      const int valid = min(4, a.d_in - c0);
+      const float g = a.z[row];
+      const __nv_bfloat16* q = a.Q + (int64_t)row * a.ldq + c0;
+      __nv_bfloat16* o = a.Qz + (int64_t)row * a.ldqz + c0;
+      if (valid == 4) {   // Q and Qz rows are 16-byte aligned with ld % 8 == 0: 8-byte accesses are aligned
+        const uint2 raw = *reinterpret_cast<const uint2*>(q);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+        const float2 x = __bfloat1622float2(h[0]), y = __bfloat1622float2(h[1]);
+        __nv_bfloat162 lo = __floats2bfloat162_rn(x.x * g, x.y * g), hi = __floats2bfloat162_rn(y.x * g, y.y * g);
+        uint2 out;
+        out.x = *reinterpret_cast<uint32_t*>(&lo);
+        out.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(o) = out;
+      } else {
+        for (int i = 0; i < valid; ++i) o[i] = __float2bfloat16_rn(__bfloat162float(q[i]) * g);
+      }
+    } else {
+      const int k = (int)(u - n_p - n_q - n_qz);
+      float s = 0.f;
+      for (int p = 0; p < a.n_part; ++p) s += a.dz_part[(int64_t)p * a.r + k];
+      const float v = s * a.dz_dla[k];
+      a.dlog_alpha[k] = a.accumulate ? a.dlog_alpha[k] + v : v;
+    }
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 fill_zero_2d_kernel(T* __restrict__ out, int64_t ld, int rows, int cols) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (int64_t)rows * cols) return;
   out[(i / cols) * ld + (i % cols)] = from_f32<T>(0.f);
