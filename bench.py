@@ -104,7 +104,7 @@ class ClockSampler:
 class Job:
     """Device state of one workload: inputs, outputs and scratch of every matrix."""
 
-    def __init__(self, w: I.Workload, device, seed: int):
+    def __init__(self, w: I.Workload, device, seed: int, n_streams: int = 1):
         import torch
         from paper_1910_04732_b200 import binding as b
         self.w, self.b, self.torch = w, b, torch
@@ -144,7 +144,14 @@ class Job:
             e["dQ"] = self.wgrad[pos:pos + m.r * r8(m.d_in)].view(m.r, r8(m.d_in))[:, :m.d_in]; pos += m.r * r8(m.d_in)
             ws_bytes = max(ws_bytes, b.workspace_bytes(b.OP_BWD, w.T, m.d_in, m.d_out, m.r, b.BF16))
             self.mats.append(e)
-        self.ws = b.alloc_workspace(ws_bytes, device)
+        # independent matrices are issued round-robin on a few streams, each with its own scratch, so
+        # that the tail of one matrix's kernels overlaps the head of another's
+        self.n_streams = max(1, n_streams)
+        self.streams = [torch.cuda.Stream(device=device) for _ in range(self.n_streams)] if self.n_streams > 1 else []
+        self.wss = [b.alloc_workspace(ws_bytes, device) for _ in range(self.n_streams)]
+        self.ws = self.wss[0]
+        self.ev_gates = torch.cuda.Event()
+        self.ev_done = [torch.cuda.Event() for _ in range(self.n_streams)]
         self.ws_l0 = b.alloc_workspace(b.workspace_bytes(b.OP_L0, self.n_gates, 0, 0, len(sizes), b.F32), device)
         self.step_no = 0
         self.world = 1
@@ -152,12 +159,12 @@ class Job:
     def input_bytes(self) -> int:
         return sum(e["X"].numel() * 2 + e["dY"].numel() * 2 for e in self.mats)
 
-    def run_matrix(self, e):
+    def run_matrix(self, e, ws=None):
         b = self.b
         z, dzd = self.z[e["lo"]:e["hi"]], self.dz_dla[e["lo"]:e["hi"]]
         b.gated_lowrank_fwd(e["X"], e["Q"], e["P"], z, e["Y"], e["H"], None)
         b.gated_lowrank_bwd(e["dY"], e["X"], e["Q"], e["P"], z, dzd, e["H"], e["dX"], e["dP"], e["dQ"],
-                            self.dlog_alpha[e["lo"]:e["hi"]], self.ws)
+                            self.dlog_alpha[e["lo"]:e["hi"]], self.ws if ws is None else ws)
 
     def sample_gates(self):
         # one launch for all gates of all layers; every rank uses the same (seed, offset): one mask per global batch
@@ -173,9 +180,23 @@ class Job:
             dist.all_reduce(self.dlog_alpha)
 
     def step(self):
+        torch = self.torch
         self.sample_gates()
-        for e in self.mats:
-            self.run_matrix(e)
+        if self.n_streams == 1:
+            for e in self.mats:
+                self.run_matrix(e)
+        else:
+            main = torch.cuda.current_stream()
+            self.ev_gates.record(main)
+            for s in self.streams:
+                s.wait_event(self.ev_gates)
+            for i, e in enumerate(self.mats):
+                k = i % self.n_streams
+                with torch.cuda.stream(self.streams[k]):
+                    self.run_matrix(e, self.wss[k])
+            for k, s in enumerate(self.streams):
+                self.ev_done[k].record(s)
+                main.wait_event(self.ev_done[k])
         self.finish()
 
 
@@ -309,6 +330,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--streams", type=int, default=1, help="streams over which independent matrices are issued")
     args = ap.parse_args()
     w = I.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -333,7 +355,7 @@ def main():
     from paper_1910_04732_b200 import binding as b
     b.load_library()
 
-    job = Job(w, torch.device("cuda", local), seed=1234 + rank)
+    job = Job(w, torch.device("cuda", local), seed=1234 + rank, n_streams=args.streams)
     job.world = world
     for _ in range(args.warmup):
         job.step()
@@ -379,7 +401,7 @@ def main():
         "pct_of_bf16_peak_measured_sustained": 100.0 * tflops / world / peaks["bf16_tflops_sustained"],
         "config": {"workload": w.name, "T": w.T, "layers": w.layers,
                    "matrices": [[m.name, m.d_in, m.d_out, m.r] for m in w.matrices],
-                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}",
+                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}", "streams": args.streams,
                    "l2": f"inputs larger than L2: {job.input_bytes() / 1e6:.0f} MB of X and dY per step, each matrix its own buffers"},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": peaks["bf16_tflops_sustained"],

@@ -84,6 +84,23 @@ int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launche
 int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt,
                          size_t* out_bytes);
 
+/* The tensor-core GEMM every bf16 path is built from (Section 4.1: the layer is
+ * "simple matrix multiplications"): D[M,N] = sum_k A(m,k) B(n,k), bf16 operands,
+ * fp32 accumulation.  An operand is K-major (memory [MN rows, K cols],
+ * *_mn_major = 0) or MN-major (memory [K rows, MN cols], *_mn_major = 1).
+ * Supported pairs: (K,K) and (K,MN) store bf16 D (ld ldd), each column times the
+ * optional col_scale[n]; (MN,MN) writes fp32 split-K slices
+ * slices[s][m*ldN + n] with ldN = N rounded up to 4 and slice stride M*ldN, which
+ * the caller adds up (the buffer must hold 32 slices unless splits is given).
+ * bn (64, 128, 192, 256), cta2 (0: one CTA per 128-row tile; 1: a CTA pair per
+ * 256-row tile) and splits fix the tile shape; bn = 0, cta2 = -1, splits = 0 leave
+ * each choice to the library.  *n_slices_out (HOST, nullable) receives the number
+ * of slices written (1 for a bf16 store). */
+int flop_tc_gemm(const void* A, int64_t lda, int a_mn_major, const void* B, int64_t ldb,
+                 int b_mn_major, void* D, int64_t ldd, const float* col_scale, float* slices,
+                 int64_t M, int64_t N, int64_t K, int bn, int cta2, int splits, int* n_slices_out,
+                 void* stream);
+
 /* Gate sampling (Section 3, the inverse CDF G(u; alpha) of the hard-concrete
  * distribution), for gates j = 0..n-1:
  *     u_j   = ((x_j >> 9) + 1/2) 2^-23, x_j = word (j mod 4) of the Philox4x32-10

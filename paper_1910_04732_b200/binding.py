@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 
 EXPORTS = ("flop_status_string", "flop_device_status", "flop_launch_count", "flop_gemm_timing_begin",
-           "flop_gemm_timing_end", "flop_workspace_bytes", "flop_gate_sample",
+           "flop_gemm_timing_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_expected_l0_lagrangian",
            "flop_expected_l0_lagrangian_noalloc",
            "flop_compact_ranks", "flop_compact_fwd")
@@ -57,6 +57,8 @@ def load_library() -> ctypes.CDLL:
     lib.flop_gemm_timing_begin.argtypes = []
     lib.flop_gemm_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                          ctypes.POINTER(ctypes.c_int64)]
+    lib.flop_tc_gemm.argtypes = [vp, i64, ci, vp, i64, ci, vp, i64, vp, vp, i64, i64, i64, ci, ci, ci,
+                                 ctypes.POINTER(ctypes.c_int), vp]
     lib.flop_gate_sample.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
     lib.flop_gated_lowrank_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
                                            i64, i64, i64, i64, ci, vp, sz, vp]
@@ -146,6 +148,16 @@ def padded(rows: int, cols: int, dtype, device="cuda", multiple: int = 8) -> tor
     elements (bf16 operands need 16-byte aligned rows)."""
     ld = (cols + multiple - 1) // multiple * multiple
     return torch.zeros(rows, max(ld, multiple), dtype=dtype, device=device)[:, :cols]
+
+
+def tc_gemm(A, a_mn_major: bool, B, b_mn_major: bool, M: int, N: int, K: int, D=None, col_scale=None, slices=None,
+            bn: int = 0, cta2: int = -1, splits: int = 0) -> int:
+    """flop_tc_gemm: D[M,N] = sum_k A(m,k) B(n,k).  Returns the number of fp32 slices written (1 for a bf16 D)."""
+    n = ctypes.c_int(0)
+    _check(load_library().flop_tc_gemm(_ptr(A), _ld(A), int(a_mn_major), _ptr(B), _ld(B), int(b_mn_major),
+                                       _ptr(D), _ld(D) if D is not None else 0, _ptr(col_scale), _ptr(slices),
+                                       M, N, K, bn, cta2, splits, ctypes.byref(n), _stream()), "flop_tc_gemm")
+    return int(n.value)
 
 
 def gate_sample(log_alpha: torch.Tensor, hc, seed: int, offset: int, z: torch.Tensor,

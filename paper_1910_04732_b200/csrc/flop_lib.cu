@@ -20,6 +20,7 @@
 #include "gate_sample.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc2.cuh"
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
 
@@ -142,44 +143,61 @@ struct Arena {
 // ------------------------------------------------------------------ tensor-core GEMM planning
 struct TcPlan {
   int bn, stages, tiles_m, tiles_n, splits, kb_per_split, num_kb;
+  int cta2;   // 1: pairs of CTAs compute 256 x bn tiles (gemm2_kernel); 0: one CTA per 128 x bn tile
 };
 
 constexpr int kSmemBudget = 227 * 1024 - 1024;   // opt-in maximum minus room for the static __shared__ variables
-constexpr int kSmemBarrierBytes = 8 * (2 * tc::kMaxStages + 4);
+constexpr int kSmemBarrierBytes = 8 * (2 * tc::kMaxStages + 5);
 
-// Picks the N tile and the split-K factor by a small cost model: waves over the SMs times
-// (k-blocks per work item x the slower of MMA issue and operand fetch, plus the epilogue).
-TcPlan plan_tc(int64_t M, int64_t N, int64_t K, bool allow_split) {
+inline int env_int(const char* name) { const char* e = getenv(name); return e ? atoi(e) : 0; }
+
+// Picks the tile shape (one CTA: 128 x bn; CTA pair: 256 x bn), and the split-K factor, by a small
+// cost model in SM cycles: waves over the machine x (k-blocks per work item x the slower of MMA
+// issue and shared-memory fill, plus the epilogue).  The fill rate of one SM's shared memory was
+// measured at about 54 bytes per cycle; a 128 x bn x 64 MMA block takes 2*bn cycles.
+// FLOP_TC_BN, FLOP_TC_STAGES, FLOP_TC_CTA2 (1 = force pairs, 2 = forbid pairs) override for tuning.
+TcPlan plan_tc(int64_t M, int64_t N, int64_t K, bool allow_split, bool b_mn_major) {
   const int sms = num_sms();
   const int num_kb = (int)((K + tc::BK - 1) / tc::BK);
+  static const int force_bn = env_int("FLOP_TC_BN"), force_stages = env_int("FLOP_TC_STAGES"), force_cta2 = env_int("FLOP_TC_CTA2");
   TcPlan best{};
   double best_cost = 1e300;
   const int bns[4] = {256, 192, 128, 64};
-  for (int bi = 0; bi < 4; ++bi) {
-    const int bn = bns[bi];
-    if (bn > 64 && bn - 64 >= N) continue;   // a smaller tile already covers N
-    const int tiles_m = (int)((M + tc::BM - 1) / tc::BM), tiles_n = (int)((N + bn - 1) / bn);
-    const int max_split = allow_split ? std::min(num_kb, 32) : 1;
-    for (int s = 1; s <= max_split; ++s) {
-      const int kbps = (num_kb + s - 1) / s;
-      const int splits = (num_kb + kbps - 1) / kbps;
-      if (splits != s) continue;
-      const double items = (double)tiles_m * tiles_n * splits;
-      const double waves = ceil(items / sms);
-      const double mma = 2.0 * bn;                                  // cycles per k-block at full rate
-      const double fetch = (double)tc::stage_bytes(bn) / 80.0;      // cycles per k-block at ~80 B/clk/SM
-      const double epi = 600.0 + 10.0 * bn;
-      double cost = waves * (kbps * std::max(mma, fetch) + epi);
-      if (splits > 1) cost += 0.002 * (double)splits * (double)M * (double)N / sms + 3000.0;   // ordered reduction pass
-      if (cost < best_cost) {
-        best_cost = cost;
-        best.bn = bn; best.tiles_m = tiles_m; best.tiles_n = tiles_n;
-        best.splits = splits; best.kb_per_split = kbps; best.num_kb = num_kb;
+  for (int pass = 0; pass < 2 && best_cost == 1e300; ++pass)   // second pass: overrides that fit no tile are dropped
+  for (int cta2 = 0; cta2 <= 1; ++cta2) {
+    if (pass == 0 && ((force_cta2 == 1 && !cta2) || (force_cta2 == 2 && cta2))) continue;
+    for (int bi = 0; bi < 4; ++bi) {
+      const int bn = bns[bi];
+      const bool forced_bn = pass == 0 && force_bn;
+      if (forced_bn && bn != force_bn) continue;
+      if (!forced_bn && bn > 64 && bn - 64 >= N) continue;   // a smaller tile already covers N
+      if (cta2 && b_mn_major && (bn / 2) % 64 != 0) continue;  // MN-major halves come in 64-wide boxes
+      const int bm = cta2 ? tc::BM2 : tc::BM;
+      const int units = cta2 ? sms / 2 : sms;                 // CTA pairs or CTAs that run at once
+      const int tiles_m = (int)((M + bm - 1) / bm), tiles_n = (int)((N + bn - 1) / bn);
+      const int max_split = allow_split ? std::min(num_kb, 32) : 1;
+      const double bytes = cta2 ? (double)tc::stage_bytes2(bn) : (double)tc::stage_bytes(bn);
+      for (int sp = 1; sp <= max_split; ++sp) {
+        const int kbps = (num_kb + sp - 1) / sp;
+        const int splits = (num_kb + kbps - 1) / kbps;
+        if (splits != sp) continue;
+        const double items = (double)tiles_m * tiles_n * splits;
+        const double waves = ceil(items / units);
+        const double per_kb = std::max(2.0 * bn, bytes / 54.0);
+        const double epi = 600.0 + 10.0 * bn;
+        double cost = waves * (kbps * per_kb + epi) + 3000.0;
+        if (splits > 1) cost += 0.004 * (double)splits * (double)M * (double)N / sms;   // ordered reduction pass
+        if (cost < best_cost) {
+          best_cost = cost;
+          best.bn = bn; best.tiles_m = tiles_m; best.tiles_n = tiles_n; best.cta2 = cta2;
+          best.splits = splits; best.kb_per_split = kbps; best.num_kb = num_kb;
+        }
       }
     }
   }
-  const int sb = (int)tc::stage_bytes(best.bn);
+  const int sb = best.cta2 ? (int)tc::stage_bytes2(best.bn) : (int)tc::stage_bytes(best.bn);
   best.stages = std::min(tc::kMaxStages, (kSmemBudget - 1024 - kSmemBarrierBytes) / sb);
+  if (force_stages > 0) best.stages = std::min(best.stages, force_stages);
   return best;
 }
 
@@ -238,19 +256,33 @@ struct TcEpilogue {
 };
 
 template <bool A_MN, bool B_MN, int EPI>
-int launch_tc_inst(const CUtensorMap& ta, const CUtensorMap& tb, const tc::Params& p, cudaStream_t st) {
+int launch_tc_inst(const CUtensorMap& ta, const CUtensorMap& tb, const tc::Params& p, int cta2, cudaStream_t st) {
   static bool configured = false;
-  auto kern = tc::gemm_kernel<A_MN, B_MN, EPI>;
+  auto kern1 = tc::gemm_kernel<A_MN, B_MN, EPI>;
+  auto kern2 = tc::gemm2_kernel<A_MN, B_MN, EPI>;
   if (!configured) {
-    FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    FLOP_CUDA(cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    FLOP_CUDA(cudaFuncSetAttribute(kern2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     configured = true;
   }
-  const int smem = 1024 + p.stages * (int)tc::stage_bytes(p.bn) + kSmemBarrierBytes;
   const int total = p.tiles_m * p.tiles_n * p.splits;
-  const int grid = std::min(total, num_sms());
-  {
-    GemmTimer timer(st, 2.0 * p.M * (double)p.N * p.K);
-    launch_k(kern, dim3(grid), dim3(tc::kThreads), (size_t)(smem), st, ta, tb, p);
+  GemmTimer timer(st, 2.0 * p.M * (double)p.N * p.K);
+  if (!cta2) {
+    const int smem = 1024 + p.stages * (int)tc::stage_bytes(p.bn) + kSmemBarrierBytes;
+    launch_k(kern1, dim3(std::min(total, num_sms())), dim3(tc::kThreads), (size_t)smem, st, ta, tb, p);
+  } else {
+    const int smem = 1024 + p.stages * (int)tc::stage_bytes2(p.bn) + kSmemBarrierBytes;
+    const int pairs = std::min(total, num_sms() / 2);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_on() ? 2 : 1;
+    cudaLaunchKernelEx(&cfg, kern2, ta, tb, p);
   }
   count_launch();
   FLOP_CUDA(cudaGetLastError());
@@ -264,7 +296,7 @@ int launch_tc(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t 
   CUtensorMap ta, tb;
   if (!A.mn_major) FLOP_TRY(make_tmap(&ta, A.ptr, M, K, A.ld, tc::BK, tc::BM));
   else             FLOP_TRY(make_tmap(&ta, A.ptr, K, M, A.ld, tc::kBoxMN, tc::BK));
-  if (!B.mn_major) FLOP_TRY(make_tmap(&tb, B.ptr, N, K, B.ld, tc::BK, (uint32_t)pl.bn));
+  if (!B.mn_major) FLOP_TRY(make_tmap(&tb, B.ptr, N, K, B.ld, tc::BK, (uint32_t)(pl.cta2 ? pl.bn / 2 : pl.bn)));
   else             FLOP_TRY(make_tmap(&tb, B.ptr, K, N, B.ld, tc::kBoxMN, tc::BK));
   tc::Params p{};
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
@@ -273,9 +305,9 @@ int launch_tc(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t 
   p.out = ep.out; p.ldo = ep.ldo; p.col_scale = ep.col_scale;
   p.slices = ep.slices; p.slice_elems = ep.slice_elems; p.ld_slice = ep.ld_slice;
   p.qdot = ep.qdot; p.ldq = ep.ldq; p.dz_part = ep.dz_part; p.dz_stride = ep.dz_stride;
-  if (!A.mn_major && !B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, false, tc::EPI_STORE>(ta, tb, p, st);
-  if (!A.mn_major && B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, true, tc::EPI_STORE>(ta, tb, p, st);
-  if (A.mn_major && B.mn_major && ep.kind == tc::EPI_SLICE) return launch_tc_inst<true, true, tc::EPI_SLICE>(ta, tb, p, st);
+  if (!A.mn_major && !B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, false, tc::EPI_STORE>(ta, tb, p, pl.cta2, st);
+  if (!A.mn_major && B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, true, tc::EPI_STORE>(ta, tb, p, pl.cta2, st);
+  if (A.mn_major && B.mn_major && ep.kind == tc::EPI_SLICE) return launch_tc_inst<true, true, tc::EPI_SLICE>(ta, tb, p, pl.cta2, st);
   return FLOP_ERR_UNSUPPORTED;
 }
 
@@ -342,8 +374,8 @@ BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, 
   int sp = 1, sq = 1;
   w.n_part = 1;
   if (dt == FLOP_BF16) {
-    w.plan_p = plan_tc(d_out, r, T, true);
-    w.plan_q = plan_tc(r, d_in, T, true);
+    w.plan_p = plan_tc(d_out, r, T, true, true);
+    w.plan_q = plan_tc(r, d_in, T, true, true);
     sp = std::max(1, w.plan_p.splits);
     sq = std::max(1, w.plan_q.splits);
     w.n_part = sq * std::max(1, w.plan_q.tiles_n);
@@ -466,6 +498,43 @@ int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launche
   return FLOP_OK;
 }
 
+int flop_tc_gemm(const void* A, int64_t lda, int a_mn_major, const void* B, int64_t ldb, int b_mn_major, void* D,
+                 int64_t ldd, const float* col_scale, float* slices, int64_t M, int64_t N, int64_t K, int bn, int cta2,
+                 int splits, int* n_slices_out, void* stream) {
+  if (M < 0 || N < 0 || K < 0 || !A || !B) return FLOP_ERR_INVALID_ARG;
+  if (!bf16_ok(A, lda) || !bf16_ok(B, ldb)) return FLOP_ERR_UNSUPPORTED;
+  const bool slice = a_mn_major && b_mn_major;
+  if (a_mn_major && !b_mn_major) return FLOP_ERR_UNSUPPORTED;
+  if (slice ? (slices == nullptr) : (D == nullptr || !bf16_ok(D, ldd) || ldd < N)) return FLOP_ERR_INVALID_ARG;
+  TcPlan pl = plan_tc(M, N, K, slice, b_mn_major != 0);
+  if (bn > 0 || cta2 >= 0 || splits > 0) {   // explicit tile shape
+    if (bn > 0) pl.bn = bn;
+    if (cta2 >= 0) pl.cta2 = cta2;
+    if (pl.bn != 64 && pl.bn != 128 && pl.bn != 192 && pl.bn != 256) return FLOP_ERR_INVALID_ARG;
+    if (pl.cta2 && b_mn_major && (pl.bn / 2) % 64 != 0) return FLOP_ERR_UNSUPPORTED;
+    const int bm = pl.cta2 ? tc::BM2 : tc::BM;
+    pl.tiles_m = (int)((M + bm - 1) / bm);
+    pl.tiles_n = (int)((N + pl.bn - 1) / pl.bn);
+    pl.num_kb = (int)((K + tc::BK - 1) / tc::BK);
+    int sp = splits > 0 ? splits : pl.splits;
+    if (!slice) sp = 1;
+    sp = std::max(1, std::min(sp, std::max(pl.num_kb, 1)));
+    pl.kb_per_split = (pl.num_kb + sp - 1) / sp;
+    pl.splits = pl.kb_per_split > 0 ? (pl.num_kb + pl.kb_per_split - 1) / pl.kb_per_split : 1;
+    const int sb = pl.cta2 ? (int)tc::stage_bytes2(pl.bn) : (int)tc::stage_bytes(pl.bn);
+    pl.stages = std::min(tc::kMaxStages, (kSmemBudget - 1024 - kSmemBarrierBytes) / sb);
+  }
+  TcEpilogue e{};
+  if (slice) {
+    e.kind = tc::EPI_SLICE; e.slices = slices; e.ld_slice = round_up(std::max<int64_t>(N, 1), 4); e.slice_elems = M * e.ld_slice;
+  } else {
+    e = store_epilogue(D, ldd, col_scale);
+  }
+  FLOP_TRY(launch_tc({A, lda, a_mn_major != 0}, {B, ldb, b_mn_major != 0}, M, N, K, pl, e, (cudaStream_t)stream));
+  if (n_slices_out) *n_slices_out = pl.splits;
+  return FLOP_OK;
+}
+
 int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt, size_t* out_bytes) {
   if (!out_bytes || T < 0 || d_in < 0 || d_out < 0 || r < 0 || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
   Arena ar{nullptr, 0, 0};
@@ -513,10 +582,10 @@ static int fwd_impl(const void* X, int64_t ldx, const void* Q, int64_t ldq, cons
       return FLOP_OK;
     }
     // GEMM1: H' = (X Q^T) * z, gate applied to column k in the epilogue
-    const TcPlan p1 = plan_tc(T, r, d_in, false);
+    const TcPlan p1 = plan_tc(T, r, d_in, false, false);
     FLOP_TRY(launch_tc({X, ldx, false}, {Q, ldq, false}, T, r, d_in, p1, store_epilogue(H, ldh, z), st));
     // GEMM2: Y = H' P^T
-    const TcPlan p2 = plan_tc(T, d_out, r, false);
+    const TcPlan p2 = plan_tc(T, d_out, r, false, false);
     FLOP_TRY(launch_tc({H, ldh, false}, {P, ldp, false}, T, d_out, r, p2, store_epilogue(Y, ldy, nullptr), st));
   } else {
     FLOP_TRY(launch_simt((const float*)X, ldx, 1, (const float*)Q, ldq, 1, (float*)H, ldh, T, r, d_in, z, nullptr, 0, st));
@@ -569,9 +638,9 @@ int flop_compact_fwd(const void* X, int64_t ldx, const void* Qc, int64_t ldqc, c
   const FwdWs w = plan_fwd_ws(ar, T, k, dt);
   if (dt == FLOP_BF16) {
     if (!bf16_ok(Y, ldy) || !bf16_ok(X, ldx) || !bf16_ok(Qc, ldqc) || !bf16_ok(Pc, ldpc)) return FLOP_ERR_UNSUPPORTED;
-    const TcPlan p1 = plan_tc(T, k, d_in, false);
+    const TcPlan p1 = plan_tc(T, k, d_in, false, false);
     FLOP_TRY(launch_tc({X, ldx, false}, {Qc, ldqc, false}, T, k, d_in, p1, store_epilogue(w.H, w.ldh, nullptr), st));
-    const TcPlan p2 = plan_tc(T, d_out, k, false);
+    const TcPlan p2 = plan_tc(T, d_out, k, false, false);
     FLOP_TRY(launch_tc({w.H, w.ldh, false}, {Pc, ldpc, false}, T, d_out, k, p2, store_epilogue(Y, ldy, nullptr), st));
   } else {
     FLOP_TRY(launch_simt((const float*)X, ldx, 1, (const float*)Qc, ldqc, 1, (float*)w.H, w.ldh, T, k, d_in, nullptr, nullptr, 0, st));
@@ -621,7 +690,7 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
 
   if (dt == FLOP_BF16) {
     // dH' = dY P            (A = dY K-major over d_out; B(n=k_rank, k=i) = P[i, k_rank]: MN-major)
-    const TcPlan ph = plan_tc(T, r, d_out, false);
+    const TcPlan ph = plan_tc(T, r, d_out, false, true);
     FLOP_TRY(launch_tc({dY, lddy, false}, {P, ldp, true}, T, r, d_out, ph, store_epilogue(w.dH, w.lddh, nullptr), st));
     if (dP) {
       // dP = dY^T H'        (contract over tokens: both operands MN-major), fp32 split-K slices
@@ -656,7 +725,7 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
     }
     if (dX) {
       // dX = dH' (diag(z) Q)   (B(n=j, k=k_rank) = Qz[k_rank, j]: MN-major)
-      const TcPlan px = plan_tc(T, d_in, r, false);
+      const TcPlan px = plan_tc(T, d_in, r, false, true);
       FLOP_TRY(launch_tc({w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, T, d_in, r, px, store_epilogue(dX, lddx, nullptr), st));
     }
   } else {

@@ -170,6 +170,73 @@ __device__ __forceinline__ WorkItem decode(const Params& p, int w) {
   return it;
 }
 
+// One 32-column chunk of one accumulator row (held by this thread) through the epilogue.
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32], int row, bool row_ok, int n0, int split,
+                                               float& dot) {
+    const bool full_chunk = n0 + 32 <= p.N;
+    if (EPI == EPI_STORE) {
+      if (row_ok) {
+        __nv_bfloat16* o = p.out + (int64_t)row * p.ldo + n0;
+        if (full_chunk) {
+          uint32_t packed[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float a = __uint_as_float(v[2 * i]), b = __uint_as_float(v[2 * i + 1]);
+            if (p.col_scale) { a *= __ldg(p.col_scale + n0 + 2 * i); b *= __ldg(p.col_scale + n0 + 2 * i + 1); }
+            __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+            packed[i] = *reinterpret_cast<uint32_t*>(&h);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint4*>(o + 8 * i) = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (n0 + i < p.N) {
+              float a = __uint_as_float(v[i]);
+              if (p.col_scale) a *= __ldg(p.col_scale + n0 + i);
+              o[i] = __float2bfloat16_rn(a);
+            }
+          }
+        }
+      }
+    } else {
+      if (row_ok) {
+        float* o = p.slices + (int64_t)split * p.slice_elems + (int64_t)row * p.ld_slice + n0;
+        if (full_chunk) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<uint4*>(o + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (n0 + i < p.N) o[i] = __uint_as_float(v[i]);
+        }
+        if (p.qdot) {
+          const __nv_bfloat16* qr = p.qdot + (int64_t)row * p.ldq + n0;
+          if (full_chunk) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint4 raw = __ldg(reinterpret_cast<const uint4*>(qr + 8 * i));
+              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 f = __bfloat1622float2(h[j]);
+                dot = fmaf(__uint_as_float(v[8 * i + 2 * j]), f.x, dot);
+                dot = fmaf(__uint_as_float(v[8 * i + 2 * j + 1]), f.y, dot);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+          }
+        }
+      }
+    }
+}
+
 template <bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
@@ -305,67 +372,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         uint32_t v[32];
         tmem_ld32(t_row + (uint32_t)(c * 32), v);
         tmem_ld_wait();
-        const bool full_chunk = n0 + 32 <= p.N;
-        if (EPI == EPI_STORE) {
-          if (row_ok) {
-            __nv_bfloat16* o = p.out + (int64_t)row * p.ldo + n0;
-            if (full_chunk) {
-              uint32_t packed[16];
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                float a = __uint_as_float(v[2 * i]), b = __uint_as_float(v[2 * i + 1]);
-                if (p.col_scale) { a *= __ldg(p.col_scale + n0 + 2 * i); b *= __ldg(p.col_scale + n0 + 2 * i + 1); }
-                __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-                packed[i] = *reinterpret_cast<uint32_t*>(&h);
-              }
-#pragma unroll
-              for (int i = 0; i < 4; ++i)
-                *reinterpret_cast<uint4*>(o + 8 * i) = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                if (n0 + i < p.N) {
-                  float a = __uint_as_float(v[i]);
-                  if (p.col_scale) a *= __ldg(p.col_scale + n0 + i);
-                  o[i] = __float2bfloat16_rn(a);
-                }
-              }
-            }
-          }
-        } else {
-          if (row_ok) {
-            float* o = p.slices + (int64_t)it.split * p.slice_elems + (int64_t)row * p.ld_slice + n0;
-            if (full_chunk) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                *reinterpret_cast<uint4*>(o + 4 * i) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (n0 + i < p.N) o[i] = __uint_as_float(v[i]);
-            }
-            if (p.qdot) {
-              const __nv_bfloat16* qr = p.qdot + (int64_t)row * p.ldq + n0;
-              if (full_chunk) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(qr + 8 * i));
-                  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    const float2 f = __bfloat1622float2(h[j]);
-                    dot = fmaf(__uint_as_float(v[8 * i + 2 * j]), f.x, dot);
-                    dot = fmaf(__uint_as_float(v[8 * i + 2 * j + 1]), f.y, dot);
-                  }
-                }
-              } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
-              }
-            }
-          }
-        }
+        epilogue_chunk<EPI>(p, v, row, row_ok, n0, it.split, dot);
       }
       if (EPI == EPI_SLICE && p.qdot && row_ok)
         p.dz_part[(int64_t)(it.split * p.tiles_n + it.tn) * p.dz_stride + row] = dot;
