@@ -104,7 +104,7 @@ class ClockSampler:
 class Job:
     """Device state of one workload: inputs, outputs and scratch of every matrix."""
 
-    def __init__(self, w: I.Workload, device, seed: int, n_streams: int = 1):
+    def __init__(self, w: I.Workload, device, seed: int, n_streams: int = 1, group: int = 0):
         import torch
         from paper_1910_04732_b200 import binding as b
         self.w, self.b, self.torch = w, b, torch
@@ -152,6 +152,21 @@ class Job:
         self.ws = self.wss[0]
         self.ev_gates = torch.cuda.Event()
         self.ev_done = [torch.cuda.Event() for _ in range(self.n_streams)]
+        # grouped issue: `group` consecutive matrices (default: the matrices of one layer) per call,
+        # every matrix with its own scratch; the argument arrays are built once
+        self.group = group
+        self.groups = []
+        if group > 0:
+            for e in self.mats:
+                e["ws"] = b.alloc_workspace(b.workspace_bytes(b.OP_BWD, w.T, e["m"].d_in, e["m"].d_out, e["m"].r, b.BF16), device)
+            for i in range(0, len(self.mats), group):
+                chunk = self.mats[i:i + group]
+                fwd = b.problem_array([b.fwd_problem(e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]], e["Y"], e["H"])
+                                       for e in chunk])
+                bwd = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]],
+                                                     self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
+                                                     self.dlog_alpha[e["lo"]:e["hi"]], e["ws"]) for e in chunk])
+                self.groups.append((fwd, bwd))
         self.ws_l0 = b.alloc_workspace(b.workspace_bytes(b.OP_L0, self.n_gates, 0, 0, len(sizes), b.F32), device)
         self.step_no = 0
         self.world = 1
@@ -182,7 +197,11 @@ class Job:
     def step(self):
         torch = self.torch
         self.sample_gates()
-        if self.n_streams == 1:
+        if self.group > 0:
+            for fwd, bwd in self.groups:
+                self.b.gated_lowrank_fwd_grouped(fwd)
+                self.b.gated_lowrank_bwd_grouped(bwd)
+        elif self.n_streams == 1:
             for e in self.mats:
                 self.run_matrix(e)
         else:
@@ -330,6 +349,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--group", type=int, default=-1, help="matrices per grouped call (0: one call per matrix; default: one layer)")
     ap.add_argument("--streams", type=int, default=1, help="streams over which independent matrices are issued")
     args = ap.parse_args()
     w = I.WORKLOADS[args.workload]
@@ -355,7 +375,8 @@ def main():
     from paper_1910_04732_b200 import binding as b
     b.load_library()
 
-    job = Job(w, torch.device("cuda", local), seed=1234 + rank, n_streams=args.streams)
+    group = len(w.matrices) if args.group < 0 else args.group
+    job = Job(w, torch.device("cuda", local), seed=1234 + rank, n_streams=args.streams, group=group)
     job.world = world
     for _ in range(args.warmup):
         job.step()
@@ -401,7 +422,7 @@ def main():
         "pct_of_bf16_peak_measured_sustained": 100.0 * tflops / world / peaks["bf16_tflops_sustained"],
         "config": {"workload": w.name, "T": w.T, "layers": w.layers,
                    "matrices": [[m.name, m.d_in, m.d_out, m.r] for m in w.matrices],
-                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}", "streams": args.streams,
+                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}", "streams": args.streams, "matrices_per_grouped_call": group,
                    "l2": f"inputs larger than L2: {job.input_bytes() / 1e6:.0f} MB of X and dY per step, each matrix its own buffers"},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": peaks["bf16_tflops_sustained"],

@@ -141,6 +141,35 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
                            int64_t d_out, int64_t r, int dt, int wgrad_dt, void* ws,
                            size_t ws_bytes, void* stream);
 
+/* Grouped forms: n independent problems (different weight matrices, e.g. the
+ * Q/K/V projections that share an input, or all matrices of a layer whose weight
+ * gradients are due together) run through the SAME sequence of kernels as n single
+ * calls, but each GEMM stage is one persistent launch over the tiles of all problems,
+ * so pipeline fill, epilogue drain and launch gaps are paid once per stage instead
+ * of once per matrix (Section 4.1's products, batched).  Results match the single
+ * calls within the storage-type tolerance (tile shapes and split-K factors may
+ * differ).  `problems` is a HOST array; the pointers inside follow the conventions of
+ * the single calls.  Forward: H_save is required (there is no scratch argument).
+ * Backward: every problem brings its own workspace of at least
+ * flop_workspace_bytes(FLOP_OP_BWD, ...) bytes; workspaces must not overlap. */
+typedef struct {
+  const void* X; int64_t ldx; const void* Q; int64_t ldq; const void* P; int64_t ldp;
+  const float* z; void* Y; int64_t ldy; void* H_save; int64_t ldh;
+  int64_t T, d_in, d_out, r;
+} flop_fwd_problem_t;
+
+typedef struct {
+  const void* dY; int64_t lddy; const void* X; int64_t ldx; const void* Q; int64_t ldq;
+  const void* P; int64_t ldp; const float* z; const float* dz_dla; const void* H_save; int64_t ldh;
+  void* dX; int64_t lddx; void* dP; int64_t lddp; void* dQ; int64_t lddq; float* dlog_alpha;
+  int64_t T, d_in, d_out, r;
+  void* ws; size_t ws_bytes;
+} flop_bwd_problem_t;
+
+int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* problems, int n, int dt, void* stream);
+int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* problems, int n, int accumulate, int dt,
+                                   int wgrad_dt, void* stream);
+
 /* Expected size and augmented-Lagrangian penalty over all gates of all
  * matrices at once (Eq. 3 and Section 4.3).  Segment i (one weight matrix)
  * owns gates seg_off[i]..seg_off[i+1]-1 of log_alpha; each of its gates

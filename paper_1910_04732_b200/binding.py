@@ -22,13 +22,31 @@ OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 
 EXPORTS = ("flop_status_string", "flop_device_status", "flop_launch_count", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample",
-           "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_expected_l0_lagrangian",
+           "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
+           "flop_gated_lowrank_bwd_grouped", "flop_expected_l0_lagrangian",
            "flop_expected_l0_lagrangian_noalloc",
            "flop_compact_ranks", "flop_compact_fwd")
 
 
 class HcParams(ctypes.Structure):
     _fields_ = [("beta", ctypes.c_float), ("gamma", ctypes.c_float), ("zeta", ctypes.c_float)]
+
+
+class FwdProblem(ctypes.Structure):
+    _fields_ = [("X", ctypes.c_void_p), ("ldx", ctypes.c_int64), ("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64),
+                ("P", ctypes.c_void_p), ("ldp", ctypes.c_int64), ("z", ctypes.c_void_p), ("Y", ctypes.c_void_p),
+                ("ldy", ctypes.c_int64), ("H_save", ctypes.c_void_p), ("ldh", ctypes.c_int64),
+                ("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64)]
+
+
+class BwdProblem(ctypes.Structure):
+    _fields_ = [("dY", ctypes.c_void_p), ("lddy", ctypes.c_int64), ("X", ctypes.c_void_p), ("ldx", ctypes.c_int64),
+                ("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64), ("P", ctypes.c_void_p), ("ldp", ctypes.c_int64),
+                ("z", ctypes.c_void_p), ("dz_dla", ctypes.c_void_p), ("H_save", ctypes.c_void_p), ("ldh", ctypes.c_int64),
+                ("dX", ctypes.c_void_p), ("lddx", ctypes.c_int64), ("dP", ctypes.c_void_p), ("lddp", ctypes.c_int64),
+                ("dQ", ctypes.c_void_p), ("lddq", ctypes.c_int64), ("dlog_alpha", ctypes.c_void_p),
+                ("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
+                ("ws", ctypes.c_void_p), ("ws_bytes", ctypes.c_size_t)]
 
 
 class FlopError(RuntimeError):
@@ -65,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.flop_gated_lowrank_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, i64,
                                            vp, i64, vp, i64, vp, i64, vp, ci,
                                            i64, i64, i64, i64, ci, ci, vp, sz, vp]
+    lib.flop_gated_lowrank_fwd_grouped.argtypes = [ctypes.POINTER(FwdProblem), ci, ci, vp]
+    lib.flop_gated_lowrank_bwd_grouped.argtypes = [ctypes.POINTER(BwdProblem), ci, ci, ci, ci, vp]
     lib.flop_expected_l0_lagrangian.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp,
                                                 vp, sz, vp]
     lib.flop_expected_l0_lagrangian_noalloc.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp, vp]
@@ -187,6 +207,42 @@ def gated_lowrank_bwd(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws
         _ptr(dQ), _ld(dQ) if dQ is not None else 0, _ptr(dlog_alpha), int(accumulate),
         T, d_in, d_out, r, _dt(X), wdt, _ptr(ws), ws.numel() if ws is not None else 0, _stream()),
         "flop_gated_lowrank_bwd")
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def fwd_problem(X, Q, P, z, Y, H_save) -> FwdProblem:
+    T, d_in = X.shape
+    d_out, r = P.shape
+    return FwdProblem(_p(X), _ld(X), _p(Q), _ld(Q), _p(P), _ld(P), _p(z), _p(Y), _ld(Y), _p(H_save), _ld(H_save),
+                      T, d_in, d_out, r)
+
+
+def bwd_problem(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws) -> BwdProblem:
+    T, d_in = X.shape
+    d_out, r = P.shape
+    ld = lambda t: _ld(t) if t is not None else 0
+    return BwdProblem(_p(dY), _ld(dY), _p(X), _ld(X), _p(Q), _ld(Q), _p(P), _ld(P), _p(z), _p(dz_dla), _p(H_save),
+                      _ld(H_save), _p(dX), ld(dX), _p(dP), ld(dP), _p(dQ), ld(dQ), _p(dlog_alpha), T, d_in, d_out, r,
+                      _p(ws), ws.numel() if ws is not None else 0)
+
+
+def problem_array(problems):
+    """ctypes array of FwdProblem / BwdProblem; build it once and reuse it when the pointers do not change."""
+    return (type(problems[0]) * len(problems))(*problems)
+
+
+def gated_lowrank_fwd_grouped(problems, dt: int = BF16) -> None:
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_gated_lowrank_fwd_grouped(arr, len(arr), dt, _stream()), "flop_gated_lowrank_fwd_grouped")
+
+
+def gated_lowrank_bwd_grouped(problems, accumulate: bool = False, dt: int = BF16, wgrad_dt: int = BF16) -> None:
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_gated_lowrank_bwd_grouped(arr, len(arr), int(accumulate), dt, wgrad_dt, _stream()),
+           "flop_gated_lowrank_bwd_grouped")
 
 
 def expected_l0_lagrangian(log_alpha, seg_off, seg_size, hc, target, lam, out4, seg_expected=None,

@@ -21,6 +21,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
+#include "gemm_tc_group.cuh"
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
 
@@ -156,7 +157,7 @@ inline int env_int(const char* name) { const char* e = getenv(name); return e ? 
 // issue and shared-memory fill, plus the epilogue).  The fill rate of one SM's shared memory was
 // measured at about 54 bytes per cycle; a 128 x bn x 64 MMA block takes 2*bn cycles.
 // FLOP_TC_BN, FLOP_TC_STAGES, FLOP_TC_CTA2 (1 = force pairs, 2 = forbid pairs) override for tuning.
-TcPlan plan_tc(int64_t M, int64_t N, int64_t K, bool allow_split, bool b_mn_major) {
+TcPlan plan_tc(int64_t M, int64_t N, int64_t K, bool allow_split, bool b_mn_major, bool allow_cta2 = true) {
   const int sms = num_sms();
   const int num_kb = (int)((K + tc::BK - 1) / tc::BK);
   static const int force_bn = env_int("FLOP_TC_BN"), force_stages = env_int("FLOP_TC_STAGES"), force_cta2 = env_int("FLOP_TC_CTA2");
@@ -165,7 +166,8 @@ TcPlan plan_tc(int64_t M, int64_t N, int64_t K, bool allow_split, bool b_mn_majo
   const int bns[4] = {256, 192, 128, 64};
   for (int pass = 0; pass < 2 && best_cost == 1e300; ++pass)   // second pass: overrides that fit no tile are dropped
   for (int cta2 = 0; cta2 <= 1; ++cta2) {
-    if (pass == 0 && ((force_cta2 == 1 && !cta2) || (force_cta2 == 2 && cta2))) continue;
+    if (cta2 && !allow_cta2) continue;
+    if (pass == 0 && allow_cta2 && ((force_cta2 == 1 && !cta2) || (force_cta2 == 2 && cta2))) continue;
     for (int bi = 0; bi < 4; ++bi) {
       const int bn = bns[bi];
       const bool forced_bn = pass == 0 && force_bn;
@@ -317,6 +319,74 @@ TcEpilogue store_epilogue(void* out, int64_t ldo, const float* col_scale) {
   return e;
 }
 
+// ---- grouped launches: several independent GEMMs of the same kind in one persistent kernel
+struct TcJob {
+  Operand A, B;
+  int64_t M, N, K;
+  TcPlan pl;       // one-CTA plan (pl.cta2 == 0)
+  TcEpilogue ep;
+};
+
+template <bool A_MN, bool B_MN, int EPI>
+int launch_group_inst(const tc::GroupParams& gp, double flops, cudaStream_t st) {
+  static bool configured = false;
+  auto kern = tc::gemm_group_kernel<A_MN, B_MN, EPI>;
+  if (!configured) {
+    FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    configured = true;
+  }
+  const int smem = 1024 + gp.stages * (int)tc::stage_bytes(gp.bn_max) + kSmemBarrierBytes;
+  {
+    GemmTimer timer(st, flops);
+    launch_k(kern, dim3(std::min(gp.total_work, num_sms())), dim3(tc::kThreads), (size_t)smem, st, gp);
+  }
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
+  size_t i = 0;
+  while (i < jobs.size()) {
+    tc::GroupParams gp;
+    memset(&gp, 0, sizeof(gp));
+    double flops = 0.0;
+    const TcJob& first = jobs[i];
+    for (; i < jobs.size() && gp.n < tc::kMaxGroup; ++i) {
+      const TcJob& j = jobs[i];
+      if (j.M <= 0 || j.N <= 0 || j.K <= 0) continue;
+      if (j.M > INT32_MAX || j.N > INT32_MAX || j.K > INT32_MAX || j.pl.cta2) return FLOP_ERR_UNSUPPORTED;
+      if (j.A.mn_major != first.A.mn_major || j.B.mn_major != first.B.mn_major || j.ep.kind != first.ep.kind) return FLOP_ERR_INVALID_ARG;
+      tc::GroupProblem& pr = gp.prob[gp.n];
+      if (!j.A.mn_major) FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.M, j.K, j.A.ld, tc::BK, tc::BM));
+      else               FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.K, j.M, j.A.ld, tc::kBoxMN, tc::BK));
+      if (!j.B.mn_major) FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.N, j.K, j.B.ld, tc::BK, (uint32_t)j.pl.bn));
+      else               FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.K, j.N, j.B.ld, tc::kBoxMN, tc::BK));
+      tc::Params& p = pr.p;
+      p.M = (int)j.M; p.N = (int)j.N; p.K = (int)j.K;
+      p.bn = j.pl.bn; p.stages = 0; p.tiles_m = j.pl.tiles_m; p.tiles_n = j.pl.tiles_n;
+      p.splits = j.pl.splits; p.kb_per_split = j.pl.kb_per_split; p.num_kb = j.pl.num_kb;
+      p.out = j.ep.out; p.ldo = j.ep.ldo; p.col_scale = j.ep.col_scale;
+      p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
+      p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
+      pr.work_begin = gp.total_work;
+      gp.total_work += p.tiles_m * p.tiles_n * p.splits;
+      gp.bn_max = std::max(gp.bn_max, p.bn);
+      flops += 2.0 * j.M * (double)j.N * j.K;
+      ++gp.n;
+    }
+    if (gp.n == 0) continue;
+    gp.stages = std::min(tc::kMaxStages, (kSmemBudget - 1024 - kSmemBarrierBytes) / (int)tc::stage_bytes(gp.bn_max));
+    const bool a_mn = first.A.mn_major, b_mn = first.B.mn_major;
+    int rc = FLOP_ERR_UNSUPPORTED;
+    if (!a_mn && !b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, false, tc::EPI_STORE>(gp, flops, st);
+    else if (!a_mn && b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, true, tc::EPI_STORE>(gp, flops, st);
+    else if (a_mn && b_mn && first.ep.kind == tc::EPI_SLICE) rc = launch_group_inst<true, true, tc::EPI_SLICE>(gp, flops, st);
+    FLOP_TRY(rc);
+  }
+  return FLOP_OK;
+}
+
 int launch_simt(const float* A, int64_t a_sm, int64_t a_sk, const float* B, int64_t b_sn, int64_t b_sk, float* C,
                 int64_t ldc, int64_t M, int64_t N, int64_t K, const float* col_scale, const float* row_scale,
                 int accumulate, cudaStream_t st) {
@@ -363,7 +433,7 @@ struct BwdWs {
   TcPlan plan_p, plan_q;
   size_t bytes;
 };
-BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt) {
+BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt, bool grouped = false) {
   BwdWs w{};
   w.lddh = round_up(std::max<int64_t>(r, 1), 8);
   w.dH = ar.take((size_t)T * w.lddh * elt(dt));
@@ -374,11 +444,11 @@ BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, 
   int sp = 1, sq = 1;
   w.n_part = 1;
   if (dt == FLOP_BF16) {
-    w.plan_p = plan_tc(d_out, r, T, true, true);
-    w.plan_q = plan_tc(r, d_in, T, true, true);
+    w.plan_p = plan_tc(d_out, r, T, true, true, !grouped);
+    w.plan_q = plan_tc(r, d_in, T, true, true, !grouped);
     sp = std::max(1, w.plan_p.splits);
     sq = std::max(1, w.plan_q.splits);
-    w.n_part = sq * std::max(1, w.plan_q.tiles_n);
+    w.n_part = 2 * sq * std::max(1, w.plan_q.tiles_n);   // per split, N tile and epilogue-warp half
   }
   w.slice_elems_p = d_out * w.ld_slice_p;
   w.slice_elems_q = r * w.ld_slice_q;
@@ -541,7 +611,13 @@ int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t
   switch (op) {
     case FLOP_OP_FWD:
     case FLOP_OP_COMPACT_FWD: plan_fwd_ws(ar, T, r, dt); break;
-    case FLOP_OP_BWD: plan_bwd_ws(ar, T, d_in, d_out, r, dt); break;
+    case FLOP_OP_BWD: {   // large enough for the single call and for the grouped call (their split-K plans may differ)
+      Arena g{nullptr, 0, 0};
+      plan_bwd_ws(ar, T, d_in, d_out, r, dt, false);
+      plan_bwd_ws(g, T, d_in, d_out, r, dt, true);
+      ar.used = std::max(ar.used, g.used);
+      break;
+    }
     case FLOP_OP_L0: ar.used = l0_ws_bytes(T, r); break;
     case FLOP_OP_COMPACT: ar.used = 0; break;
     default: return FLOP_ERR_INVALID_ARG;
@@ -755,6 +831,126 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
       FLOP_TRY(launch_simt(dHf, w.lddh, 1, (const float*)w.Qz, 1, w.ldqz, (float*)dX, lddx, T, d_in, r, nullptr, nullptr, 0, st));
     }
   }
+  return FLOP_OK;
+}
+
+int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, void* stream) {
+  if (n < 0 || (n > 0 && !pr) || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  bool grouped = dt == FLOP_BF16;
+  for (int i = 0; i < n; ++i) {
+    const flop_fwd_problem_t& a = pr[i];
+    if (a.T < 0 || a.d_in < 0 || a.d_out < 0 || a.r < 0) return FLOP_ERR_INVALID_ARG;
+    if (a.T > 0 && a.r > 0 && !a.H_save) return FLOP_ERR_INVALID_ARG;   // the grouped call has no scratch: H' goes to H_save
+    if (a.T == 0 || a.d_in == 0 || a.d_out == 0 || a.r == 0) grouped = false;
+  }
+  if (!grouped) {   // fp32 storage or an empty problem: one call per problem
+    for (int i = 0; i < n; ++i) {
+      const flop_fwd_problem_t& a = pr[i];
+      FLOP_TRY(flop_gated_lowrank_fwd(a.X, a.ldx, a.Q, a.ldq, a.P, a.ldp, a.z, a.Y, a.ldy, a.H_save, a.ldh, a.T, a.d_in, a.d_out,
+                                      a.r, dt, nullptr, 0, stream));
+    }
+    return FLOP_OK;
+  }
+  std::vector<TcJob> g1, g2;
+  for (int i = 0; i < n; ++i) {
+    const flop_fwd_problem_t& a = pr[i];
+    if (!check_mat(a.Y, a.ldy, a.d_out) || !a.z || !check_mat(a.P, a.ldp, a.r) || !check_mat(a.X, a.ldx, a.d_in) ||
+        !check_mat(a.Q, a.ldq, a.d_in) || a.ldh < a.r)
+      return FLOP_ERR_INVALID_ARG;
+    if (!bf16_ok(a.Y, a.ldy) || !bf16_ok(a.P, a.ldp) || !bf16_ok(a.H_save, a.ldh) || !bf16_ok(a.X, a.ldx) || !bf16_ok(a.Q, a.ldq))
+      return FLOP_ERR_UNSUPPORTED;
+    g1.push_back({{a.X, a.ldx, false}, {a.Q, a.ldq, false}, a.T, a.r, a.d_in, plan_tc(a.T, a.r, a.d_in, false, false, false),
+                  store_epilogue(a.H_save, a.ldh, a.z)});
+    g2.push_back({{a.H_save, a.ldh, false}, {a.P, a.ldp, false}, a.T, a.d_out, a.r, plan_tc(a.T, a.d_out, a.r, false, false, false),
+                  store_epilogue(a.Y, a.ldy, nullptr)});
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  FLOP_TRY(launch_tc_group(g1, st));   // H' = (X Q^T) * z for every problem
+  FLOP_TRY(launch_tc_group(g2, st));   // Y = H' P^T
+  return FLOP_OK;
+}
+
+int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accumulate, int dt, int wgrad_dt, void* stream) {
+  if (n < 0 || (n > 0 && !pr) || !valid_dt(dt) || !valid_dt(wgrad_dt)) return FLOP_ERR_INVALID_ARG;
+  if (dt == FLOP_F32 && wgrad_dt != FLOP_F32) return FLOP_ERR_UNSUPPORTED;
+  bool grouped = dt == FLOP_BF16;
+  for (int i = 0; i < n; ++i) {
+    const flop_bwd_problem_t& a = pr[i];
+    if (a.T < 0 || a.d_in < 0 || a.d_out < 0 || a.r < 0) return FLOP_ERR_INVALID_ARG;
+    if (a.T == 0 || a.d_in == 0 || a.d_out == 0 || a.r == 0) grouped = false;
+  }
+  if (!grouped) {
+    for (int i = 0; i < n; ++i) {
+      const flop_bwd_problem_t& a = pr[i];
+      FLOP_TRY(flop_gated_lowrank_bwd(a.dY, a.lddy, a.X, a.ldx, a.Q, a.ldq, a.P, a.ldp, a.z, a.dz_dla, a.H_save, a.ldh, a.dX,
+                                      a.lddx, a.dP, a.lddp, a.dQ, a.lddq, a.dlog_alpha, accumulate, a.T, a.d_in, a.d_out, a.r, dt,
+                                      wgrad_dt, a.ws, a.ws_bytes, stream));
+    }
+    return FLOP_OK;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  std::vector<TcJob> g3, g4, g5, g6;
+  std::vector<BwdFinishArgs> fin;
+  for (int i = 0; i < n; ++i) {
+    const flop_bwd_problem_t& a = pr[i];
+    if ((a.dX && a.lddx < a.d_in) || (a.dP && a.lddp < a.r) || (a.dQ && a.lddq < a.d_in) || (a.dlog_alpha && !a.dz_dla))
+      return FLOP_ERR_INVALID_ARG;
+    if (!check_mat(a.dY, a.lddy, a.d_out) || !check_mat(a.X, a.ldx, a.d_in) || !check_mat(a.Q, a.ldq, a.d_in) ||
+        !check_mat(a.P, a.ldp, a.r) || !a.z || !check_mat(a.H_save, a.ldh, a.r))
+      return FLOP_ERR_INVALID_ARG;
+    if ((a.dX && !bf16_ok(a.dX, a.lddx)) || !bf16_ok(a.dY, a.lddy) || !bf16_ok(a.X, a.ldx) || !bf16_ok(a.Q, a.ldq) ||
+        !bf16_ok(a.P, a.ldp) || !bf16_ok(a.H_save, a.ldh))
+      return FLOP_ERR_UNSUPPORTED;
+    Arena probe{nullptr, 0, 0};
+    FLOP_TRY(check_ws(a.ws, a.ws_bytes, plan_bwd_ws(probe, a.T, a.d_in, a.d_out, a.r, dt, true).bytes));
+    Arena ar{(unsigned char*)a.ws, a.ws_bytes, 0};
+    const BwdWs w = plan_bwd_ws(ar, a.T, a.d_in, a.d_out, a.r, dt, true);
+    const bool need_m = a.dQ || a.dlog_alpha;
+    g3.push_back({{a.dY, a.lddy, false}, {a.P, a.ldp, true}, a.T, a.r, a.d_out, plan_tc(a.T, a.r, a.d_out, false, true, false),
+                  store_epilogue(w.dH, w.lddh, nullptr)});
+    if (a.dP) {
+      TcEpilogue e{};
+      e.kind = tc::EPI_SLICE; e.slices = w.slices_p; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
+      g4.push_back({{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, w.plan_p, e});
+    }
+    if (need_m) {
+      TcEpilogue e{};
+      e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
+      if (a.dlog_alpha) { e.qdot = (const bf16*)a.Q; e.ldq = a.ldq; e.dz_part = w.dz_part; e.dz_stride = a.r; }
+      g5.push_back({{w.dH, w.lddh, true}, {a.X, a.ldx, true}, a.r, a.d_in, a.T, w.plan_q, e});
+    }
+    BwdFinishArgs f{};
+    f.slices_p = w.slices_p; f.n_slices_p = w.plan_p.splits; f.slice_elems_p = w.slice_elems_p; f.ld_slice_p = w.ld_slice_p;
+    f.d_out = (int)a.d_out; f.r = (int)a.r; f.dP = a.dP; f.lddp = a.lddp;
+    f.slices_q = w.slices_q; f.n_slices_q = w.plan_q.splits; f.slice_elems_q = w.slice_elems_q; f.ld_slice_q = w.ld_slice_q;
+    f.d_in = (int)a.d_in; f.dQ = a.dQ; f.lddq = a.lddq; f.z = a.z;
+    f.Q = (const bf16*)a.Q; f.ldq = a.ldq; f.Qz = a.dX ? (bf16*)w.Qz : nullptr; f.ldqz = w.ldqz;
+    f.dz_part = w.dz_part; f.n_part = w.n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.dlog_alpha; f.accumulate = accumulate;
+    fin.push_back(f);
+    if (a.dX)
+      g6.push_back({{w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, a.T, a.d_in, a.r, plan_tc(a.T, a.d_in, a.r, false, true, false),
+                    store_epilogue(a.dX, a.lddx, nullptr)});
+  }
+  FLOP_TRY(launch_tc_group(g3, st));   // dH' = dY P
+  FLOP_TRY(launch_tc_group(g4, st));   // dY^T H' slices
+  FLOP_TRY(launch_tc_group(g5, st));   // dH'^T X slices + fused <Q, .> row dots
+  for (size_t i = 0; i < fin.size(); i += kFinishGroup) {
+    BwdFinishGroup g;
+    memset(&g, 0, sizeof(g));
+    for (; g.n < kFinishGroup && i + g.n < fin.size(); ++g.n) {
+      g.a[g.n] = fin[i + g.n];
+      g.unit_begin[g.n + 1] = g.unit_begin[g.n] + bwd_finish_units(g.a[g.n]);
+    }
+    const int64_t units = g.unit_begin[g.n];
+    if (units > 0) {
+      const int grid = (int)std::min<int64_t>((units + 255) / 256, (int64_t)num_sms() * 8);
+      if (wgrad_dt == FLOP_BF16) launch_k(bwd_finish_group_kernel<bf16>, dim3(grid), dim3(256), (size_t)0, st, g);
+      else                       launch_k(bwd_finish_group_kernel<float>, dim3(grid), dim3(256), (size_t)0, st, g);
+      count_launch();
+      FLOP_CUDA(cudaGetLastError());
+    }
+  }
+  FLOP_TRY(launch_tc_group(g6, st));   // dX = dH' (diag(z) Q)
   return FLOP_OK;
 }
 

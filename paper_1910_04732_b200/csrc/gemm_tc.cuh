@@ -30,7 +30,8 @@ namespace tc {
 constexpr int BM = 128;          // rows of D per tile = TMEM lanes
 constexpr int BK = 64;           // K per stage = one 128-byte swizzle row of bf16
 constexpr int UMMA_K = 16;
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;                 // two warps per TMEM lane quarter, each takes every other 32-column chunk
+constexpr int kThreads = 64 + 32 * kEpiWarps;  // warp 0: TMA, warp 1: MMA, warps 2..9: epilogue
 constexpr int kMaxStages = 8;
 constexpr uint32_t kATileBytes = BM * BK * 2;     // 16 KB
 constexpr uint32_t kBoxMN = 64;                   // MN-major operands arrive in 64(mn) x 64(k) boxes
@@ -237,6 +238,53 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
     }
 }
 
+// Epilogue of one accumulator tile for one epilogue warp.  Lane quarter q = warp & 3 fixes the
+// 32 accumulator rows this warp may read; h = 0/1 picks the even or odd 32-column chunks.  Two
+// chunks are fetched from tensor memory per wait, and the accumulator is handed back to the MMA
+// warp (arrive on `release_bar`, a CTA-local or cluster address) as soon as the last fetch has
+// landed in registers, before the conversion and the global stores.
+template <int EPI, bool kClusterArrive>
+__device__ __forceinline__ void run_epilogue(const Params& p, uint32_t t_acc, int row0, int n_base, int split, int tn,
+                                             int warp, int lane, uint32_t release_bar) {
+  const int q = warp & 3, h = (warp - 2) >> 2;
+  const int row = row0 + q * 32 + lane;
+  const bool row_ok = row < p.M;
+  const uint32_t t_row = t_acc + ((uint32_t)(q * 32) << 16);
+  int nchunks = (min(p.bn, p.N - n_base) + 31) >> 5;      // chunks that hold columns of D
+  const int mine = (nchunks - h + 1) >> 1;                // chunks h, h+2, ... of this warp
+  float dot = 0.f;
+  bool released = false;
+  for (int i = 0; i < mine; i += 2) {
+    const int c0 = h + 2 * i, c1 = c0 + 2;
+    const bool two = i + 1 < mine;
+    uint32_t v0[32], v1[32];
+    tmem_ld32(t_row + (uint32_t)(c0 * 32), v0);
+    if (two) tmem_ld32(t_row + (uint32_t)(c1 * 32), v1);
+    tmem_ld_wait();
+    if (i + 2 >= mine) {
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (kClusterArrive) asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(release_bar) : "memory");
+        else mbar_arrive(release_bar);
+      }
+      released = true;
+    }
+    epilogue_chunk<EPI>(p, v0, row, row_ok, n_base + c0 * 32, split, dot);
+    if (two) epilogue_chunk<EPI>(p, v1, row, row_ok, n_base + c1 * 32, split, dot);
+  }
+  if (!released) {   // this warp had no chunk in the tile
+    tcgen05_fence_before();
+    __syncwarp();
+    if (lane == 0) {
+      if (kClusterArrive) asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(release_bar) : "memory");
+      else mbar_arrive(release_bar);
+    }
+  }
+  if (EPI == EPI_SLICE && p.qdot && row_ok)
+    p.dz_part[(int64_t)((split * p.tiles_n + tn) * 2 + h) * p.dz_stride + row] = dot;
+}
+
 template <bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
@@ -258,7 +306,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   if (threadIdx.x == 0) {
     s_abort = 0;
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kEpiWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tmap_a);
     prefetch_tmap(&tmap_b);
@@ -351,7 +399,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------ epilogue warps
-    const int q = warp & 3;                    // TMEM lane quarter this warp may read
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -361,24 +408,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      const int row = it.tm * BM + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      const int n_base = it.tn * p.bn;
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.bn);
-      float dot = 0.f;
-      for (int c = 0; c < p.bn / 32; ++c) {
-        const int n0 = n_base + c * 32;
-        if (n0 >= p.N) break;                  // uniform across the warp
-        uint32_t v[32];
-        tmem_ld32(t_row + (uint32_t)(c * 32), v);
-        tmem_ld_wait();
-        epilogue_chunk<EPI>(p, v, row, row_ok, n0, it.split, dot);
-      }
-      if (EPI == EPI_SLICE && p.qdot && row_ok)
-        p.dz_part[(int64_t)(it.split * p.tiles_n + it.tn) * p.dz_stride + row] = dot;
-      tcgen05_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      run_epilogue<EPI, false>(p, tmem_base + (uint32_t)(acc * p.bn), it.tm * BM, it.tn * p.bn, it.split, it.tn, warp, lane,
+                               tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }

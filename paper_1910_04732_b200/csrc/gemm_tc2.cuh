@@ -13,7 +13,7 @@
 //   empty[s]   one per CTA; rank 0's MMA thread releases a stage in both CTAs with one
 //              tcgen05.commit ... multicast::cluster
 //   tfull[a]   one per CTA, signalled the same way when an accumulator is complete
-//   tempty[a]  lives in rank 0, expects the 4 epilogue warps of each CTA (remote arrivals)
+//   tempty[a]  lives in rank 0, expects the epilogue warps of both CTAs (remote arrivals)
 // The accumulator rows 0..127 sit in rank 0's tensor memory, rows 128..255 in rank 1's; each
 // CTA's epilogue warps drain their own half.  No TMA load uses multicast.
 // All mbarrier waits are bounded as in the one-CTA kernel; before tensor memory is freed the
@@ -123,7 +123,7 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
   if (threadIdx.x == 0) {
     s_abort = 0;
     for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * kEpiWarps); }
     mbar_init(exit_bar, 2);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tmap_a);
@@ -211,7 +211,6 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------ epilogue warps (both CTAs)
-    const int q = warp & 3;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -221,24 +220,8 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      const int row = it.tm * BM2 + (int)rank * BM + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      const int n_base = it.tn * p.bn;
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.bn);
-      float dot = 0.f;
-      for (int c = 0; c < p.bn / 32; ++c) {
-        const int n0 = n_base + c * 32;
-        if (n0 >= p.N) break;
-        uint32_t v[32];
-        tmem_ld32(t_row + (uint32_t)(c * 32), v);
-        tmem_ld_wait();
-        epilogue_chunk<EPI>(p, v, row, row_ok, n0, it.split, dot);
-      }
-      if (EPI == EPI_SLICE && p.qdot && row_ok)
-        p.dz_part[(int64_t)(it.split * p.tiles_n + it.tn) * p.dz_stride + row] = dot;
-      tcgen05_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+      run_epilogue<EPI, true>(p, tmem_base + (uint32_t)(acc * p.bn), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.split, it.tn,
+                              warp, lane, map_to_cta(tempty_bar(acc), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }

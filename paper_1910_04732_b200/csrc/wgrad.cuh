@@ -150,56 +150,89 @@ __device__ __forceinline__ void reduce_unit(const float* __restrict__ slices, in
   store4<TW>(out + (int64_t)row * ldo + c0, acc, valid, accumulate, vec_out);
 }
 
+// Number of work units (4 consecutive columns of one row, or one gate) of one problem.
+__host__ __device__ inline int64_t bwd_finish_units(const BwdFinishArgs& a) {
+  const int64_t c4r = (a.r + 3) >> 2, c4d = (a.d_in + 3) >> 2;
+  return (a.dP ? (int64_t)a.d_out * c4r : 0) + ((a.dQ ? 1 : 0) + (a.Qz ? 1 : 0)) * (int64_t)a.r * c4d +
+         (a.dlog_alpha ? (int64_t)a.r : 0);
+}
+
+template <typename TW>
+__device__ __forceinline__ void bwd_finish_unit(const BwdFinishArgs& a, int64_t u) {
+  const int c4r = (a.r + 3) >> 2, c4d = (a.d_in + 3) >> 2;
+  const int64_t n_p = a.dP ? (int64_t)a.d_out * c4r : 0;
+  const int64_t n_q = a.dQ ? (int64_t)a.r * c4d : 0;
+  const int64_t n_qz = a.Qz ? (int64_t)a.r * c4d : 0;
+  constexpr int al = sizeof(TW) == 4 ? 15 : 7;   // 4 outputs: 16 B (fp32) or 8 B (bf16)
+  if (u < n_p) {
+    const bool vec_p = ((reinterpret_cast<uintptr_t>(a.dP) & al) == 0) && (a.lddp % 4 == 0);
+    const int row = (int)(u / c4r), c0 = (int)(u % c4r) * 4;
+    reduce_unit<TW>(a.slices_p, a.n_slices_p, a.slice_elems_p, a.ld_slice_p, row, c0, a.r, 1.f, (TW*)a.dP, a.lddp,
+                    a.accumulate, vec_p);
+  } else if (u < n_p + n_q) {
+    const bool vec_q = ((reinterpret_cast<uintptr_t>(a.dQ) & al) == 0) && (a.lddq % 4 == 0);
+    const int64_t v = u - n_p;
+    const int row = (int)(v / c4d), c0 = (int)(v % c4d) * 4;
+    reduce_unit<TW>(a.slices_q, a.n_slices_q, a.slice_elems_q, a.ld_slice_q, row, c0, a.d_in, a.z[row], (TW*)a.dQ, a.lddq,
+                    a.accumulate, vec_q);
+  } else if (u < n_p + n_q + n_qz) {
+    const int64_t v = u - n_p - n_q;
+    const int row = (int)(v / c4d), c0 = (int)(v % c4d) * 4;
+    const int valid = min(4, a.d_in - c0);
+    const float g = a.z[row];
+    const __nv_bfloat16* q = a.Q + (int64_t)row * a.ldq + c0;
+    __nv_bfloat16* o = a.Qz + (int64_t)row * a.ldqz + c0;
+    if (valid == 4) {   // Q and Qz rows are 16-byte aligned with ld % 8 == 0: 8-byte accesses are aligned
+      const uint2 raw = *reinterpret_cast<const uint2*>(q);
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      const float2 x = __bfloat1622float2(h[0]), y = __bfloat1622float2(h[1]);
+      __nv_bfloat162 lo = __floats2bfloat162_rn(x.x * g, x.y * g), hi = __floats2bfloat162_rn(y.x * g, y.y * g);
+      uint2 out;
+      out.x = *reinterpret_cast<uint32_t*>(&lo);
+      out.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(o) = out;
+    } else {
+      for (int i = 0; i < valid; ++i) o[i] = __float2bfloat16_rn(__bfloat162float(q[i]) * g);
+    }
+  } else {
+    const int k = (int)(u - n_p - n_q - n_qz);
+    float s = 0.f;
+    for (int p = 0; p < a.n_part; ++p) s += a.dz_part[(int64_t)p * a.r + k];
+    const float v = s * a.dz_dla[k];
+    a.dlog_alpha[k] = a.accumulate ? a.dlog_alpha[k] + v : v;
+  }
+}
+
 template <typename TW>
 __global__ void __launch_bounds__(256)
 bwd_finish_kernel(const BwdFinishArgs a) {
   pdl_wait();
   pdl_launch_dependents();
-  const int c4r = (a.r + 3) >> 2, c4d = (a.d_in + 3) >> 2;
-  const int64_t n_p = a.dP ? (int64_t)a.d_out * c4r : 0;
-  const int64_t n_q = a.dQ ? (int64_t)a.r * c4d : 0;
-  const int64_t n_qz = a.Qz ? (int64_t)a.r * c4d : 0;
-  const int64_t n_a = a.dlog_alpha ? (int64_t)a.r : 0;
-  const int64_t total = n_p + n_q + n_qz + n_a;
-  constexpr int al = sizeof(TW) == 4 ? 15 : 7;   // 4 outputs: 16 B (fp32) or 8 B (bf16)
-  const bool vec_p = a.dP && ((reinterpret_cast<uintptr_t>(a.dP) & al) == 0) && (a.lddp % 4 == 0);
-  const bool vec_q = a.dQ && ((reinterpret_cast<uintptr_t>(a.dQ) & al) == 0) && (a.lddq % 4 == 0);
+  const int64_t total = bwd_finish_units(a);
+  for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x)
+    bwd_finish_unit<TW>(a, u);
+}
+
+// The same for up to kFinishGroup matrices in one launch (grouped backward).
+constexpr int kFinishGroup = 8;
+struct BwdFinishGroup {
+  BwdFinishArgs a[kFinishGroup];
+  int64_t unit_begin[kFinishGroup + 1];
+  int n;
+};
+
+template <typename TW>
+__global__ void __launch_bounds__(256)
+bwd_finish_group_kernel(const __grid_constant__ BwdFinishGroup g) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int64_t total = g.unit_begin[g.n];
   for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x) {
-    if (u < n_p) {
-      const int row = (int)(u / c4r), c0 = (int)(u % c4r) * 4;
-      reduce_unit<TW>(a.slices_p, a.n_slices_p, a.slice_elems_p, a.ld_slice_p, row, c0, a.r, 1.f, (TW*)a.dP, a.lddp,
-                      a.accumulate, vec_p);
-    } else if (u < n_p + n_q) {
-      const int64_t v = u - n_p;
-      const int row = (int)(v / c4d), c0 = (int)(v % c4d) * 4;
-      reduce_unit<TW>(a.slices_q, a.n_slices_q, a.slice_elems_q, a.ld_slice_q, row, c0, a.d_in, a.z[row], (TW*)a.dQ, a.lddq,
-                      a.accumulate, vec_q);
-    } else if (u < n_p + n_q + n_qz) {
-      const int64_t v = u - n_p - n_q;
-      const int row = (int)(v / c4d), c0 = (int)(v % c4d) * 4;
-      const int valid = min(4, a.d_in - c0);
-      const float g = a.z[row];
-      const __nv_bfloat16* q = a.Q + (int64_t)row * a.ldq + c0;
-      __nv_bfloat16* o = a.Qz + (int64_t)row * a.ldqz + c0;
-      if (valid == 4) {   // Q and Qz rows are 16-byte aligned with ld % 8 == 0: 8-byte accesses are aligned
-        const uint2 raw = *reinterpret_cast<const uint2*>(q);
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
-        const float2 x = __bfloat1622float2(h[0]), y = __bfloat1622float2(h[1]);
-        __nv_bfloat162 lo = __floats2bfloat162_rn(x.x * g, x.y * g), hi = __floats2bfloat162_rn(y.x * g, y.y * g);
-        uint2 out;
-        out.x = *reinterpret_cast<uint32_t*>(&lo);
-        out.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(o) = out;
-      } else {
-        for (int i = 0; i < valid; ++i) o[i] = __float2bfloat16_rn(__bfloat162float(q[i]) * g);
-      }
-    } else {
-      const int k = (int)(u - n_p - n_q - n_qz);
-      float s = 0.f;
-      for (int p = 0; p < a.n_part; ++p) s += a.dz_part[(int64_t)p * a.r + k];
-      const float v = s * a.dz_dla[k];
-      a.dlog_alpha[k] = a.accumulate ? a.dlog_alpha[k] + v : v;
-    }
+    int i = 0;
+#pragma unroll
+    for (int j = 1; j < kFinishGroup; ++j)
+      if (j < g.n && u >= g.unit_begin[j]) i = j;
+    bwd_finish_unit<TW>(g.a[i], u - g.unit_begin[i]);
   }
 }
 
