@@ -255,6 +255,7 @@ struct TcEpilogue {
   bf16* out; int64_t ldo; const float* col_scale;
   float* slices; int64_t slice_elems, ld_slice;
   const bf16* qdot; int64_t ldq; float* dz_part; int64_t dz_stride;
+  void* wg_out; int wg_f32; const float* row_scale; int accumulate;   // tc::EPI_WGRAD (ldo is shared with out)
 };
 
 template <bool A_MN, bool B_MN, int EPI>
@@ -307,9 +308,11 @@ int launch_tc(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t 
   p.out = ep.out; p.ldo = ep.ldo; p.col_scale = ep.col_scale;
   p.slices = ep.slices; p.slice_elems = ep.slice_elems; p.ld_slice = ep.ld_slice;
   p.qdot = ep.qdot; p.ldq = ep.ldq; p.dz_part = ep.dz_part; p.dz_stride = ep.dz_stride;
+  p.wg_out = ep.wg_out; p.wg_f32 = ep.wg_f32; p.row_scale = ep.row_scale; p.accumulate = ep.accumulate;
   if (!A.mn_major && !B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, false, tc::EPI_STORE>(ta, tb, p, pl.cta2, st);
   if (!A.mn_major && B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, true, tc::EPI_STORE>(ta, tb, p, pl.cta2, st);
   if (A.mn_major && B.mn_major && ep.kind == tc::EPI_SLICE) return launch_tc_inst<true, true, tc::EPI_SLICE>(ta, tb, p, pl.cta2, st);
+  if (A.mn_major && B.mn_major && ep.kind == tc::EPI_WGRAD) return launch_tc_inst<true, true, tc::EPI_WGRAD>(ta, tb, p, pl.cta2, st);
   return FLOP_ERR_UNSUPPORTED;
 }
 
@@ -369,6 +372,7 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       p.out = j.ep.out; p.ldo = j.ep.ldo; p.col_scale = j.ep.col_scale;
       p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
       p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
+      p.wg_out = j.ep.wg_out; p.wg_f32 = j.ep.wg_f32; p.row_scale = j.ep.row_scale; p.accumulate = j.ep.accumulate;
       pr.work_begin = gp.total_work;
       gp.total_work += p.tiles_m * p.tiles_n * p.splits;
       gp.bn_max = std::max(gp.bn_max, p.bn);
@@ -382,9 +386,22 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     if (!a_mn && !b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, false, tc::EPI_STORE>(gp, flops, st);
     else if (!a_mn && b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, true, tc::EPI_STORE>(gp, flops, st);
     else if (a_mn && b_mn && first.ep.kind == tc::EPI_SLICE) rc = launch_group_inst<true, true, tc::EPI_SLICE>(gp, flops, st);
+    else if (a_mn && b_mn && first.ep.kind == tc::EPI_WGRAD) rc = launch_group_inst<true, true, tc::EPI_WGRAD>(gp, flops, st);
     FLOP_TRY(rc);
   }
   return FLOP_OK;
+}
+
+
+// Weight gradient written straight from the GEMM epilogue (no split-K, no fp32 slices).
+TcEpilogue wgrad_epilogue(void* out, int64_t ldo, int wgrad_dt, const float* row_scale, int accumulate) {
+  TcEpilogue e{};
+  e.kind = tc::EPI_WGRAD; e.wg_out = out; e.ldo = ldo; e.wg_f32 = wgrad_dt == FLOP_F32; e.row_scale = row_scale; e.accumulate = accumulate;
+  return e;
+}
+// The direct epilogue stores 16-byte vectors: rows of the output must allow that.
+bool wgrad_direct_ok(const void* out, int64_t ldo, int wgrad_dt) {
+  return aligned16(out) && (ldo % (wgrad_dt == FLOP_F32 ? 4 : 8)) == 0;
 }
 
 int launch_simt(const float* A, int64_t a_sm, int64_t a_sk, const float* B, int64_t b_sn, int64_t b_sk, float* C,
@@ -454,7 +471,9 @@ BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, 
   w.slice_elems_q = r * w.ld_slice_q;
   w.slices_p = dt == FLOP_BF16 ? (float*)ar.take((size_t)sp * w.slice_elems_p * 4) : nullptr;
   w.slices_q = (float*)ar.take((size_t)sq * w.slice_elems_q * 4);
-  w.dz_part = (float*)ar.take((size_t)w.n_part * std::max<int64_t>(r, 1) * 4);
+  // room for the partials of any tile shape: the direct-epilogue path may use another N tile than plan_q
+  const int64_t part_cap = std::max<int64_t>(w.n_part, 2 * ((d_in + 63) / 64));
+  w.dz_part = (float*)ar.take((size_t)part_cap * std::max<int64_t>(r, 1) * 4);
   w.bytes = ar.used;
   return w;
 }
@@ -768,16 +787,22 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
     // dH' = dY P            (A = dY K-major over d_out; B(n=k_rank, k=i) = P[i, k_rank]: MN-major)
     const TcPlan ph = plan_tc(T, r, d_out, false, true);
     FLOP_TRY(launch_tc({dY, lddy, false}, {P, ldp, true}, T, r, d_out, ph, store_epilogue(w.dH, w.lddh, nullptr), st));
+    // A weight-gradient GEMM that needs no split-K writes its result straight from the epilogue;
+    // otherwise it writes fp32 slices that the finishing kernel adds up in order.
+    const bool direct_p = dP && w.plan_p.splits == 1 && wgrad_direct_ok(dP, lddp, wgrad_dt);
+    const bool direct_q = need_m && w.plan_q.splits == 1 && (!dQ || wgrad_direct_ok(dQ, lddq, wgrad_dt));
     if (dP) {
-      // dP = dY^T H'        (contract over tokens: both operands MN-major), fp32 split-K slices
+      // dP = dY^T H'        (contract over tokens: both operands MN-major)
       TcEpilogue e{};
-      e.kind = tc::EPI_SLICE; e.slices = w.slices_p; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
+      if (direct_p) e = wgrad_epilogue(dP, lddp, wgrad_dt, nullptr, accumulate);
+      else { e.kind = tc::EPI_SLICE; e.slices = w.slices_p; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p; }
       FLOP_TRY(launch_tc({dY, lddy, true}, {H_save, ldh, true}, d_out, r, T, w.plan_p, e, st));
     }
     if (need_m) {
       // M = dH'^T X; dQ = diag(z) M; dz_k = <Q[k,:], M[k,:]> fused into the GEMM epilogue per tile
       TcEpilogue e{};
-      e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
+      if (direct_q) e = dQ ? wgrad_epilogue(dQ, lddq, wgrad_dt, z, accumulate) : wgrad_epilogue(w.slices_q, w.ld_slice_q, FLOP_F32, nullptr, 0);
+      else { e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q; }
       if (dlog_alpha) { e.qdot = (const bf16*)Q; e.ldq = ldq; e.dz_part = w.dz_part; e.dz_stride = r; }
       FLOP_TRY(launch_tc({w.dH, w.lddh, true}, {X, ldx, true}, r, d_in, T, w.plan_q, e, st));
     }
@@ -785,12 +810,12 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
       // one launch: ordered split-K sums -> dP, diag(z)-scaled dQ; diag(z) Q for the dX GEMM; dlog_alpha
       BwdFinishArgs a{};
       a.slices_p = w.slices_p; a.n_slices_p = w.plan_p.splits; a.slice_elems_p = w.slice_elems_p; a.ld_slice_p = w.ld_slice_p;
-      a.d_out = (int)d_out; a.r = (int)r; a.dP = dP; a.lddp = lddp;
+      a.d_out = (int)d_out; a.r = (int)r; a.dP = direct_p ? nullptr : dP; a.lddp = lddp;
       a.slices_q = w.slices_q; a.n_slices_q = w.plan_q.splits; a.slice_elems_q = w.slice_elems_q; a.ld_slice_q = w.ld_slice_q;
-      a.d_in = (int)d_in; a.dQ = dQ; a.lddq = lddq; a.z = z;
+      a.d_in = (int)d_in; a.dQ = direct_q ? nullptr : dQ; a.lddq = lddq; a.z = z;
       a.Q = (const bf16*)Q; a.ldq = ldq; a.Qz = dX ? (bf16*)w.Qz : nullptr; a.ldqz = w.ldqz;
       a.dz_part = w.dz_part; a.n_part = w.n_part; a.dz_dla = dz_dla; a.dlog_alpha = dlog_alpha; a.accumulate = accumulate;
-      const int64_t units = (dP ? d_out * ((r + 3) / 4) : 0) + ((dQ ? 1 : 0) + (dX ? 1 : 0)) * r * ((d_in + 3) / 4) + (dlog_alpha ? r : 0);
+      const int64_t units = bwd_finish_units(a);
       if (units > 0) {
         const int grid = (int)std::min<int64_t>((units + 255) / 256, (int64_t)num_sms() * 8);
         if (wgrad_dt == FLOP_BF16) launch_k(bwd_finish_kernel<bf16>, dim3(grid), dim3(256), (size_t)(0), st, a);
@@ -891,6 +916,8 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
   cudaStream_t st = (cudaStream_t)stream;
   std::vector<TcJob> g3, g4, g5, g6;
   std::vector<BwdFinishArgs> fin;
+  std::vector<BwdWs> wss;
+  bool direct = true;   // weight gradients straight from the GEMM epilogue (no split-K, no fp32 slices)
   for (int i = 0; i < n; ++i) {
     const flop_bwd_problem_t& a = pr[i];
     if ((a.dX && a.lddx < a.d_in) || (a.dP && a.lddp < a.r) || (a.dQ && a.lddq < a.d_in) || (a.dlog_alpha && !a.dz_dla))
@@ -904,32 +931,88 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     Arena probe{nullptr, 0, 0};
     FLOP_TRY(check_ws(a.ws, a.ws_bytes, plan_bwd_ws(probe, a.T, a.d_in, a.d_out, a.r, dt, true).bytes));
     Arena ar{(unsigned char*)a.ws, a.ws_bytes, 0};
-    const BwdWs w = plan_bwd_ws(ar, a.T, a.d_in, a.d_out, a.r, dt, true);
+    wss.push_back(plan_bwd_ws(ar, a.T, a.d_in, a.d_out, a.r, dt, true));
+    if ((a.dP && !wgrad_direct_ok(a.dP, a.lddp, wgrad_dt)) || (a.dQ && !wgrad_direct_ok(a.dQ, a.lddq, wgrad_dt))) direct = false;
+  }
+  // One N tile for all weight-gradient GEMMs of the call: enough work items to fill the machine
+  // without splitting K?  Cost in SM cycles as in plan_tc.
+  int wg_bn = 0;
+  if (direct) {
+    double best = 1e300;
+    const int sms = num_sms();
+    const int cand[3] = {256, 192, 128};
+    for (int c = 0; c < 3; ++c) {
+      const int bn = cand[c];
+      double items = 0, cost_kb = 0;
+      for (int i = 0; i < n; ++i) {
+        const flop_bwd_problem_t& a = pr[i];
+        const double kb = (double)((a.T + tc::BK - 1) / tc::BK);
+        if (a.dP) { const double t = (double)((a.d_out + tc::BM - 1) / tc::BM) * ((a.r + bn - 1) / bn); items += t; cost_kb += t * kb; }
+        if (a.dQ || a.dlog_alpha) { const double t = (double)((a.r + tc::BM - 1) / tc::BM) * ((a.d_in + bn - 1) / bn); items += t; cost_kb += t * kb; }
+      }
+      if (items < sms) continue;
+      const double per_kb = std::max(2.0 * bn, (double)tc::stage_bytes(bn) / 54.0);
+      const double rounds = ceil(items / sms);
+      const double cost = rounds * (cost_kb / items) * per_kb + rounds * (600.0 + 10.0 * bn);
+      if (cost < best) { best = cost; wg_bn = bn; }
+    }
+    if (wg_bn == 0) direct = false;
+  }
+  auto direct_plan = [&](int64_t M, int64_t N, int64_t K) {
+    TcPlan pl{};
+    pl.bn = wg_bn; pl.cta2 = 0; pl.splits = 1;
+    pl.tiles_m = (int)((M + tc::BM - 1) / tc::BM); pl.tiles_n = (int)((N + wg_bn - 1) / wg_bn);
+    pl.num_kb = (int)((K + tc::BK - 1) / tc::BK); pl.kb_per_split = pl.num_kb;
+    return pl;
+  };
+  for (int i = 0; i < n; ++i) {
+    const flop_bwd_problem_t& a = pr[i];
+    const BwdWs& w = wss[i];
     const bool need_m = a.dQ || a.dlog_alpha;
     g3.push_back({{a.dY, a.lddy, false}, {a.P, a.ldp, true}, a.T, a.r, a.d_out, plan_tc(a.T, a.r, a.d_out, false, true, false),
                   store_epilogue(w.dH, w.lddh, nullptr)});
+    int n_part = w.n_part;
     if (a.dP) {
-      TcEpilogue e{};
-      e.kind = tc::EPI_SLICE; e.slices = w.slices_p; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
-      g4.push_back({{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, w.plan_p, e});
+      if (direct) {
+        g4.push_back({{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, direct_plan(a.d_out, a.r, a.T),
+                      wgrad_epilogue(a.dP, a.lddp, wgrad_dt, nullptr, accumulate)});
+      } else {
+        TcEpilogue e{};
+        e.kind = tc::EPI_SLICE; e.slices = w.slices_p; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
+        g4.push_back({{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, w.plan_p, e});
+      }
     }
     if (need_m) {
       TcEpilogue e{};
-      e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
+      TcPlan pl = w.plan_q;
+      if (direct) {
+        // dQ = diag(z) (dH'^T X) stored in place (dQ may be absent when only dlog_alpha is wanted: then
+        // the product still runs for the fused row dots and its values go to the slice buffer)
+        pl = direct_plan(a.r, a.d_in, a.T);
+        if (a.dQ) e = wgrad_epilogue(a.dQ, a.lddq, wgrad_dt, a.z, accumulate);
+        else      e = wgrad_epilogue(w.slices_q, w.ld_slice_q, FLOP_F32, nullptr, 0);
+        n_part = 2 * pl.tiles_n;
+      } else {
+        e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
+      }
       if (a.dlog_alpha) { e.qdot = (const bf16*)a.Q; e.ldq = a.ldq; e.dz_part = w.dz_part; e.dz_stride = a.r; }
-      g5.push_back({{w.dH, w.lddh, true}, {a.X, a.ldx, true}, a.r, a.d_in, a.T, w.plan_q, e});
+      g5.push_back({{w.dH, w.lddh, true}, {a.X, a.ldx, true}, a.r, a.d_in, a.T, pl, e});
     }
     BwdFinishArgs f{};
     f.slices_p = w.slices_p; f.n_slices_p = w.plan_p.splits; f.slice_elems_p = w.slice_elems_p; f.ld_slice_p = w.ld_slice_p;
-    f.d_out = (int)a.d_out; f.r = (int)a.r; f.dP = a.dP; f.lddp = a.lddp;
+    f.d_out = (int)a.d_out; f.r = (int)a.r; f.dP = direct ? nullptr : a.dP; f.lddp = a.lddp;
     f.slices_q = w.slices_q; f.n_slices_q = w.plan_q.splits; f.slice_elems_q = w.slice_elems_q; f.ld_slice_q = w.ld_slice_q;
-    f.d_in = (int)a.d_in; f.dQ = a.dQ; f.lddq = a.lddq; f.z = a.z;
+    f.d_in = (int)a.d_in; f.dQ = direct ? nullptr : a.dQ; f.lddq = a.lddq; f.z = a.z;
     f.Q = (const bf16*)a.Q; f.ldq = a.ldq; f.Qz = a.dX ? (bf16*)w.Qz : nullptr; f.ldqz = w.ldqz;
-    f.dz_part = w.dz_part; f.n_part = w.n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.dlog_alpha; f.accumulate = accumulate;
+    f.dz_part = w.dz_part; f.n_part = n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.dlog_alpha; f.accumulate = accumulate;
     fin.push_back(f);
     if (a.dX)
       g6.push_back({{w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, a.T, a.d_in, a.r, plan_tc(a.T, a.d_in, a.r, false, true, false),
                     store_epilogue(a.dX, a.lddx, nullptr)});
+  }
+  if (direct) {   // both weight-gradient products of every matrix in one work list
+    g4.insert(g4.end(), g5.begin(), g5.end());
+    g5.clear();
   }
   FLOP_TRY(launch_tc_group(g3, st));   // dH' = dY P
   FLOP_TRY(launch_tc_group(g4, st));   // dY^T H' slices

@@ -51,9 +51,11 @@ struct Params {
   float* slices; int64_t slice_elems; int64_t ld_slice;
   const __nv_bfloat16* qdot; int64_t ldq;      // nullable: dz_part[(split*tiles_n+tn)*dz_stride + m] = sum_n acc*qdot[m,n]
   float* dz_part; int64_t dz_stride;
+  // EPI_WGRAD (splits == 1): wg_out[m*ldo + n] (=|+=) row_scale[m] * acc, bf16 or fp32; same fused row dot
+  void* wg_out; int wg_f32; const float* row_scale; int accumulate;
 };
 
-enum { EPI_STORE = 0, EPI_SLICE = 1 };
+enum { EPI_STORE = 0, EPI_SLICE = 1, EPI_WGRAD = 2 };
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -202,7 +204,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
           }
         }
       }
-    } else {
+    } else if (EPI == EPI_SLICE) {
       if (row_ok) {
         float* o = p.slices + (int64_t)split * p.slice_elems + (int64_t)row * p.ld_slice + n0;
         if (full_chunk) {
@@ -232,6 +234,82 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+          }
+        }
+      }
+    } else {
+      // weight gradient written in place: the fused row dot uses the unscaled accumulator, the
+      // stored value carries the gate of this row (dQ = diag(z) M) and the caller's accumulate flag
+      if (row_ok) {
+        if (p.qdot) {
+          const __nv_bfloat16* qr = p.qdot + (int64_t)row * p.ldq + n0;
+          if (full_chunk) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint4 raw = __ldg(reinterpret_cast<const uint4*>(qr + 8 * i));
+              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 f = __bfloat1622float2(h[j]);
+                dot = fmaf(__uint_as_float(v[8 * i + 2 * j]), f.x, dot);
+                dot = fmaf(__uint_as_float(v[8 * i + 2 * j + 1]), f.y, dot);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+          }
+        }
+        const float rs = p.row_scale ? __ldg(p.row_scale + row) : 1.f;
+        if (p.wg_f32) {
+          float* o = reinterpret_cast<float*>(p.wg_out) + (int64_t)row * p.ldo + n0;
+          if (full_chunk) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float4 w = make_float4(__uint_as_float(v[4 * i]) * rs, __uint_as_float(v[4 * i + 1]) * rs,
+                                     __uint_as_float(v[4 * i + 2]) * rs, __uint_as_float(v[4 * i + 3]) * rs);
+              if (p.accumulate) {
+                const float4 c = *reinterpret_cast<const float4*>(o + 4 * i);
+                w.x += c.x; w.y += c.y; w.z += c.z; w.w += c.w;
+              }
+              *reinterpret_cast<float4*>(o + 4 * i) = w;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (n0 + i < p.N) o[i] = (p.accumulate ? o[i] : 0.f) + __uint_as_float(v[i]) * rs;
+          }
+        } else {
+          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.wg_out) + (int64_t)row * p.ldo + n0;
+          if (full_chunk) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float w[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) w[j] = __uint_as_float(v[8 * i + j]) * rs;
+              if (p.accumulate) {
+                const uint4 c = *reinterpret_cast<const uint4*>(o + 8 * i);
+                const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&c);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const float2 f = __bfloat1622float2(h[j]);
+                  w[2 * j] += f.x; w[2 * j + 1] += f.y;
+                }
+              }
+              uint32_t pk[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                __nv_bfloat162 hh = __floats2bfloat162_rn(w[2 * j], w[2 * j + 1]);
+                pk[j] = *reinterpret_cast<uint32_t*>(&hh);
+              }
+              *reinterpret_cast<uint4*>(o + 8 * i) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (n0 + i < p.N)
+                o[i] = __float2bfloat16_rn((p.accumulate ? __bfloat162float(o[i]) : 0.f) + __uint_as_float(v[i]) * rs);
           }
         }
       }
@@ -281,7 +359,7 @@ __device__ __forceinline__ void run_epilogue(const Params& p, uint32_t t_acc, in
       else mbar_arrive(release_bar);
     }
   }
-  if (EPI == EPI_SLICE && p.qdot && row_ok)
+  if (EPI != EPI_STORE && p.qdot && row_ok)
     p.dz_part[(int64_t)((split * p.tiles_n + tn) * 2 + h) * p.dz_stride + row] = dot;
 }
 

@@ -1,4 +1,4 @@
-// Grouped form of the one-CTA tensor-core GEMM: up to kMaxGroup independent problems
+// Grouped form of the one-CTA tensor-core GEMM: up to kMaxGroup (16) independent problems
 // D_g = A_g B_g^T (same operand majors and epilogue kind, any sizes) in ONE persistent launch.
 //
 // Why: the GEMMs of a BERT- or Transformer-XL-sized factorized matrix are 3-20 GFLOP each,
@@ -18,7 +18,7 @@
 namespace flop {
 namespace tc {
 
-constexpr int kMaxGroup = 8;
+constexpr int kMaxGroup = 16;   // 16 x 384 B of kernel parameters (the limit is 32 KB)
 
 struct alignas(64) GroupProblem {
   CUtensorMap ta, tb;
