@@ -22,6 +22,7 @@
 #include "gemm_tc.cuh"
 #include "gemm_tc2.cuh"
 #include "gemm_tc_group.cuh"
+#include "gemm_tc2_group.cuh"
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
 
@@ -331,17 +332,34 @@ struct TcJob {
 };
 
 template <bool A_MN, bool B_MN, int EPI>
-int launch_group_inst(const tc::GroupParams& gp, double flops, cudaStream_t st) {
+int launch_group_inst(const tc::GroupParams& gp, int cta2, double flops, cudaStream_t st) {
   static bool configured = false;
-  auto kern = tc::gemm_group_kernel<A_MN, B_MN, EPI>;
+  auto kern1 = tc::gemm_group_kernel<A_MN, B_MN, EPI>;
+  auto kern2 = tc::gemm2_group_kernel<A_MN, B_MN, EPI>;
   if (!configured) {
-    FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    FLOP_CUDA(cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    FLOP_CUDA(cudaFuncSetAttribute(kern2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     configured = true;
   }
-  const int smem = 1024 + gp.stages * (int)tc::stage_bytes(gp.bn_max) + kSmemBarrierBytes;
   {
     GemmTimer timer(st, flops);
-    launch_k(kern, dim3(std::min(gp.total_work, num_sms())), dim3(tc::kThreads), (size_t)smem, st, gp);
+    if (!cta2) {
+      const int smem = 1024 + gp.stages * (int)tc::stage_bytes(gp.bn_max) + kSmemBarrierBytes;
+      launch_k(kern1, dim3(std::min(gp.total_work, num_sms())), dim3(tc::kThreads), (size_t)smem, st, gp);
+    } else {
+      const int smem = 1024 + gp.stages * (int)tc::stage_bytes2(gp.bn_max) + kSmemBarrierBytes;
+      const int pairs = std::min(gp.total_work, num_sms() / 2);
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
+      cudaLaunchAttribute attr[2];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[1].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = pdl_on() ? 2 : 1;
+      cudaLaunchKernelEx(&cfg, kern2, gp);
+    }
   }
   count_launch();
   FLOP_CUDA(cudaGetLastError());
@@ -358,12 +376,13 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     for (; i < jobs.size() && gp.n < tc::kMaxGroup; ++i) {
       const TcJob& j = jobs[i];
       if (j.M <= 0 || j.N <= 0 || j.K <= 0) continue;
-      if (j.M > INT32_MAX || j.N > INT32_MAX || j.K > INT32_MAX || j.pl.cta2) return FLOP_ERR_UNSUPPORTED;
+      if (j.M > INT32_MAX || j.N > INT32_MAX || j.K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+      if (j.pl.cta2 != first.pl.cta2) return FLOP_ERR_INVALID_ARG;
       if (j.A.mn_major != first.A.mn_major || j.B.mn_major != first.B.mn_major || j.ep.kind != first.ep.kind) return FLOP_ERR_INVALID_ARG;
       tc::GroupProblem& pr = gp.prob[gp.n];
       if (!j.A.mn_major) FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.M, j.K, j.A.ld, tc::BK, tc::BM));
       else               FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.K, j.M, j.A.ld, tc::kBoxMN, tc::BK));
-      if (!j.B.mn_major) FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.N, j.K, j.B.ld, tc::BK, (uint32_t)j.pl.bn));
+      if (!j.B.mn_major) FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.N, j.K, j.B.ld, tc::BK, (uint32_t)(j.pl.cta2 ? j.pl.bn / 2 : j.pl.bn)));
       else               FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.K, j.N, j.B.ld, tc::kBoxMN, tc::BK));
       tc::Params& p = pr.p;
       p.M = (int)j.M; p.N = (int)j.N; p.K = (int)j.K;
@@ -380,18 +399,68 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       ++gp.n;
     }
     if (gp.n == 0) continue;
-    gp.stages = std::min(tc::kMaxStages, (kSmemBudget - 1024 - kSmemBarrierBytes) / (int)tc::stage_bytes(gp.bn_max));
+    const int cta2 = first.pl.cta2;
+    gp.stages = std::min(tc::kMaxStages, (kSmemBudget - 1024 - kSmemBarrierBytes) /
+                                             (int)(cta2 ? tc::stage_bytes2(gp.bn_max) : tc::stage_bytes(gp.bn_max)));
     const bool a_mn = first.A.mn_major, b_mn = first.B.mn_major;
     int rc = FLOP_ERR_UNSUPPORTED;
-    if (!a_mn && !b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, false, tc::EPI_STORE>(gp, flops, st);
-    else if (!a_mn && b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, true, tc::EPI_STORE>(gp, flops, st);
-    else if (a_mn && b_mn && first.ep.kind == tc::EPI_SLICE) rc = launch_group_inst<true, true, tc::EPI_SLICE>(gp, flops, st);
-    else if (a_mn && b_mn && first.ep.kind == tc::EPI_WGRAD) rc = launch_group_inst<true, true, tc::EPI_WGRAD>(gp, flops, st);
+    if (!a_mn && !b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, false, tc::EPI_STORE>(gp, cta2, flops, st);
+    else if (!a_mn && b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, true, tc::EPI_STORE>(gp, cta2, flops, st);
+    else if (a_mn && b_mn && first.ep.kind == tc::EPI_SLICE) rc = launch_group_inst<true, true, tc::EPI_SLICE>(gp, cta2, flops, st);
+    else if (a_mn && b_mn && first.ep.kind == tc::EPI_WGRAD) rc = launch_group_inst<true, true, tc::EPI_WGRAD>(gp, cta2, flops, st);
     FLOP_TRY(rc);
   }
   return FLOP_OK;
 }
 
+
+// ---- tile shape for a whole group: one (pair?, N tile) for all jobs of a launch, no split-K
+TcPlan fixed_plan(int64_t M, int64_t N, int64_t K, int bn, int cta2) {
+  TcPlan pl{};
+  const int bm = cta2 ? tc::BM2 : tc::BM;
+  pl.bn = bn; pl.cta2 = cta2; pl.splits = 1;
+  pl.tiles_m = (int)((M + bm - 1) / bm); pl.tiles_n = (int)((N + bn - 1) / bn);
+  pl.num_kb = (int)((K + tc::BK - 1) / tc::BK); pl.kb_per_split = pl.num_kb;
+  return pl;
+}
+struct Mnk { int64_t M, N, K; };
+struct GroupShape { int bn, cta2; double items; };
+// Cost in SM cycles of running all jobs with one tile shape: rounds over the machine x (average
+// k-blocks per tile x the slower of MMA issue and shared-memory fill) + epilogues.  The fill rate
+// of an SM (about 50 B/clk) is what usually decides, which favours CTA pairs and wide tiles;
+// padding waste and the number of rounds pull the other way.  FLOP_TC_GROUP_BN / FLOP_TC_GROUP_CTA2
+// (1 = force pairs, 2 = forbid) override for tuning.
+GroupShape plan_group(const std::vector<Mnk>& jobs, bool b_mn_major) {
+  static const int force_bn = env_int("FLOP_TC_GROUP_BN"), force_cta2 = env_int("FLOP_TC_GROUP_CTA2");
+  const int sms = num_sms();
+  GroupShape best{0, 0, 0.0};
+  double best_cost = 1e300;
+  const int cand[4] = {256, 192, 128, 64};
+  for (int pass = 0; pass < 2 && best.bn == 0; ++pass)
+  for (int cta2 = 0; cta2 <= 1; ++cta2) {
+    if (pass == 0 && ((force_cta2 == 1 && !cta2) || (force_cta2 == 2 && cta2))) continue;
+    for (int c = 0; c < 4; ++c) {
+      const int bn = cand[c];
+      if (pass == 0 && force_bn && bn != force_bn) continue;
+      if (cta2 && b_mn_major && (bn / 2) % 64 != 0) continue;
+      const int bm = cta2 ? tc::BM2 : tc::BM;
+      const int units = cta2 ? sms / 2 : sms;
+      double items = 0, kb_sum = 0;
+      for (const Mnk& j : jobs) {
+        const double t = (double)((j.M + bm - 1) / bm) * (double)((j.N + bn - 1) / bn);
+        items += t;
+        kb_sum += t * (double)((j.K + tc::BK - 1) / tc::BK);
+      }
+      if (items <= 0) continue;
+      const double bytes = cta2 ? (double)tc::stage_bytes2(bn) : (double)tc::stage_bytes(bn);
+      const double per_kb = std::max(2.0 * bn, bytes / 50.0);
+      const double rounds = ceil(items / units);
+      const double cost = rounds * ((kb_sum / items) * per_kb + 400.0 + 4.0 * bn) + 3000.0;
+      if (cost < best_cost) { best_cost = cost; best = GroupShape{bn, cta2, items}; }
+    }
+  }
+  return best;
+}
 
 // Weight gradient written straight from the GEMM epilogue (no split-K, no fp32 slices).
 TcEpilogue wgrad_epilogue(void* out, int64_t ldo, int wgrad_dt, const float* row_scale, int accumulate) {
@@ -877,6 +946,12 @@ int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, 
     return FLOP_OK;
   }
   std::vector<TcJob> g1, g2;
+  std::vector<Mnk> m1, m2;
+  for (int i = 0; i < n; ++i) {
+    m1.push_back({pr[i].T, pr[i].r, pr[i].d_in});
+    m2.push_back({pr[i].T, pr[i].d_out, pr[i].r});
+  }
+  const GroupShape s1 = plan_group(m1, false), s2 = plan_group(m2, false);
   for (int i = 0; i < n; ++i) {
     const flop_fwd_problem_t& a = pr[i];
     if (!check_mat(a.Y, a.ldy, a.d_out) || !a.z || !check_mat(a.P, a.ldp, a.r) || !check_mat(a.X, a.ldx, a.d_in) ||
@@ -884,9 +959,9 @@ int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, 
       return FLOP_ERR_INVALID_ARG;
     if (!bf16_ok(a.Y, a.ldy) || !bf16_ok(a.P, a.ldp) || !bf16_ok(a.H_save, a.ldh) || !bf16_ok(a.X, a.ldx) || !bf16_ok(a.Q, a.ldq))
       return FLOP_ERR_UNSUPPORTED;
-    g1.push_back({{a.X, a.ldx, false}, {a.Q, a.ldq, false}, a.T, a.r, a.d_in, plan_tc(a.T, a.r, a.d_in, false, false, false),
+    g1.push_back({{a.X, a.ldx, false}, {a.Q, a.ldq, false}, a.T, a.r, a.d_in, fixed_plan(a.T, a.r, a.d_in, s1.bn, s1.cta2),
                   store_epilogue(a.H_save, a.ldh, a.z)});
-    g2.push_back({{a.H_save, a.ldh, false}, {a.P, a.ldp, false}, a.T, a.d_out, a.r, plan_tc(a.T, a.d_out, a.r, false, false, false),
+    g2.push_back({{a.H_save, a.ldh, false}, {a.P, a.ldp, false}, a.T, a.d_out, a.r, fixed_plan(a.T, a.d_out, a.r, s2.bn, s2.cta2),
                   store_epilogue(a.Y, a.ldy, nullptr)});
   }
   cudaStream_t st = (cudaStream_t)stream;
@@ -934,42 +1009,24 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     wss.push_back(plan_bwd_ws(ar, a.T, a.d_in, a.d_out, a.r, dt, true));
     if ((a.dP && !wgrad_direct_ok(a.dP, a.lddp, wgrad_dt)) || (a.dQ && !wgrad_direct_ok(a.dQ, a.lddq, wgrad_dt))) direct = false;
   }
-  // One N tile for all weight-gradient GEMMs of the call: enough work items to fill the machine
-  // without splitting K?  Cost in SM cycles as in plan_tc.
-  int wg_bn = 0;
-  if (direct) {
-    double best = 1e300;
-    const int sms = num_sms();
-    const int cand[3] = {256, 192, 128};
-    for (int c = 0; c < 3; ++c) {
-      const int bn = cand[c];
-      double items = 0, cost_kb = 0;
-      for (int i = 0; i < n; ++i) {
-        const flop_bwd_problem_t& a = pr[i];
-        const double kb = (double)((a.T + tc::BK - 1) / tc::BK);
-        if (a.dP) { const double t = (double)((a.d_out + tc::BM - 1) / tc::BM) * ((a.r + bn - 1) / bn); items += t; cost_kb += t * kb; }
-        if (a.dQ || a.dlog_alpha) { const double t = (double)((a.r + tc::BM - 1) / tc::BM) * ((a.d_in + bn - 1) / bn); items += t; cost_kb += t * kb; }
-      }
-      if (items < sms) continue;
-      const double per_kb = std::max(2.0 * bn, (double)tc::stage_bytes(bn) / 54.0);
-      const double rounds = ceil(items / sms);
-      const double cost = rounds * (cost_kb / items) * per_kb + rounds * (600.0 + 10.0 * bn);
-      if (cost < best) { best = cost; wg_bn = bn; }
-    }
-    if (wg_bn == 0) direct = false;
+  // One tile shape per stage for all problems of the call.  The weight gradients go direct when
+  // the un-split work items fill the machine at least once.
+  std::vector<Mnk> m3, mw, m6;
+  for (int i = 0; i < n; ++i) {
+    const flop_bwd_problem_t& a = pr[i];
+    m3.push_back({a.T, a.r, a.d_out});
+    if (a.dP) mw.push_back({a.d_out, a.r, a.T});
+    if (a.dQ || a.dlog_alpha) mw.push_back({a.r, a.d_in, a.T});
+    if (a.dX) m6.push_back({a.T, a.d_in, a.r});
   }
-  auto direct_plan = [&](int64_t M, int64_t N, int64_t K) {
-    TcPlan pl{};
-    pl.bn = wg_bn; pl.cta2 = 0; pl.splits = 1;
-    pl.tiles_m = (int)((M + tc::BM - 1) / tc::BM); pl.tiles_n = (int)((N + wg_bn - 1) / wg_bn);
-    pl.num_kb = (int)((K + tc::BK - 1) / tc::BK); pl.kb_per_split = pl.num_kb;
-    return pl;
-  };
+  const GroupShape s3 = plan_group(m3, true), s6 = plan_group(m6, true), sw = plan_group(mw, true);
+  if (sw.bn == 0 || sw.items < (sw.cta2 ? num_sms() / 2 : num_sms())) direct = false;
+  auto direct_plan = [&](int64_t M, int64_t N, int64_t K) { return fixed_plan(M, N, K, sw.bn, sw.cta2); };
   for (int i = 0; i < n; ++i) {
     const flop_bwd_problem_t& a = pr[i];
     const BwdWs& w = wss[i];
     const bool need_m = a.dQ || a.dlog_alpha;
-    g3.push_back({{a.dY, a.lddy, false}, {a.P, a.ldp, true}, a.T, a.r, a.d_out, plan_tc(a.T, a.r, a.d_out, false, true, false),
+    g3.push_back({{a.dY, a.lddy, false}, {a.P, a.ldp, true}, a.T, a.r, a.d_out, fixed_plan(a.T, a.r, a.d_out, s3.bn, s3.cta2),
                   store_epilogue(w.dH, w.lddh, nullptr)});
     int n_part = w.n_part;
     if (a.dP) {
@@ -1007,7 +1064,7 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     f.dz_part = w.dz_part; f.n_part = n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.dlog_alpha; f.accumulate = accumulate;
     fin.push_back(f);
     if (a.dX)
-      g6.push_back({{w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, a.T, a.d_in, a.r, plan_tc(a.T, a.d_in, a.r, false, true, false),
+      g6.push_back({{w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, a.T, a.d_in, a.r, fixed_plan(a.T, a.d_in, a.r, s6.bn, s6.cta2),
                     store_epilogue(a.dX, a.lddx, nullptr)});
   }
   if (direct) {   // both weight-gradient products of every matrix in one work list
