@@ -150,6 +150,7 @@ struct TcPlan {
 
 constexpr int kSmemBudget = 227 * 1024 - 1024;   // opt-in maximum minus room for the static __shared__ variables
 constexpr int kSmemBarrierBytes = 8 * (2 * tc::kMaxStages + 5);
+constexpr int kSmemFixed = 1024 + (int)tc::kStoreBufTotal + kSmemBarrierBytes;   // alignment slack + epilogue staging + barriers
 
 inline int env_int(const char* name) { const char* e = getenv(name); return e ? atoi(e) : 0; }
 
@@ -259,64 +260,6 @@ struct TcEpilogue {
   void* wg_out; int wg_f32; const float* row_scale; int accumulate;   // tc::EPI_WGRAD (ldo is shared with out)
 };
 
-template <bool A_MN, bool B_MN, int EPI>
-int launch_tc_inst(const CUtensorMap& ta, const CUtensorMap& tb, const tc::Params& p, int cta2, cudaStream_t st) {
-  static bool configured = false;
-  auto kern1 = tc::gemm_kernel<A_MN, B_MN, EPI>;
-  auto kern2 = tc::gemm2_kernel<A_MN, B_MN, EPI>;
-  if (!configured) {
-    FLOP_CUDA(cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    FLOP_CUDA(cudaFuncSetAttribute(kern2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    configured = true;
-  }
-  const int total = p.tiles_m * p.tiles_n * p.splits;
-  GemmTimer timer(st, 2.0 * p.M * (double)p.N * p.K);
-  if (!cta2) {
-    const int smem = 1024 + p.stages * (int)tc::stage_bytes(p.bn) + kSmemBarrierBytes;
-    launch_k(kern1, dim3(std::min(total, num_sms())), dim3(tc::kThreads), (size_t)smem, st, ta, tb, p);
-  } else {
-    const int smem = 1024 + p.stages * (int)tc::stage_bytes2(p.bn) + kSmemBarrierBytes;
-    const int pairs = std::min(total, num_sms() / 2);
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = pdl_on() ? 2 : 1;
-    cudaLaunchKernelEx(&cfg, kern2, ta, tb, p);
-  }
-  count_launch();
-  FLOP_CUDA(cudaGetLastError());
-  return FLOP_OK;
-}
-
-int launch_tc(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, const TcPlan& pl,
-              const TcEpilogue& ep, cudaStream_t st) {
-  if (M <= 0 || N <= 0 || K <= 0) return FLOP_OK;
-  if (M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
-  CUtensorMap ta, tb;
-  if (!A.mn_major) FLOP_TRY(make_tmap(&ta, A.ptr, M, K, A.ld, tc::BK, tc::BM));
-  else             FLOP_TRY(make_tmap(&ta, A.ptr, K, M, A.ld, tc::kBoxMN, tc::BK));
-  if (!B.mn_major) FLOP_TRY(make_tmap(&tb, B.ptr, N, K, B.ld, tc::BK, (uint32_t)(pl.cta2 ? pl.bn / 2 : pl.bn)));
-  else             FLOP_TRY(make_tmap(&tb, B.ptr, K, N, B.ld, tc::kBoxMN, tc::BK));
-  tc::Params p{};
-  p.M = (int)M; p.N = (int)N; p.K = (int)K;
-  p.bn = pl.bn; p.stages = pl.stages; p.tiles_m = pl.tiles_m; p.tiles_n = pl.tiles_n;
-  p.splits = pl.splits; p.kb_per_split = pl.kb_per_split; p.num_kb = pl.num_kb;
-  p.out = ep.out; p.ldo = ep.ldo; p.col_scale = ep.col_scale;
-  p.slices = ep.slices; p.slice_elems = ep.slice_elems; p.ld_slice = ep.ld_slice;
-  p.qdot = ep.qdot; p.ldq = ep.ldq; p.dz_part = ep.dz_part; p.dz_stride = ep.dz_stride;
-  p.wg_out = ep.wg_out; p.wg_f32 = ep.wg_f32; p.row_scale = ep.row_scale; p.accumulate = ep.accumulate;
-  if (!A.mn_major && !B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, false, tc::EPI_STORE>(ta, tb, p, pl.cta2, st);
-  if (!A.mn_major && B.mn_major && ep.kind == tc::EPI_STORE) return launch_tc_inst<false, true, tc::EPI_STORE>(ta, tb, p, pl.cta2, st);
-  if (A.mn_major && B.mn_major && ep.kind == tc::EPI_SLICE) return launch_tc_inst<true, true, tc::EPI_SLICE>(ta, tb, p, pl.cta2, st);
-  if (A.mn_major && B.mn_major && ep.kind == tc::EPI_WGRAD) return launch_tc_inst<true, true, tc::EPI_WGRAD>(ta, tb, p, pl.cta2, st);
-  return FLOP_ERR_UNSUPPORTED;
-}
-
 TcEpilogue store_epilogue(void* out, int64_t ldo, const float* col_scale) {
   TcEpilogue e{};
   e.kind = tc::EPI_STORE; e.out = (bf16*)out; e.ldo = ldo; e.col_scale = col_scale;
@@ -344,10 +287,10 @@ int launch_group_inst(const tc::GroupParams& gp, int cta2, double flops, cudaStr
   {
     GemmTimer timer(st, flops);
     if (!cta2) {
-      const int smem = 1024 + gp.stages * (int)tc::stage_bytes(gp.bn_max) + kSmemBarrierBytes;
+      const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes(gp.bn_max);
       launch_k(kern1, dim3(std::min(gp.total_work, num_sms())), dim3(tc::kThreads), (size_t)smem, st, gp);
     } else {
-      const int smem = 1024 + gp.stages * (int)tc::stage_bytes2(gp.bn_max) + kSmemBarrierBytes;
+      const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes2(gp.bn_max);
       const int pairs = std::min(gp.total_work, num_sms() / 2);
       cudaLaunchConfig_t cfg{};
       cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
@@ -392,6 +335,12 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
       p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
       p.wg_out = j.ep.wg_out; p.wg_f32 = j.ep.wg_f32; p.row_scale = j.ep.row_scale; p.accumulate = j.ep.accumulate;
+      // bf16 tiles that are plainly overwritten leave through a TMA store (64 x 32 boxes of the output)
+      void* tma_dst = j.ep.kind == tc::EPI_STORE ? (void*)j.ep.out
+                      : (j.ep.kind == tc::EPI_WGRAD && !j.ep.wg_f32 && !j.ep.accumulate) ? j.ep.wg_out : nullptr;
+      static const int no_tma_store = env_int("FLOP_NO_TMA_STORE");
+      p.tma_store = (tma_dst && !no_tma_store) ? 1 : 0;
+      if (p.tma_store) FLOP_TRY(make_tmap(&pr.tout, tma_dst, j.M, j.N, j.ep.ldo, 64, 32));
       pr.work_begin = gp.total_work;
       gp.total_work += p.tiles_m * p.tiles_n * p.splits;
       gp.bn_max = std::max(gp.bn_max, p.bn);
@@ -400,7 +349,7 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     }
     if (gp.n == 0) continue;
     const int cta2 = first.pl.cta2;
-    gp.stages = std::min(tc::kMaxStages, (kSmemBudget - 1024 - kSmemBarrierBytes) /
+    gp.stages = std::min(tc::kMaxStages, (kSmemBudget - kSmemFixed) /
                                              (int)(cta2 ? tc::stage_bytes2(gp.bn_max) : tc::stage_bytes(gp.bn_max)));
     const bool a_mn = first.A.mn_major, b_mn = first.B.mn_major;
     int rc = FLOP_ERR_UNSUPPORTED;
@@ -413,6 +362,12 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
   return FLOP_OK;
 }
 
+
+// A single GEMM is a group of one.
+int launch_tc(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, const TcPlan& pl,
+              const TcEpilogue& ep, cudaStream_t st) {
+  return launch_tc_group(std::vector<TcJob>{TcJob{A, B, M, N, K, pl, ep}}, st);
+}
 
 // ---- tile shape for a whole group: one (pair?, N tile) for all jobs of a launch, no split-K
 TcPlan fixed_plan(int64_t M, int64_t N, int64_t K, int bn, int cta2) {

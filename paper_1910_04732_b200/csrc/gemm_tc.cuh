@@ -38,6 +38,7 @@ constexpr uint32_t kBoxMN = 64;                   // MN-major operands arrive in
 constexpr uint32_t kBoxBytes = kBoxMN * BK * 2;   // 8 KB
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kWaitCycles = 2000000000LL;   // ~1 s
+constexpr uint32_t kStoreBufBytes = 32 * 128;      // one epilogue warp's staging tile: 32 rows x 64 bf16
 
 struct Params {
   int M, N, K;
@@ -53,6 +54,7 @@ struct Params {
   float* dz_part; int64_t dz_stride;
   // EPI_WGRAD (splits == 1): wg_out[m*ldo + n] (=|+=) row_scale[m] * acc, bf16 or fp32; same fused row dot
   void* wg_out; int wg_f32; const float* row_scale; int accumulate;
+  int tma_store;   // 1: bf16 output tiles leave through shared memory and a TMA store (tensor map given)
 };
 
 enum { EPI_STORE = 0, EPI_SLICE = 1, EPI_WGRAD = 2 };
@@ -103,6 +105,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the staging buffer may be overwritten once the earlier stores have read it
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -159,6 +174,8 @@ __device__ __forceinline__ uint32_t instr_desc(bool a_mn, bool b_mn, int n) {
 }
 
 __host__ __device__ inline uint32_t stage_bytes(int bn) { return kATileBytes + (uint32_t)bn * BK * 2; }
+// shared memory after the stage ring: the epilogue warps' staging tiles, then the barriers
+constexpr uint32_t kStoreBufTotal = kEpiWarps * kStoreBufBytes;
 
 struct WorkItem { int tm, tn, split, kb0, kb1; };
 __device__ __forceinline__ WorkItem decode(const Params& p, int w) {
@@ -316,30 +333,96 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
     }
 }
 
+// The row dot product <Q[row, n0..n0+31], acc> of the fused dz reduction, for the TMA-store path
+// (the other paths compute it inside epilogue_chunk).
+__device__ __forceinline__ void qdot_chunk(const Params& p, const uint32_t (&v)[32], int row, int n0, float& dot) {
+  const __nv_bfloat16* qr = p.qdot + (int64_t)row * p.ldq + n0;
+  if (n0 + 32 <= p.N) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(qr + 8 * i));
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = __bfloat1622float2(h[j]);
+        dot = fmaf(__uint_as_float(v[8 * i + 2 * j]), f.x, dot);
+        dot = fmaf(__uint_as_float(v[8 * i + 2 * j + 1]), f.y, dot);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+  }
+}
+
+// Converts one 32-column chunk of this thread's accumulator row to bf16 (times the column gate
+// or the row gate) and writes it as four 16-byte pieces into the warp's staging tile, laid out
+// as the 128-byte-swizzled box the TMA store expects: row = lane, piece c at (c ^ (lane & 7)).
+template <int EPI>
+__device__ __forceinline__ void stage_chunk(const Params& p, const uint32_t (&v)[32], int row, int n0, uint32_t buf,
+                                            int piece0, int lane) {
+  float sc[32];
+  if (EPI == EPI_STORE && p.col_scale) {
+    if (n0 + 32 <= p.N && (reinterpret_cast<uintptr_t>(p.col_scale + n0) & 15) == 0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float4 f = __ldg(reinterpret_cast<const float4*>(p.col_scale + n0) + i);
+        sc[4 * i] = f.x; sc[4 * i + 1] = f.y; sc[4 * i + 2] = f.z; sc[4 * i + 3] = f.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) sc[i] = n0 + i < p.N ? __ldg(p.col_scale + n0 + i) : 0.f;
+    }
+  } else {
+    const float rs = (EPI == EPI_WGRAD && p.row_scale && row < p.M) ? __ldg(p.row_scale + row) : 1.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) sc[i] = rs;
+  }
+  const uint32_t row_addr = buf + (uint32_t)lane * 128u;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t pk[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * j]) * sc[8 * i + 2 * j],
+                                               __uint_as_float(v[8 * i + 2 * j + 1]) * sc[8 * i + 2 * j + 1]);
+      pk[j] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    st_shared_v4(row_addr + (uint32_t)(((piece0 + i) ^ (lane & 7)) << 4), pk[0], pk[1], pk[2], pk[3]);
+  }
+}
+
 // Epilogue of one accumulator tile for one epilogue warp.  Lane quarter q = warp & 3 fixes the
-// 32 accumulator rows this warp may read; h = 0/1 picks the even or odd 32-column chunks.  Two
-// chunks are fetched from tensor memory per wait, and the accumulator is handed back to the MMA
-// warp (arrive on `release_bar`, a CTA-local or cluster address) as soon as the last fetch has
-// landed in registers, before the conversion and the global stores.
+// 32 accumulator rows this warp may read; h = 0/1 picks the even or odd 64-column groups.  A group
+// (two 32-column chunks) is fetched from tensor memory per wait, and the accumulator is handed back
+// to the MMA warp (arrive on `release_bar`, a CTA-local or cluster address) as soon as the last
+// fetch has landed in registers, before conversion and stores.
+// Output path: with p.tma_store the 32 x 64 bf16 block is staged in shared memory (`store_buf`,
+// this warp's 4 KB) and leaves with one TMA store -- a thread owns a ROW of the accumulator, so
+// direct global stores would touch 32 different rows per instruction (32 partial sectors), which
+// measured ~7000 cycles per block against the ~400 of the staged store; the tensor map also clips
+// the ragged edges.  Otherwise (fp32 outputs, accumulate, split-K slices) each thread stores its row.
 template <int EPI, bool kClusterArrive>
-__device__ __forceinline__ void run_epilogue(const Params& p, uint32_t t_acc, int row0, int n_base, int split, int tn,
-                                             int warp, int lane, uint32_t release_bar) {
+__device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap* tmap_out, uint32_t store_buf, uint32_t t_acc,
+                                             int row0, int n_base, int split, int tn, int warp, int lane,
+                                             uint32_t release_bar) {
   const int q = warp & 3, h = (warp - 2) >> 2;
   const int row = row0 + q * 32 + lane;
   const bool row_ok = row < p.M;
   const uint32_t t_row = t_acc + ((uint32_t)(q * 32) << 16);
-  int nchunks = (min(p.bn, p.N - n_base) + 31) >> 5;      // chunks that hold columns of D
-  const int mine = (nchunks - h + 1) >> 1;                // chunks h, h+2, ... of this warp
+  const int nchunks = (min(p.bn, p.N - n_base) + 31) >> 5;   // 32-column chunks that hold columns of D
+  const int ngroups = (nchunks + 1) >> 1;                    // 64-column groups
   float dot = 0.f;
   bool released = false;
-  for (int i = 0; i < mine; i += 2) {
-    const int c0 = h + 2 * i, c1 = c0 + 2;
-    const bool two = i + 1 < mine;
+  for (int g = h; g < ngroups; g += 2) {
+    const int c0 = 2 * g, c1 = c0 + 1;
+    const bool two = c1 < nchunks;
     uint32_t v0[32], v1[32];
     tmem_ld32(t_row + (uint32_t)(c0 * 32), v0);
     if (two) tmem_ld32(t_row + (uint32_t)(c1 * 32), v1);
     tmem_ld_wait();
-    if (i + 2 >= mine) {
+    if (g + 2 >= ngroups) {
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -348,10 +431,25 @@ __device__ __forceinline__ void run_epilogue(const Params& p, uint32_t t_acc, in
       }
       released = true;
     }
-    epilogue_chunk<EPI>(p, v0, row, row_ok, n_base + c0 * 32, split, dot);
-    if (two) epilogue_chunk<EPI>(p, v1, row, row_ok, n_base + c1 * 32, split, dot);
+    const int n0 = n_base + c0 * 32;
+    if (p.tma_store) {
+      if (EPI != EPI_STORE && p.qdot && row_ok) {
+        qdot_chunk(p, v0, row, n0, dot);
+        if (two) qdot_chunk(p, v1, row, n0 + 32, dot);
+      }
+      if (lane == 0) tma_store_wait_read();   // the previous block has left the staging tile
+      __syncwarp();
+      stage_chunk<EPI>(p, v0, row, n0, store_buf, 0, lane);
+      if (two) stage_chunk<EPI>(p, v1, row, n0 + 32, store_buf, 4, lane);
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0 && row0 + q * 32 < p.M) tma_store_2d(tmap_out, n0, row0 + q * 32, store_buf);   // never start a store outside the tensor
+    } else {
+      epilogue_chunk<EPI>(p, v0, row, row_ok, n0, split, dot);
+      if (two) epilogue_chunk<EPI>(p, v1, row, row_ok, n0 + 32, split, dot);
+    }
   }
-  if (!released) {   // this warp had no chunk in the tile
+  if (!released) {   // this warp had no group in the tile
     tcgen05_fence_before();
     __syncwarp();
     if (lane == 0) {
@@ -361,142 +459,6 @@ __device__ __forceinline__ void run_epilogue(const Params& p, uint32_t t_acc, in
   }
   if (EPI != EPI_STORE && p.qdot && row_ok)
     p.dz_part[(int64_t)((split * p.tiles_n + tn) * 2 + h) * p.dz_stride + row] = dot;
-}
-
-template <bool A_MN, bool B_MN, int EPI>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzled tiles need 1024-byte alignment
-  const uint32_t sbytes = stage_bytes(p.bn);
-  const uint32_t bar_base = smem_base + (uint32_t)p.stages * sbytes;  // 8-byte aligned
-  // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2]
-  auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (uint32_t)(kMaxStages + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + 2 + a); };
-  __shared__ uint32_t s_tmem_base;
-  __shared__ int s_abort;
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total = p.tiles_m * p.tiles_n * p.splits;
-
-  if (threadIdx.x == 0) {
-    s_abort = 0;
-    for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kEpiWarps); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tmap(&tmap_a);
-    prefetch_tmap(&tmap_b);
-  }
-  if (warp == 1) tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
-  tcgen05_fence_before();
-  __syncthreads();
-  tcgen05_fence_after();
-  const uint32_t tmem_base = s_tmem_base;
-  volatile int* abort_flag = &s_abort;
-  // Everything above touched only shared and tensor memory; from here on global memory written by
-  // earlier kernels is read (and their inputs may be overwritten), so wait for them.
-  pdl_wait();
-  pdl_launch_dependents();
-
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      int armed = 0;   // stages armed so far (capped at p.stages): all of them hold a copy until consumed
-      bool ok = true;
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        const WorkItem it = decode(p, w);
-        for (int kb = it.kb0; kb < it.kb1; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t sa = smem_base + (uint32_t)stage * sbytes, sb = sa + kATileBytes;
-          const uint32_t fb = full_bar(stage);
-          mbar_expect_tx(fb, sbytes);
-          if (!A_MN) {
-            tma_load_2d(sa, &tmap_a, kb * BK, it.tm * BM, fb);
-          } else {
-#pragma unroll
-            for (int i = 0; i < BM / (int)kBoxMN; ++i)
-              tma_load_2d(sa + i * kBoxBytes, &tmap_a, it.tm * BM + i * (int)kBoxMN, kb * BK, fb);
-          }
-          if (!B_MN) {
-            tma_load_2d(sb, &tmap_b, kb * BK, it.tn * p.bn, fb);
-          } else {
-            for (int i = 0; i < p.bn / (int)kBoxMN; ++i)
-              tma_load_2d(sb + i * kBoxBytes, &tmap_b, it.tn * p.bn + i * (int)kBoxMN, kb * BK, fb);
-          }
-          if (armed < p.stages) ++armed;
-          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-        }
-      }
-      if (!ok || *abort_flag) {
-        // Leaving early: wait (bounded) until the copies already issued have landed, so that
-        // nothing writes this CTA's shared memory after it has exited.
-        int s = stage;
-        uint32_t ph = phase;
-        for (int i = 0; i < armed; ++i) {
-          if (--s < 0) { s = p.stages - 1; ph ^= 1u; }
-          const long long t0 = clock64();
-          while (!mbar_try_wait(full_bar(s), ph) && clock64() - t0 < kWaitCycles) {}
-        }
-      }
-    }
-  } else if (warp == 1) {
-    // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = instr_desc(A_MN, B_MN, p.bn);
-      int stage = 0;
-      uint32_t phase = 0;
-      int acc = 0;
-      uint32_t acc_phase = 0;
-      bool ok = true;
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        const WorkItem it = decode(p, w);
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
-        tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.bn);
-        for (int kb = it.kb0; kb < it.kb1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
-          tcgen05_fence_after();
-          const uint32_t sa = smem_base + (uint32_t)stage * sbytes, sb = sa + kATileBytes;
-#pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t ad = smem_desc(sa + (A_MN ? k * (UMMA_K * 128) : k * (UMMA_K * 2)), A_MN);
-            const uint64_t bd = smem_desc(sb + (B_MN ? k * (UMMA_K * 128) : k * (UMMA_K * 2)), B_MN);
-            umma_bf16(d_tmem, ad, bd, idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
-          }
-          umma_commit(empty_bar(stage));       // stage reusable once these MMAs have read it
-          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-        }
-        if (!ok) break;
-        umma_commit(tfull_bar(acc));           // accumulator complete
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-      }
-    }
-  } else {
-    // ------------------------------------------------------------ epilogue warps
-    int acc = 0;
-    uint32_t acc_phase = 0;
-    bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-      const WorkItem it = decode(p, w);
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tcgen05_fence_after();
-      run_epilogue<EPI, false>(p, tmem_base + (uint32_t)(acc * p.bn), it.tm * BM, it.tn * p.bn, it.split, it.tn, warp, lane,
-                               tempty_bar(acc));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-    }
-  }
-  tcgen05_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    tcgen05_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
-  }
 }
 
 }  // namespace tc

@@ -18,7 +18,8 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sbytes = stage_bytes2(gp.bn_max);
-  const uint32_t bar_base = smem_base + (uint32_t)gp.stages * sbytes;
+  const uint32_t store_base = smem_base + (uint32_t)gp.stages * sbytes;   // 1024-byte aligned: stages are multiples of 1 KB
+  const uint32_t bar_base = store_base + kStoreBufTotal;
   auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (uint32_t)(kMaxStages + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + a); };
@@ -42,6 +43,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
   if (warp == 0 && lane < gp.n) {
     prefetch_tmap(&gp.prob[lane].ta);
     prefetch_tmap(&gp.prob[lane].tb);
+    if (gp.prob[lane].p.tma_store) prefetch_tmap(&gp.prob[lane].tout);
   }
   if (warp == 1) tmem_alloc2(smem_u32(&s_tmem_base), kTmemCols);
   tcgen05_fence_before();
@@ -138,10 +140,11 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      run_epilogue<EPI, true>(p, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.split, it.tn,
+      run_epilogue<EPI, true>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.split, it.tn,
                               warp, lane, map_to_cta(tempty_bar(acc), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) tma_store_wait_all();
   }
   // ---------------------------------------------------------------- teardown
   tcgen05_fence_before();

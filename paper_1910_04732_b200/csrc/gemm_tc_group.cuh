@@ -18,10 +18,11 @@
 namespace flop {
 namespace tc {
 
-constexpr int kMaxGroup = 16;   // 16 x 384 B of kernel parameters (the limit is 32 KB)
+constexpr int kMaxGroup = 16;   // 16 x 576 B of kernel parameters (the limit is 32 KB)
 
 struct alignas(64) GroupProblem {
   CUtensorMap ta, tb;
+  CUtensorMap tout;   // bf16 output, 64 x 32 boxes (used when p.tma_store)
   Params p;
   int work_begin;   // index of this problem's first work item in the group's list
 };
@@ -52,7 +53,8 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sbytes = stage_bytes(gp.bn_max);
-  const uint32_t bar_base = smem_base + (uint32_t)gp.stages * sbytes;
+  const uint32_t store_base = smem_base + (uint32_t)gp.stages * sbytes;   // 1024-byte aligned: stages are multiples of 1 KB
+  const uint32_t bar_base = store_base + kStoreBufTotal;
   auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (uint32_t)(kMaxStages + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (uint32_t)(2 * kMaxStages + a); };
@@ -72,6 +74,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
   if (warp == 0 && lane < gp.n) {
     prefetch_tmap(&gp.prob[lane].ta);
     prefetch_tmap(&gp.prob[lane].tb);
+    if (gp.prob[lane].p.tma_store) prefetch_tmap(&gp.prob[lane].tout);
   }
   if (warp == 1) tmem_alloc(smem_u32(&s_tmem_base), kTmemCols);
   tcgen05_fence_before();
@@ -171,10 +174,11 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      run_epilogue<EPI, false>(p, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM, it.tn * p.bn, it.split, it.tn, warp, lane,
+      run_epilogue<EPI, false>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM, it.tn * p.bn, it.split, it.tn, warp, lane,
                                tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) tma_store_wait_all();   // this warp's output blocks are written before the CTA retires
   }
   tcgen05_fence_before();
   __syncthreads();
