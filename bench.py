@@ -168,7 +168,8 @@ class Job:
                                                      self.dlog_alpha[e["lo"]:e["hi"]], e["ws"]) for e in chunk])
                 self.groups.append((fwd, bwd))
         self.ws_l0 = b.alloc_workspace(b.workspace_bytes(b.OP_L0, self.n_gates, 0, 0, len(sizes), b.F32), device)
-        self.step_no = 0
+        self.offset_dev = torch.zeros(1, dtype=torch.int64, device=device)
+        self.graph = None
         self.world = 1
 
     def input_bytes(self) -> int:
@@ -182,9 +183,11 @@ class Job:
                             self.dlog_alpha[e["lo"]:e["hi"]], self.ws if ws is None else ws)
 
     def sample_gates(self):
-        # one launch for all gates of all layers; every rank uses the same (seed, offset): one mask per global batch
-        self.b.gate_sample(self.log_alpha, HC, 0, self.step_no << 24, self.z, self.mask, self.dz_dla)
-        self.step_no += 1
+        # one launch for all gates of all layers; every rank uses the same (seed, offset): one mask per global batch.
+        # The Philox offset lives on the device and is advanced on the device, so that a step captured in a
+        # CUDA graph draws a fresh mask at every replay.
+        self.b.gate_sample_devoff(self.log_alpha, HC, 0, 0, self.offset_dev, self.z, self.mask, self.dz_dla)
+        self.offset_dev.add_(1 << 24)
 
     def finish(self):
         self.b.expected_l0_lagrangian(self.log_alpha, self.seg_off, self.seg_size, HC, self.target, self.lam,
@@ -219,9 +222,27 @@ class Job:
         self.finish()
 
 
-def time_steps(job: Job, steps: int, world: int):
+def capture_step(job: Job):
+    """One whole step captured in a CUDA graph (the library's launches, programmatic dependent
+    launch edges included); replays cost one host call instead of ~25."""
+    import torch
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        job.step()                      # every kernel configured before capture
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            job.step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    job.graph = g
+
+
+def time_steps(job: Job, steps: int, world: int, use_graph: bool = False):
     """K steps between two synchronisation points, timed with CUDA events on the launching stream."""
     import torch
+    run = job.graph.replay if (use_graph and job.graph is not None) else job.step
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
@@ -229,7 +250,7 @@ def time_steps(job: Job, steps: int, world: int):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
-        job.step()
+        run()
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
@@ -349,6 +370,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="issue every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--group", type=int, default=-1, help="matrices per grouped call (0: one call per matrix; default: one layer)")
     ap.add_argument("--streams", type=int, default=1, help="streams over which independent matrices are issued")
     args = ap.parse_args()
@@ -387,8 +409,15 @@ def main():
     if rank == 0:
         sampler.start()
     n0 = b.launch_count()
-    ms = time_steps(job, args.steps, world)
-    launches = (b.launch_count() - n0) // args.steps
+    job.step()
+    launches = b.launch_count() - n0            # kernels of this library per step (the same inside a graph replay)
+    use_graph = not args.no_graph and world == 1   # NCCL all-reduces stay outside graphs here
+    if use_graph:
+        capture_step(job)
+        for _ in range(3):
+            job.graph.replay()
+    torch.cuda.synchronize()
+    ms = time_steps(job, args.steps, world, use_graph)
     # second pass of the same steps with CUDA events around every tensor-core GEMM launch
     b.gemm_timing_begin()
     ms_timed_pass = time_steps(job, args.steps, world)
@@ -422,7 +451,7 @@ def main():
         "pct_of_bf16_peak_measured_sustained": 100.0 * tflops / world / peaks["bf16_tflops_sustained"],
         "config": {"workload": w.name, "T": w.T, "layers": w.layers,
                    "matrices": [[m.name, m.d_in, m.d_out, m.r] for m in w.matrices],
-                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}", "streams": args.streams, "matrices_per_grouped_call": group,
+                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}", "streams": args.streams, "matrices_per_grouped_call": group, "cuda_graph": bool(use_graph),
                    "l2": f"inputs larger than L2: {job.input_bytes() / 1e6:.0f} MB of X and dY per step, each matrix its own buffers"},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": peaks["bf16_tflops_sustained"],

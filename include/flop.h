@@ -114,6 +114,15 @@ int flop_tc_gemm(const void* A, int64_t lda, int a_mn_major, const void* B, int6
 int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed,
                      uint64_t offset, float* z, uint8_t* mask, float* dz_dla, void* stream);
 
+/* The same sampler with the Philox counter offset taken from device memory:
+ * gate j uses counter offset + *offset_dev + j/4 (Section 3 draws a fresh u for
+ * every training batch).  A training step captured once in a CUDA graph keeps its
+ * kernel arguments; with the offset on the device the caller advances it between
+ * replays (any device-side add) and every replay draws a new mask. */
+int flop_gate_sample_devoff(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed,
+                            uint64_t offset, const uint64_t* offset_dev, float* z, uint8_t* mask,
+                            float* dz_dla, void* stream);
+
 /* Forward of the gated factorized layer (Section 4.1):
  *     H' = (X Q^T) * z   (column k times z_k, applied in the first GEMM's epilogue)
  *     Y  = H' P^T

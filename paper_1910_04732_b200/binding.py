@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 
 EXPORTS = ("flop_status_string", "flop_device_status", "flop_launch_count", "flop_gemm_timing_begin",
-           "flop_gemm_timing_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample",
+           "flop_gemm_timing_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_expected_l0_lagrangian",
            "flop_expected_l0_lagrangian_noalloc",
@@ -78,6 +78,7 @@ def load_library() -> ctypes.CDLL:
     lib.flop_tc_gemm.argtypes = [vp, i64, ci, vp, i64, ci, vp, i64, vp, vp, i64, i64, i64, ci, ci, ci,
                                  ctypes.POINTER(ctypes.c_int), vp]
     lib.flop_gate_sample.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
+    lib.flop_gate_sample_devoff.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp, vp]
     lib.flop_gated_lowrank_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
                                            i64, i64, i64, i64, ci, vp, sz, vp]
     lib.flop_gated_lowrank_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, i64,
@@ -185,6 +186,15 @@ def gate_sample(log_alpha: torch.Tensor, hc, seed: int, offset: int, z: torch.Te
     n = log_alpha.numel()
     _check(load_library().flop_gate_sample(_ptr(log_alpha), n, _hc(hc), seed, offset, _ptr(z), _ptr(mask),
                                            _ptr(dz_dla), _stream()), "flop_gate_sample")
+
+
+def gate_sample_devoff(log_alpha: torch.Tensor, hc, seed: int, offset: int, offset_dev: torch.Tensor, z: torch.Tensor,
+                       mask: Optional[torch.Tensor] = None, dz_dla: Optional[torch.Tensor] = None) -> None:
+    """Gate sampling with counter offset `offset + offset_dev[0]` (offset_dev: one 64-bit integer on the device)."""
+    assert offset_dev.element_size() == 8 and offset_dev.numel() >= 1
+    _check(load_library().flop_gate_sample_devoff(_ptr(log_alpha), log_alpha.numel(), _hc(hc), seed, offset,
+                                                  _ptr(offset_dev), _ptr(z), _ptr(mask), _ptr(dz_dla), _stream()),
+           "flop_gate_sample_devoff")
 
 
 def gated_lowrank_fwd(X, Q, P, z, Y, H_save=None, ws=None) -> None:

@@ -669,8 +669,8 @@ int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t
   return FLOP_OK;
 }
 
-int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed, uint64_t offset, float* z,
-                     uint8_t* mask, float* dz_dla, void* stream) {
+static int gate_sample_impl(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed, uint64_t offset,
+                            const uint64_t* offset_dev, float* z, uint8_t* mask, float* dz_dla, void* stream) {
   if (n < 0 || !valid_hc(hc)) return FLOP_ERR_INVALID_ARG;
   if (n == 0) return FLOP_OK;
   if (!log_alpha || !z) return FLOP_ERR_INVALID_ARG;
@@ -685,10 +685,21 @@ int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uin
   const int64_t want = (nblk + 255) / 256;
   const int grid = (int)std::min<int64_t>(want, (int64_t)num_sms() * 16);
   launch_k(gate_sample_kernel, dim3(grid), dim3(256), (size_t)(0), (cudaStream_t)stream, log_alpha, n, g, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)),
-                                                             offset, z, mask, dz_dla, vec_ok);
+                                                             offset, offset_dev, z, mask, dz_dla, vec_ok);
   count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
+}
+
+int flop_gate_sample(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed, uint64_t offset, float* z,
+                     uint8_t* mask, float* dz_dla, void* stream) {
+  return gate_sample_impl(log_alpha, n, hc, seed, offset, nullptr, z, mask, dz_dla, stream);
+}
+
+int flop_gate_sample_devoff(const float* log_alpha, int64_t n, flop_hc_params_t hc, uint64_t seed, uint64_t offset,
+                            const uint64_t* offset_dev, float* z, uint8_t* mask, float* dz_dla, void* stream) {
+  if (!offset_dev) return FLOP_ERR_INVALID_ARG;
+  return gate_sample_impl(log_alpha, n, hc, seed, offset, offset_dev, z, mask, dz_dla, stream);
 }
 
 static int fwd_impl(const void* X, int64_t ldx, const void* Q, int64_t ldq, const void* P, int64_t ldp, const float* z,

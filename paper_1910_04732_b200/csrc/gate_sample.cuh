@@ -65,10 +65,13 @@ __device__ __forceinline__ void gate_one(float alpha, uint32_t bits, const GateC
 }
 
 __global__ void __launch_bounds__(256)
-gate_sample_kernel(const float* __restrict__ log_alpha, int64_t n, GateConsts g, uint2 key, uint64_t offset,
+gate_sample_kernel(const float* __restrict__ log_alpha, int64_t n, GateConsts g, uint2 key, uint64_t offset_host,
+                   const uint64_t* __restrict__ offset_dev,
                    float* __restrict__ z, uint8_t* __restrict__ mask, float* __restrict__ dz_dla, int vec_ok) {
   pdl_wait();
   pdl_launch_dependents();
+  // the counter offset may also live in device memory, so that a captured launch can advance it
+  const uint64_t offset = offset_host + (offset_dev ? *offset_dev : 0ull);
   const int64_t nblk = (n + 3) >> 2;
   for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
     const uint64_t ctr = offset + (uint64_t)b;

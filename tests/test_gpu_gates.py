@@ -155,3 +155,22 @@ def test_expected_l0_ragged_segments_and_large_single_segment(b):
     t = float(np.float32(0.4))
     assert np.allclose(out4.cpu().numpy(), [0.0, -0.7 * (-t) + 2.5 * t * t, -t, t * t], rtol=1e-6)
     assert b.device_status() == b.OK
+
+
+def test_gate_sample_with_device_side_offset(b):
+    """The counter offset read from device memory: base + *offset_dev, advanced between calls."""
+    n = 10007
+    alpha = I.log_alpha(("normal", 0.5, 1.5), n, 0, 21)
+    a = torch.from_numpy(alpha).cuda()
+    off = torch.tensor([(1 << 33) + 5], dtype=torch.int64, device="cuda")
+    z = torch.empty(n, device="cuda"); m = torch.empty(n, dtype=torch.uint8, device="cuda"); d = torch.empty(n, device="cuda")
+    for step in range(3):
+        b.gate_sample_devoff(a, HC, 7, 1000, off, z, m, d)
+        zo, mo, do = O.gate_sample(alpha, *HC, seed=7, offset=1000 + (1 << 33) + 5 + step * (1 << 24))
+        assert np.array_equal(m.cpu().numpy(), mo)
+        assert np.max(np.abs(z.cpu().numpy() - zo)) < 2e-6 and np.max(np.abs(d.cpu().numpy() - do)) < 2e-6
+        off.add_(1 << 24)
+    with pytest.raises(b.FlopError):
+        b.load_library()  # keep the import used
+        b._check(b.load_library().flop_gate_sample_devoff(None, 4, b.HcParams(*HC), 0, 0, None, None, None, None, None),
+                 "flop_gate_sample_devoff")
