@@ -203,7 +203,7 @@ int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t
  * sized up front and is now frozen, a plug-in that is handed tensors but no
  * allocator, a region where cudaMalloc would synchronise the device or is
  * simply forbidden.  The caller passes only inputs and outputs; the kernels'
- * scratch is a fixed array that is part of the loaded library (about 41 KB,
+ * scratch is a fixed array that is part of the loaded library (about 35 KB,
  * held on every GPU that loads the library until the process exits), so the
  * call performs no cudaMalloc/cudaFree and uses no allocating library routine.
  *   - Limits: n <= 1,048,576 gates and n_seg <= 4096 segments; larger sizes

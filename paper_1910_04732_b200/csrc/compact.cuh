@@ -164,7 +164,7 @@ gather_p_kernel(const T* __restrict__ P, int64_t ldp, const int32_t* __restrict_
     }
     __syncthreads();
     T* o = Pc + (int64_t)i * ldpc;
-    for (int c = threadIdx.x; c < k; c += blockDim.x) o[c] = row[idx[c]];
+    for (int c = threadIdx.x; c < k; c += blockDim.x) o[c] = row[idx[c]];   // 2-byte stores, coalesced across the warp
     __syncthreads();
   }
 }

@@ -1148,7 +1148,7 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
     const size_t es = elt(dt);
     const int vq = aligned16(Q) && aligned16(Qc) && (ldq * es) % 16 == 0 && (ldqc * es) % 16 == 0;
     const int vp = aligned16(P) && (ldp * es) % 16 == 0;
-    const int rows_per_block = 4;
+    const int rows_per_block = 1;   // one P row per block: many resident blocks overlap one row's load with another's gather
     const size_t smem = (size_t)r * es;
     if (smem > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
     if (dt == FLOP_BF16) {

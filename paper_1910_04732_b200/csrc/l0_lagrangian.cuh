@@ -14,7 +14,7 @@
 namespace flop {
 
 constexpr int kL0Threads = 256;
-constexpr int kL0PerThread = 4;
+constexpr int kL0PerThread = 32;                    // eight 16-byte vectors per thread
 constexpr int kL0Chunk = kL0Threads * kL0PerThread;  // gates per block
 constexpr int kL0MaxSeg = 4096;
 
@@ -28,28 +28,27 @@ struct L0Scratch {         // layout of the caller's workspace
 // shared memory.  Serial per 16 segments per thread, then a block scan.
 __device__ __forceinline__ void l0_chunk_table(const int64_t* __restrict__ seg_off, int n_seg, int* first_chunk,
                                                int* scan_scratch) {
-  constexpr int per = kL0MaxSeg / kL0Threads;  // 16
+  // thread t owns segments [t*per, (t+1)*per): per = 1 for up to 256 segments, so the table costs
+  // one 16-byte read per thread instead of a fixed sixteen
+  const int per = (n_seg + kL0Threads - 1) / kL0Threads;
   const int s0 = threadIdx.x * per;
-  int cnt[per];
   int sum = 0;
-#pragma unroll
   for (int i = 0; i < per; ++i) {
     const int s = s0 + i;
-    int c = 0;
     if (s < n_seg) {
       const int64_t len = seg_off[s + 1] - seg_off[s];
-      c = len > 0 ? (int)((len + kL0Chunk - 1) / kL0Chunk) : 0;
+      sum += len > 0 ? (int)((len + kL0Chunk - 1) / kL0Chunk) : 0;
     }
-    cnt[i] = c;
-    sum += c;
   }
   int total;
   int base = block_exclusive_scan(sum, scan_scratch, &total);
-#pragma unroll
   for (int i = 0; i < per; ++i) {
     const int s = s0 + i;
-    if (s < n_seg) first_chunk[s] = base;
-    base += cnt[i];
+    if (s < n_seg) {
+      first_chunk[s] = base;
+      const int64_t len = seg_off[s + 1] - seg_off[s];
+      base += len > 0 ? (int)((len + kL0Chunk - 1) / kL0Chunk) : 0;
+    }
   }
   if (threadIdx.x == 0) first_chunk[n_seg] = total;
   __syncthreads();
@@ -65,7 +64,7 @@ __device__ __forceinline__ int l0_find_segment(const int* first_chunk, int n_seg
   return lo;
 }
 
-__device__ __forceinline__ float l0_pi(float a, float thr) { return 1.0f / (1.0f + expf(-(a - thr))); }
+__device__ __forceinline__ float l0_pi(float a, float thr) { return __fdividef(1.0f, 1.0f + __expf(-(a - thr))); }
 
 template <bool kGrad>
 __global__ void __launch_bounds__(kL0Threads)
@@ -85,43 +84,56 @@ l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__
   const int seg = l0_find_segment(first_chunk, n_seg, b);
   const int64_t lo = seg_off[seg] + (int64_t)(b - first_chunk[seg]) * kL0Chunk;
   const int64_t hi = min(seg_off[seg + 1], lo + (int64_t)kL0Chunk);
-  const int64_t j0 = lo + (int64_t)threadIdx.x * kL0PerThread;
-  float a[kL0PerThread];
-  const bool vec = (j0 + kL0PerThread <= hi) && ((reinterpret_cast<uintptr_t>(log_alpha + j0) & 15) == 0);
-  if (vec) {
-    const float4 v = *reinterpret_cast<const float4*>(log_alpha + j0);
-    a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w;
-  } else {
-#pragma unroll
-    for (int i = 0; i < kL0PerThread; ++i) a[i] = (j0 + i < hi) ? log_alpha[j0 + i] : 0.f;
+  // vector v of thread t covers gates lo + (v*256 + t)*4 .. +3: consecutive threads, consecutive 16 bytes
+  constexpr int kVec = kL0PerThread / 4;
+  const bool al_a = (reinterpret_cast<uintptr_t>(log_alpha + lo) & 15) == 0;
+  double sum = 0.0;
+  float w = 0.f;
+  bool al_g = false;
+  if (kGrad) {
+    w = (float)(sc->coef * (double)seg_size[seg]);
+    al_g = al_a && (reinterpret_cast<uintptr_t>(dlog_alpha + lo) & 15) == 0;
   }
-  if (!kGrad) {
-    double sum = 0.0;
 #pragma unroll
-    for (int i = 0; i < kL0PerThread; ++i)
-      if (j0 + i < hi) sum += (double)l0_pi(a[i], thr);
-    sum = block_sum_f64(sum, red);
-    if (threadIdx.x == 0) sc->partial[b] = sum;
-  } else {
-    const float w = (float)(sc->coef * (double)seg_size[seg]);
-    float gsum[kL0PerThread];
-#pragma unroll
-    for (int i = 0; i < kL0PerThread; ++i) {
-      // pi (1 - pi) = e / (1 + e)^2 with e = exp(-|alpha - thr|): no cancellation near pi = 1
-      const float e = expf(-fabsf(a[i] - thr));
-      const float q = 1.0f / (1.0f + e);
-      gsum[i] = w * e * q * q;
-    }
-    const bool vecg = vec && ((reinterpret_cast<uintptr_t>(dlog_alpha + j0) & 15) == 0);
-    if (vecg) {
-      float4 g = *reinterpret_cast<float4*>(dlog_alpha + j0);
-      g.x += gsum[0]; g.y += gsum[1]; g.z += gsum[2]; g.w += gsum[3];
-      *reinterpret_cast<float4*>(dlog_alpha + j0) = g;
+  for (int v = 0; v < kVec; ++v) {
+    const int64_t j0 = lo + ((int64_t)v * kL0Threads + threadIdx.x) * 4;
+    if (j0 >= hi) continue;
+    float a[4];
+    const bool full = j0 + 4 <= hi;
+    if (full && al_a) {
+      const float4 t = *reinterpret_cast<const float4*>(log_alpha + j0);
+      a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
     } else {
 #pragma unroll
-      for (int i = 0; i < kL0PerThread; ++i)
-        if (j0 + i < hi) dlog_alpha[j0 + i] += gsum[i];
+      for (int i = 0; i < 4; ++i) a[i] = (j0 + i < hi) ? log_alpha[j0 + i] : 0.f;
     }
+    if (!kGrad) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (j0 + i < hi) sum += (double)l0_pi(a[i], thr);
+    } else {
+      float gsum[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        // pi (1 - pi) = e / (1 + e)^2 with e = exp(-|alpha - thr|): no cancellation near pi = 1
+        const float e = __expf(-fabsf(a[i] - thr));
+        const float q = __fdividef(1.0f, 1.0f + e);
+        gsum[i] = w * e * q * q;
+      }
+      if (full && al_g) {
+        float4 g = *reinterpret_cast<float4*>(dlog_alpha + j0);
+        g.x += gsum[0]; g.y += gsum[1]; g.z += gsum[2]; g.w += gsum[3];
+        *reinterpret_cast<float4*>(dlog_alpha + j0) = g;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (j0 + i < hi) dlog_alpha[j0 + i] += gsum[i];
+      }
+    }
+  }
+  if (!kGrad) {
+    sum = block_sum_f64(sum, red);
+    if (threadIdx.x == 0) sc->partial[b] = sum;
   }
 }
 

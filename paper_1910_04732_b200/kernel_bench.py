@@ -1,0 +1,140 @@
+"""Timing of the memory-bound kernels and of the pruned-inference path.
+
+    python -m paper_1910_04732_b200.kernel_bench [--small]
+
+The per-step gate vectors of the workloads are a few tens of thousands of elements
+(launch-latency bound), so the HBM figures are taken on scaled inputs that are far
+larger than L2: 2^26 gates for the sampler and the expected-L0 / Lagrangian term,
+and a 65536 x 16384 factor pair for the rank gather.  Bytes are the algorithmic
+bytes of each call (what must be read and written once), time is the mean of CUDA
+event timings after warm-up.  The second table is the inference configuration:
+compaction once, then the compact forward against the uncompacted gated forward
+(both replayed from CUDA graphs so that host launch cost does not hide the kernels).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+from . import binding as b
+from . import build, inputs as I
+
+HC = tuple(float(np.float32(v)) for v in (I.BETA, I.GAMMA, I.ZETA))
+
+
+def timed(fn, iters=10, warmup=3, graph=False):
+    """Mean seconds per call.  graph=True replays a captured CUDA graph of one call, which takes
+    the host's launch cost (tens of microseconds from Python) out of microsecond-sized calls."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if graph:
+        g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        fn = g.replay
+        fn()
+        torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters * 1e-3
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--small", action="store_true", help="sizes for a profiler capture (a few hundred MB)")
+    args = ap.parse_args()
+    build.build()
+    b.load_library()
+    peak = 6650.0
+    try:
+        peak = float(json.load(open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))),
+                                                 "MEASURED_PEAKS.json")))["hbm_gbs"])
+    except Exception:
+        pass
+    rows = []
+    g = torch.Generator(device="cuda"); g.manual_seed(0)
+
+    # ---- gate sampler: 4 B read + 4 + 4 + 1 B written per gate
+    n = 1 << (24 if args.small else 26)
+    la = torch.randn(n, generator=g, device="cuda") * 1.5 + 1.0
+    z, d, m = torch.empty(n, device="cuda"), torch.empty(n, device="cuda"), torch.empty(n, dtype=torch.uint8, device="cuda")
+    t = timed(lambda: b.gate_sample(la, HC, 0, 0, z, m, d))
+    rows.append(("gate_sample_kernel", f"n = 2^{n.bit_length() - 1} gates", 13 * n, t))
+
+    # ---- expected L0 + Lagrangian with gradient: 4 B (pass 1) + 4 + 8 B (pass 2) per gate
+    n_seg = 64
+    off = torch.linspace(0, n, n_seg + 1).round().to(torch.int64).cuda()
+    size = torch.rand(n_seg, generator=g, device="cuda") * 4000 + 500
+    tg, lm = torch.tensor([0.3], device="cuda"), torch.tensor([0.3, 1.7], device="cuda")
+    out4, dla = torch.empty(4, device="cuda"), torch.zeros(n, device="cuda")
+    ws = b.alloc_workspace(b.workspace_bytes(b.OP_L0, n, 0, 0, n_seg, b.F32))
+    t = timed(lambda: b.expected_l0_lagrangian(la, off, size, HC, tg, lm, out4, None, dla, ws))
+    rows.append(("l0_chunk_kernel<0>+finalize+<1>", f"n = 2^{n.bit_length() - 1} gates, {n_seg} segments", 16 * n, t))
+    t = timed(lambda: b.expected_l0_lagrangian(la, off, size, HC, tg, lm, out4, None, None, ws))
+    rows.append(("l0_chunk_kernel<0>+finalize (no gradient)", "same", 4 * n, t))
+    del z, d, m, dla
+
+    # ---- rank compaction and gather, ~35 % of the components survive
+    r, d_in, d_out = (4096, 4096, 16384) if args.small else (16384, 16384, 65536)
+    a = torch.where(torch.rand(r, generator=g, device="cuda") < 0.35, 4.0, -4.0) + 0.1 * torch.randn(r, generator=g, device="cuda")
+    P = torch.randn(d_out, r, generator=g, device="cuda", dtype=torch.float32).bfloat16()
+    Q = torch.randn(r, d_in, generator=g, device="cuda", dtype=torch.float32).bfloat16()
+    Pc, Qc = torch.empty_like(P), torch.empty_like(Q)
+    idx, kd, zd = torch.empty(r, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda"), torch.empty(r, device="cuda")
+    t_sel = timed(lambda: b.compact_ranks(a, 0, HC, idx, kd, zd))
+    t_all = timed(lambda: b.compact_ranks(a, 0, HC, idx, kd, zd, P, Q, Pc, Qc))
+    k = int(kd.item())
+    rows.append(("compact_select_kernel", f"r = {r}", 4 * r * 6, t_sel))
+    rows.append(("gather_p_kernel + gather_q_kernel", f"r = {r}, d_in = {d_in}, d_out = {d_out}, k = {k}",
+                 2 * d_out * r + 2 * k * d_out + 4 * k * d_in + 4 * r, t_all - t_sel))
+    del P, Q, Pc, Qc
+
+    print(f"HBM peak used: {peak:.0f} GB/s (measured copy)\n")
+    print(f"{'kernel(s)':44s} {'size':58s} {'MB':>9s} {'us':>9s} {'GB/s':>8s} {'of peak':>8s}")
+    for name, what, nbytes, t in rows:
+        print(f"{name:44s} {what:58s} {nbytes / 1e6:9.1f} {t * 1e6:9.1f} {nbytes / t / 1e9:8.0f} {nbytes / t / 1e9 / peak:8.2f}")
+
+    # ---- pruned inference: d_in = 1024, d_out = 4096, r = 1024, ~35 % survive
+    w = I.WORKLOADS["infer"]
+    mtx = w.matrices[0]
+    prob = I.layer_problem(w, 0, 0, T=4096)
+    bf = torch.bfloat16
+
+    def dev(x):
+        t_ = b.padded(x.shape[0], x.shape[1], bf)
+        t_.copy_(torch.from_numpy(x).to(bf))
+        return t_
+    P, Q, X = dev(prob["P"]), dev(prob["Q"]), dev(prob["X"])
+    la = torch.from_numpy(prob["log_alpha"]).cuda()
+    idx, kd, zd = torch.empty(mtx.r, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda"), torch.empty(mtx.r, device="cuda")
+    Pc, Qc = b.padded(mtx.d_out, mtx.r, bf), b.padded(mtx.r, mtx.d_in, bf)
+    t_c = timed(lambda: b.compact_ranks(la, 0, HC, idx, kd, zd, P, Q, Pc, Qc))
+    k = int(kd.item())
+    print(f"\npruned inference, d_in={mtx.d_in} d_out={mtx.d_out} r={mtx.r}: k = {k} survive; compaction (select + gather) {t_c * 1e6:.1f} us")
+    print(f"{'T':>6s} {'compact fwd us':>15s} {'gated fwd us':>13s} {'speed-up':>9s} {'compact GFLOP/s':>16s} {'weight GB/s':>12s}")
+    for T in (1, 16, 256, 4096):
+        Xt = X[:T]
+        Y, H = b.padded(T, mtx.d_out, bf), b.padded(T, mtx.r, bf)
+        wsc = b.alloc_workspace(b.workspace_bytes(b.OP_COMPACT_FWD, T, mtx.d_in, mtx.d_out, k, b.BF16))
+        tc_ = timed(lambda: b.compact_fwd(Xt, Qc[:k], Pc[:, :k], Y, k, wsc), iters=50, graph=True)
+        tg_ = timed(lambda: b.gated_lowrank_fwd(Xt, Q, P, zd, Y, H, None), iters=50, graph=True)
+        flops = 2.0 * T * k * (mtx.d_in + mtx.d_out)
+        wbytes = 2.0 * k * (mtx.d_in + mtx.d_out)
+        print(f"{T:6d} {tc_ * 1e6:15.1f} {tg_ * 1e6:13.1f} {tg_ / tc_:9.2f} {flops / tc_ / 1e9:16.0f} {wbytes / tc_ / 1e9:12.0f}")
+    assert b.device_status() == b.OK
+
+
+if __name__ == "__main__":
+    main()

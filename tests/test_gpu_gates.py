@@ -135,8 +135,8 @@ def test_expected_l0_accumulates_and_is_bit_reproducible(b):
 
 def test_expected_l0_ragged_segments_and_large_single_segment(b):
     # segments with 0, 1, chunk-1, chunk, chunk+1 gates, and one segment spanning many chunks
-    counts = [0, 1, 1023, 1024, 1025, 0, 300000, 7]
-    sizes = [10.0, 820.0, 2510.0, 1.0, 4096.0, 5.0, 1536.0, 64.0]
+    counts = [0, 1, 1023, 4095, 4096, 4097, 0, 300000, 7]
+    sizes = [10.0, 820.0, 2510.0, 1.0, 4096.0, 77.0, 5.0, 1536.0, 64.0]
     w_alpha = np.random.default_rng(1).normal(0.5, 2.0, sum(counts)).astype(np.float32)
     offs = np.concatenate([[0], np.cumsum(counts)])
     dev = lambda a, dt: torch.from_numpy(np.asarray(a, dtype=dt)).cuda()
