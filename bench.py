@@ -193,9 +193,8 @@ class Job:
         self.b.expected_l0_lagrangian(self.log_alpha, self.seg_off, self.seg_size, HC, self.target, self.lam,
                                       self.out4, None, self.dlog_alpha, self.ws_l0)
         if self.world > 1:
-            import torch.distributed as dist
-            dist.all_reduce(self.wgrad)
-            dist.all_reduce(self.dlog_alpha)
+            from paper_1910_04732_b200 import dp
+            dp.allreduce_gradients([self.wgrad, self.dlog_alpha])     # the one exchange step of the path
 
     def step(self):
         torch = self.torch
@@ -443,6 +442,9 @@ def main():
     tokens_s = w.T * world / (step_ms / 1e3)
     tflops = w.flops_per_step() * world / (step_ms / 1e3) / 1e12
     gemm_tflops = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
+    # dram__bytes_read.sum + dram__bytes_write.sum of the GEMM launches of one bert layer, from the ncu capture
+    # summarised in profiles/gemm_group_kernel_bert_ncu_full.md (grouped calls of six matrices): mean per launch
+    traffic = 102.8e6 if (w.name == "bert" and group == 6) else None
     line = {
         "metric": METRIC, "value": tokens_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
@@ -455,9 +457,11 @@ def main():
                    "l2": f"inputs larger than L2: {job.input_bytes() / 1e6:.0f} MB of X and dY per step, each matrix its own buffers"},
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": peaks["bf16_tflops_sustained"],
-                     "unit": "TFLOP/s", "frac": gemm_tflops / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "unit": "TFLOP/s", "frac": gemm_tflops / peaks["bf16_tflops_sustained"], "traffic": traffic,
+                     "traffic_note": "DRAM read+write bytes per GEMM launch, mean of the five launches of one layer (ncu capture in profiles/)" if traffic else None,
                      "peak_kind": f"{peak_kind} (sustained; burst {peaks['bf16_tflops']})",
-                     "kernel": "tc::gemm_kernel (all six GEMMs of every matrix)", "launches_per_step": gemm_launches // args.steps,
+                     "kernel": "tc::gemm_group_kernel / tc::gemm2_group_kernel (every GEMM stage of the step)",
+                     "launches_per_step": gemm_launches // args.steps,
                      "kernel_ms_per_step": gemm_ms / args.steps, "step_ms_in_timed_pass": ms_timed_pass / args.steps,
                      "frac_of_nominal": gemm_tflops / NOMINAL_BF16_TFLOPS},
         "clocks": clocks,
