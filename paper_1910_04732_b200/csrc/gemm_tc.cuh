@@ -1,24 +1,27 @@
-// bf16 tensor-core GEMM for sm_100a: D[M,N] = sum_k A(m,k) B(n,k), fp32 accumulate.
+// bf16 tensor-core GEMM for sm_100a, shared pieces: D[M,N] = sum_k A(m,k) B(n,k), fp32 accumulate.
 //
-// One persistent, warp-specialised kernel serves all six GEMMs of the gated
-// factorized layer W = P diag(z) Q (Section 4.1 of the paper):
+// The kernels built from this header (gemm_group_kernel in gemm_tc_group.cuh, one CTA per
+// 128 x BN tile, and gemm2_group_kernel in gemm_tc2_group.cuh, a CTA pair per 256 x BN tile)
+// serve all six GEMMs of the gated factorized layer W = P diag(z) Q (Section 4.1 of the paper).
+// Both are persistent and warp-specialised:
 //   warp 0      TMA producer: cp.async.bulk.tensor (no multicast) into a ring of
 //               128-byte-swizzled shared-memory stages, completion on mbarriers
-//   warp 1      MMA issuer: one thread issues tcgen05.mma (128 x BN x 16, bf16 in,
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (K = 16 per instruction, bf16 in,
 //               fp32 accumulators in tensor memory), tcgen05.commit frees stages
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (one output row per thread),
-//               apply the gate / write bf16, or write fp32 split-K slices and the
-//               fused per-row dot product that becomes dz (hence dlog_alpha)
-// Two accumulator buffers in tensor memory let the epilogue of one tile overlap
-// the main loop of the next.  Operands may be K-major (rows of the row-major
-// matrix run along K) or MN-major (the backward GEMMs that contract over tokens
-// or over d_out read the same row-major tensors "transposed"), selected in the
-// shared-memory and instruction descriptors; nothing is transposed in memory.
-// Ragged sizes rely on TMA zero fill for loads and on guarded stores.
+//   warps 2..9  epilogue: tcgen05.ld the accumulator (one output row per thread), apply the
+//               gate, and either stage bf16 tiles in shared memory for a TMA store, or write
+//               weight gradients / fp32 split-K slices directly, with the fused per-row dot
+//               product that becomes dz (hence dlog_alpha)
+// Two accumulator buffers in tensor memory let the epilogue of one tile overlap the main loop
+// of the next.  Operands may be K-major (rows of the row-major matrix run along K) or MN-major
+// (the backward GEMMs that contract over tokens or over d_out read the same row-major tensors
+// "transposed"), selected in the shared-memory and instruction descriptors; nothing is
+// transposed in memory.  Ragged sizes rely on TMA zero fill for loads, TMA clipping for stores
+// and guarded per-thread stores.
 //
-// Every wait on an mbarrier is bounded: if it gives up, the kernel records
-// FLOP_ERR_TIMEOUT, all roles leave their loops, outstanding copies are waited
-// for (bounded), tensor memory is freed and the CTA returns.
+// Every wait on an mbarrier is bounded: if it gives up, the kernel records FLOP_ERR_TIMEOUT,
+// all roles leave their loops, outstanding copies are waited for (bounded), tensor memory is
+// freed and the CTA returns.
 #pragma once
 #include <cuda.h>
 

@@ -1,5 +1,6 @@
-// Two-CTA variant of the bf16 tensor-core GEMM: a cluster of two CTAs (the two SMs of a
-// TPC) computes one 256 x BN tile with tcgen05.mma.cta_group::2.
+// Two-CTA variant of the bf16 tensor-core GEMM, shared pieces (the kernel is gemm2_group_kernel
+// in gemm_tc2_group.cuh): a cluster of two CTAs (the two SMs of a TPC) computes one 256 x BN tile
+// with tcgen05.mma.cta_group::2.
 //
 // Why: in the one-CTA kernel every SM has to pull a full B tile (BN x 64) per k-block next
 // to its A tile, and the measured fill rate of an SM's shared memory (~54 B/clk) is what
@@ -8,7 +9,7 @@
 // Bytes per SM per k-block drop from 16 KB + BN*128 to 16 KB + BN*64.
 //
 // Protocol (rank = position in the pair, rank 0 leads):
-//   full[s]    lives in rank 0, expects two arrivals (one arrive.expect_tx per producer) plus
+//   full[s]    lives in rank 0, expects two arrivals (one relaxed arrive.expect_tx per producer) plus
 //              the bytes of both CTAs' TMA loads (each load names rank 0's barrier)
 //   empty[s]   one per CTA; rank 0's MMA thread releases a stage in both CTAs with one
 //              tcgen05.commit ... multicast::cluster

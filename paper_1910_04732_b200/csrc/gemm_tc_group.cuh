@@ -11,7 +11,8 @@
 //
 // Each problem keeps its own tensor maps, sizes, N tile, split-K factor and epilogue pointers in
 // a __grid_constant__ table; shared-memory stages and accumulator buffers are sized for the
-// largest N tile of the group.  Roles, barriers and bounded waits are those of gemm_kernel.
+// largest N tile of the group.  Roles, barriers, epilogues and bounded waits are described in
+// gemm_tc.cuh.  A single GEMM runs as a group of one.
 #pragma once
 #include "gemm_tc.cuh"
 
