@@ -122,3 +122,20 @@ def test_grouped_falls_back_per_problem_for_fp32_and_empty_problems(b):
     for prob, Y, *_ in es:
         assert rel_fro(host(Y), O.gated_lowrank_fwd(prob["X"], prob["Q"], prob["P"], np.ones(prob["m"].r))[2]) < 1e-5
     assert b.device_status() == b.OK
+
+
+@pytest.mark.parametrize("name", ["bert", "txl"])
+def test_grouped_full_size_layer_as_the_benchmark_issues_it(b, name):
+    """All matrices of one layer of the benchmark workload at the full token count, in ONE grouped
+    forward and ONE grouped backward call (the launch configuration bench.py times), every output
+    against the oracle."""
+    w = I.WORKLOADS[name]
+    es = _setup(b, w, 2, 0)
+    b.gated_lowrank_fwd_grouped([b.fwd_problem(e["X"], e["Q"], e["P"], e["z"], e["Yg"], e["Hg"]) for e in es])
+    b.gated_lowrank_bwd_grouped([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], e["z"], e["dzd"], e["Hg"], e["dXg"],
+                                               e["dPg"], e["dQg"], e["dlag"], e["wsg"]) for e in es])
+    assert b.device_status() == b.OK
+    for e in es:
+        _check_against_oracle(e, "g")
+        dead = e["z_np"] == 0
+        assert dead.any() and np.all(host(e["dQg"])[dead] == 0)          # closed gates: exact zeros in dQ
