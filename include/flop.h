@@ -165,6 +165,7 @@ typedef struct {
   const void* X; int64_t ldx; const void* Q; int64_t ldq; const void* P; int64_t ldp;
   const float* z; void* Y; int64_t ldy; void* H_save; int64_t ldh;
   int64_t T, d_in, d_out, r;
+  const int32_t* r_dev; /* nullable; see "Training on the active rank components" below */
 } flop_fwd_problem_t;
 
 typedef struct {
@@ -173,11 +174,49 @@ typedef struct {
   void* dX; int64_t lddx; void* dP; int64_t lddp; void* dQ; int64_t lddq; float* dlog_alpha;
   int64_t T, d_in, d_out, r;
   void* ws; size_t ws_bytes;
+  const int32_t* r_dev; /* nullable */
 } flop_bwd_problem_t;
 
 int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* problems, int n, int dt, void* stream);
 int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* problems, int n, int accumulate, int dt,
                                    int wgrad_dt, void* stream);
+
+/* Training on the active rank components only (Section 4.3, last paragraph: the
+ * mask is shared by the batch, so "parameters that are only active for the current
+ * batch" are selected and the matrix products run on smaller matrices).
+ *
+ * flop_active_ranks_gather, per problem: idx = {k : z_k > 0} ascending, pos = its
+ * inverse (-1 for closed gates), *k_dev = their number, z_c = z[idx],
+ * dz_dla_c = dz_dla[idx] (both zero beyond k), Q_c[c,:] = Q[idx[c],:] (NOT scaled by
+ * the gate), P_c[:,c] = P[:,idx[c]]; rows of Q_c / columns of P_c from k up to the
+ * next multiple of 64 are zero.  All compact buffers have the capacity of the full
+ * rank r.  bf16 only.
+ *
+ * The grouped forward/backward calls then take the compact buffers in place of
+ * P, Q, z, dz_dla, H_save, dP, dQ, dlog_alpha, with r = the capacity and
+ * r_dev = k_dev: the effective rank is read on the device, GEMM tiles beyond it are
+ * skipped and K loops stop at the 64-block holding component k-1.  Entries of the
+ * outputs beyond k are unspecified.  Y and dX are the full results.
+ *
+ * flop_active_ranks_scatter writes the full gradients: dP[:,idx] = dP_c,
+ * dQ[idx,:] = dQ_c, dlog_alpha[idx] = dlog_alpha_c and exact zeros elsewhere
+ * (accumulate != 0: += instead).  Any of the three outputs may be NULL. */
+typedef struct {
+  const float* z; const float* dz_dla; const void* P; int64_t ldp; const void* Q; int64_t ldq;
+  int64_t d_in, d_out, r;
+  int32_t* idx; int32_t* pos; int32_t* k_dev; float* z_c; float* dz_dla_c;
+  void* P_c; int64_t ldpc; void* Q_c; int64_t ldqc;
+} flop_active_gather_t;
+
+typedef struct {
+  const int32_t* idx; const int32_t* pos; const int32_t* k_dev; int64_t d_in, d_out, r;
+  const void* dP_c; int64_t lddpc; const void* dQ_c; int64_t lddqc; const float* dlog_alpha_c;
+  void* dP; int64_t lddp; void* dQ; int64_t lddq; float* dlog_alpha;
+} flop_active_scatter_t;
+
+int flop_active_ranks_gather(const flop_active_gather_t* problems, int n, int dt, void* stream);
+int flop_active_ranks_scatter(const flop_active_scatter_t* problems, int n, int accumulate, int wgrad_dt,
+                              void* stream);
 
 /* Expected size and augmented-Lagrangian penalty over all gates of all
  * matrices at once (Eq. 3 and Section 4.3).  Segment i (one weight matrix)

@@ -23,7 +23,8 @@ OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 EXPORTS = ("flop_status_string", "flop_device_status", "flop_launch_count", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
-           "flop_gated_lowrank_bwd_grouped", "flop_expected_l0_lagrangian",
+           "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
+           "flop_expected_l0_lagrangian",
            "flop_expected_l0_lagrangian_noalloc",
            "flop_compact_ranks", "flop_compact_fwd")
 
@@ -36,7 +37,8 @@ class FwdProblem(ctypes.Structure):
     _fields_ = [("X", ctypes.c_void_p), ("ldx", ctypes.c_int64), ("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64),
                 ("P", ctypes.c_void_p), ("ldp", ctypes.c_int64), ("z", ctypes.c_void_p), ("Y", ctypes.c_void_p),
                 ("ldy", ctypes.c_int64), ("H_save", ctypes.c_void_p), ("ldh", ctypes.c_int64),
-                ("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64)]
+                ("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
+                ("r_dev", ctypes.c_void_p)]
 
 
 class BwdProblem(ctypes.Structure):
@@ -46,7 +48,25 @@ class BwdProblem(ctypes.Structure):
                 ("dX", ctypes.c_void_p), ("lddx", ctypes.c_int64), ("dP", ctypes.c_void_p), ("lddp", ctypes.c_int64),
                 ("dQ", ctypes.c_void_p), ("lddq", ctypes.c_int64), ("dlog_alpha", ctypes.c_void_p),
                 ("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
-                ("ws", ctypes.c_void_p), ("ws_bytes", ctypes.c_size_t)]
+                ("ws", ctypes.c_void_p), ("ws_bytes", ctypes.c_size_t), ("r_dev", ctypes.c_void_p)]
+
+
+class ActiveGather(ctypes.Structure):
+    _fields_ = [("z", ctypes.c_void_p), ("dz_dla", ctypes.c_void_p), ("P", ctypes.c_void_p), ("ldp", ctypes.c_int64),
+                ("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64),
+                ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
+                ("idx", ctypes.c_void_p), ("pos", ctypes.c_void_p), ("k_dev", ctypes.c_void_p),
+                ("z_c", ctypes.c_void_p), ("dz_dla_c", ctypes.c_void_p),
+                ("P_c", ctypes.c_void_p), ("ldpc", ctypes.c_int64), ("Q_c", ctypes.c_void_p), ("ldqc", ctypes.c_int64)]
+
+
+class ActiveScatter(ctypes.Structure):
+    _fields_ = [("idx", ctypes.c_void_p), ("pos", ctypes.c_void_p), ("k_dev", ctypes.c_void_p),
+                ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
+                ("dP_c", ctypes.c_void_p), ("lddpc", ctypes.c_int64), ("dQ_c", ctypes.c_void_p), ("lddqc", ctypes.c_int64),
+                ("dlog_alpha_c", ctypes.c_void_p),
+                ("dP", ctypes.c_void_p), ("lddp", ctypes.c_int64), ("dQ", ctypes.c_void_p), ("lddq", ctypes.c_int64),
+                ("dlog_alpha", ctypes.c_void_p)]
 
 
 class FlopError(RuntimeError):
@@ -86,6 +106,8 @@ def load_library() -> ctypes.CDLL:
                                            i64, i64, i64, i64, ci, ci, vp, sz, vp]
     lib.flop_gated_lowrank_fwd_grouped.argtypes = [ctypes.POINTER(FwdProblem), ci, ci, vp]
     lib.flop_gated_lowrank_bwd_grouped.argtypes = [ctypes.POINTER(BwdProblem), ci, ci, ci, ci, vp]
+    lib.flop_active_ranks_gather.argtypes = [ctypes.POINTER(ActiveGather), ci, ci, vp]
+    lib.flop_active_ranks_scatter.argtypes = [ctypes.POINTER(ActiveScatter), ci, ci, ci, vp]
     lib.flop_expected_l0_lagrangian.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp,
                                                 vp, sz, vp]
     lib.flop_expected_l0_lagrangian_noalloc.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp, vp]
@@ -223,20 +245,44 @@ def _p(t: Optional[torch.Tensor]):
     return None if t is None else t.data_ptr()
 
 
-def fwd_problem(X, Q, P, z, Y, H_save) -> FwdProblem:
+def fwd_problem(X, Q, P, z, Y, H_save, r_dev=None) -> FwdProblem:
     T, d_in = X.shape
     d_out, r = P.shape
     return FwdProblem(_p(X), _ld(X), _p(Q), _ld(Q), _p(P), _ld(P), _p(z), _p(Y), _ld(Y), _p(H_save), _ld(H_save),
-                      T, d_in, d_out, r)
+                      T, d_in, d_out, r, _p(r_dev))
 
 
-def bwd_problem(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws) -> BwdProblem:
+def bwd_problem(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws, r_dev=None) -> BwdProblem:
     T, d_in = X.shape
     d_out, r = P.shape
     ld = lambda t: _ld(t) if t is not None else 0
     return BwdProblem(_p(dY), _ld(dY), _p(X), _ld(X), _p(Q), _ld(Q), _p(P), _ld(P), _p(z), _p(dz_dla), _p(H_save),
                       _ld(H_save), _p(dX), ld(dX), _p(dP), ld(dP), _p(dQ), ld(dQ), _p(dlog_alpha), T, d_in, d_out, r,
-                      _p(ws), ws.numel() if ws is not None else 0)
+                      _p(ws), ws.numel() if ws is not None else 0, _p(r_dev))
+
+
+def active_gather_problem(z, dz_dla, P, Q, idx, pos, k_dev, z_c, dz_dla_c, P_c, Q_c) -> ActiveGather:
+    d_out, r = P.shape
+    d_in = Q.shape[1]
+    return ActiveGather(_p(z), _p(dz_dla), _p(P), _ld(P), _p(Q), _ld(Q), d_in, d_out, r, _p(idx), _p(pos), _p(k_dev),
+                        _p(z_c), _p(dz_dla_c), _p(P_c), _ld(P_c), _p(Q_c), _ld(Q_c))
+
+
+def active_scatter_problem(idx, pos, k_dev, d_in, d_out, r, dP_c, dQ_c, dla_c, dP, dQ, dla) -> ActiveScatter:
+    ld = lambda t: _ld(t) if t is not None else 0
+    return ActiveScatter(_p(idx), _p(pos), _p(k_dev), d_in, d_out, r, _p(dP_c), ld(dP_c), _p(dQ_c), ld(dQ_c), _p(dla_c),
+                         _p(dP), ld(dP), _p(dQ), ld(dQ), _p(dla))
+
+
+def active_ranks_gather(problems, dt: int = BF16) -> None:
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_active_ranks_gather(arr, len(arr), dt, _stream()), "flop_active_ranks_gather")
+
+
+def active_ranks_scatter(problems, accumulate: bool = False, wgrad_dt: int = BF16) -> None:
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_active_ranks_scatter(arr, len(arr), int(accumulate), wgrad_dt, _stream()),
+           "flop_active_ranks_scatter")
 
 
 def problem_array(problems):

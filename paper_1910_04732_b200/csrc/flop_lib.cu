@@ -25,6 +25,7 @@
 #include "gemm_tc2_group.cuh"
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
+#include "active_ranks.cuh"
 
 using namespace flop;
 typedef __nv_bfloat16 bf16;
@@ -270,8 +271,11 @@ TcEpilogue store_epilogue(void* out, int64_t ldo, const float* col_scale) {
 struct TcJob {
   Operand A, B;
   int64_t M, N, K;
-  TcPlan pl;       // one-CTA plan (pl.cta2 == 0)
+  TcPlan pl;
   TcEpilogue ep;
+  const int* dyn_m = nullptr;   // effective sizes on the device (see tc::Params), nullable
+  const int* dyn_n = nullptr;
+  const int* dyn_k = nullptr;
 };
 
 template <bool A_MN, bool B_MN, int EPI>
@@ -335,6 +339,7 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
       p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
       p.wg_out = j.ep.wg_out; p.wg_f32 = j.ep.wg_f32; p.row_scale = j.ep.row_scale; p.accumulate = j.ep.accumulate;
+      p.dyn_m = j.dyn_m; p.dyn_n = j.dyn_n; p.dyn_k = j.dyn_k;
       // bf16 tiles that are plainly overwritten leave through a TMA store (64 x 32 boxes of the output)
       void* tma_dst = j.ep.kind == tc::EPI_STORE ? (void*)j.ep.out
                       : (j.ep.kind == tc::EPI_WGRAD && !j.ep.wg_f32 && !j.ep.accumulate) ? j.ep.wg_out : nullptr;
@@ -366,7 +371,8 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
 // A single GEMM is a group of one.
 int launch_tc(const Operand& A, const Operand& B, int64_t M, int64_t N, int64_t K, const TcPlan& pl,
               const TcEpilogue& ep, cudaStream_t st) {
-  return launch_tc_group(std::vector<TcJob>{TcJob{A, B, M, N, K, pl, ep}}, st);
+  TcJob j{A, B, M, N, K, pl, ep};
+  return launch_tc_group(std::vector<TcJob>{j}, st);
 }
 
 // ---- tile shape for a whole group: one (pair?, N tile) for all jobs of a launch, no split-K
@@ -906,6 +912,7 @@ int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, 
   if (!grouped) {   // fp32 storage or an empty problem: one call per problem
     for (int i = 0; i < n; ++i) {
       const flop_fwd_problem_t& a = pr[i];
+      if (a.r_dev) return FLOP_ERR_UNSUPPORTED;   // a device-side rank needs the grouped bf16 kernels
       FLOP_TRY(flop_gated_lowrank_fwd(a.X, a.ldx, a.Q, a.ldq, a.P, a.ldp, a.z, a.Y, a.ldy, a.H_save, a.ldh, a.T, a.d_in, a.d_out,
                                       a.r, dt, nullptr, 0, stream));
     }
@@ -925,10 +932,14 @@ int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, 
       return FLOP_ERR_INVALID_ARG;
     if (!bf16_ok(a.Y, a.ldy) || !bf16_ok(a.P, a.ldp) || !bf16_ok(a.H_save, a.ldh) || !bf16_ok(a.X, a.ldx) || !bf16_ok(a.Q, a.ldq))
       return FLOP_ERR_UNSUPPORTED;
-    g1.push_back({{a.X, a.ldx, false}, {a.Q, a.ldq, false}, a.T, a.r, a.d_in, fixed_plan(a.T, a.r, a.d_in, s1.bn, s1.cta2),
-                  store_epilogue(a.H_save, a.ldh, a.z)});
-    g2.push_back({{a.H_save, a.ldh, false}, {a.P, a.ldp, false}, a.T, a.d_out, a.r, fixed_plan(a.T, a.d_out, a.r, s2.bn, s2.cta2),
-                  store_epilogue(a.Y, a.ldy, nullptr)});
+    TcJob j1{{a.X, a.ldx, false}, {a.Q, a.ldq, false}, a.T, a.r, a.d_in, fixed_plan(a.T, a.r, a.d_in, s1.bn, s1.cta2),
+             store_epilogue(a.H_save, a.ldh, a.z)};
+    TcJob j2{{a.H_save, a.ldh, false}, {a.P, a.ldp, false}, a.T, a.d_out, a.r, fixed_plan(a.T, a.d_out, a.r, s2.bn, s2.cta2),
+             store_epilogue(a.Y, a.ldy, nullptr)};
+    j1.dyn_n = a.r_dev;   // only the first *r_dev rank components exist this step
+    j2.dyn_k = a.r_dev;
+    g1.push_back(j1);
+    g2.push_back(j2);
   }
   cudaStream_t st = (cudaStream_t)stream;
   FLOP_TRY(launch_tc_group(g1, st));   // H' = (X Q^T) * z for every problem
@@ -948,6 +959,7 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
   if (!grouped) {
     for (int i = 0; i < n; ++i) {
       const flop_bwd_problem_t& a = pr[i];
+      if (a.r_dev) return FLOP_ERR_UNSUPPORTED;
       FLOP_TRY(flop_gated_lowrank_bwd(a.dY, a.lddy, a.X, a.ldx, a.Q, a.ldq, a.P, a.ldp, a.z, a.dz_dla, a.H_save, a.ldh, a.dX,
                                       a.lddx, a.dP, a.lddp, a.dQ, a.lddq, a.dlog_alpha, accumulate, a.T, a.d_in, a.d_out, a.r, dt,
                                       wgrad_dt, a.ws, a.ws_bytes, stream));
@@ -992,17 +1004,23 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     const flop_bwd_problem_t& a = pr[i];
     const BwdWs& w = wss[i];
     const bool need_m = a.dQ || a.dlog_alpha;
-    g3.push_back({{a.dY, a.lddy, false}, {a.P, a.ldp, true}, a.T, a.r, a.d_out, fixed_plan(a.T, a.r, a.d_out, s3.bn, s3.cta2),
-                  store_epilogue(w.dH, w.lddh, nullptr)});
+    TcJob j3{{a.dY, a.lddy, false}, {a.P, a.ldp, true}, a.T, a.r, a.d_out, fixed_plan(a.T, a.r, a.d_out, s3.bn, s3.cta2),
+             store_epilogue(w.dH, w.lddh, nullptr)};
+    j3.dyn_n = a.r_dev;
+    g3.push_back(j3);
     int n_part = w.n_part;
     if (a.dP) {
       if (direct) {
-        g4.push_back({{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, direct_plan(a.d_out, a.r, a.T),
-                      wgrad_epilogue(a.dP, a.lddp, wgrad_dt, nullptr, accumulate)});
+        TcJob j{{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, direct_plan(a.d_out, a.r, a.T),
+                wgrad_epilogue(a.dP, a.lddp, wgrad_dt, nullptr, accumulate)};
+        j.dyn_n = a.r_dev;
+        g4.push_back(j);
       } else {
         TcEpilogue e{};
         e.kind = tc::EPI_SLICE; e.slices = w.slices_p; e.slice_elems = w.slice_elems_p; e.ld_slice = w.ld_slice_p;
-        g4.push_back({{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, w.plan_p, e});
+        TcJob j{{a.dY, a.lddy, true}, {a.H_save, a.ldh, true}, a.d_out, a.r, a.T, w.plan_p, e};
+        j.dyn_n = a.r_dev;
+        g4.push_back(j);
       }
     }
     if (need_m) {
@@ -1019,7 +1037,9 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
         e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
       }
       if (a.dlog_alpha) { e.qdot = (const bf16*)a.Q; e.ldq = a.ldq; e.dz_part = w.dz_part; e.dz_stride = a.r; }
-      g5.push_back({{w.dH, w.lddh, true}, {a.X, a.ldx, true}, a.r, a.d_in, a.T, pl, e});
+      TcJob j5{{w.dH, w.lddh, true}, {a.X, a.ldx, true}, a.r, a.d_in, a.T, pl, e};
+      j5.dyn_m = a.r_dev;
+      g5.push_back(j5);
     }
     BwdFinishArgs f{};
     f.slices_p = w.slices_p; f.n_slices_p = w.plan_p.splits; f.slice_elems_p = w.slice_elems_p; f.ld_slice_p = w.ld_slice_p;
@@ -1029,9 +1049,12 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     f.Q = (const bf16*)a.Q; f.ldq = a.ldq; f.Qz = a.dX ? (bf16*)w.Qz : nullptr; f.ldqz = w.ldqz;
     f.dz_part = w.dz_part; f.n_part = n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.dlog_alpha; f.accumulate = accumulate;
     fin.push_back(f);
-    if (a.dX)
-      g6.push_back({{w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, a.T, a.d_in, a.r, fixed_plan(a.T, a.d_in, a.r, s6.bn, s6.cta2),
-                    store_epilogue(a.dX, a.lddx, nullptr)});
+    if (a.dX) {
+      TcJob j6{{w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, a.T, a.d_in, a.r, fixed_plan(a.T, a.d_in, a.r, s6.bn, s6.cta2),
+               store_epilogue(a.dX, a.lddx, nullptr)};
+      j6.dyn_k = a.r_dev;
+      g6.push_back(j6);
+    }
   }
   if (direct) {   // both weight-gradient products of every matrix in one work list
     g4.insert(g4.end(), g5.begin(), g5.end());
@@ -1057,6 +1080,70 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     }
   }
   FLOP_TRY(launch_tc_group(g6, st));   // dX = dH' (diag(z) Q)
+  return FLOP_OK;
+}
+
+int flop_active_ranks_gather(const flop_active_gather_t* pr, int n, int dt, void* stream) {
+  if (n < 0 || (n > 0 && !pr)) return FLOP_ERR_INVALID_ARG;
+  if (dt != FLOP_BF16) return FLOP_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int i0 = 0; i0 < n; i0 += kActiveGroup) {
+    ActiveGatherGroup g;
+    memset(&g, 0, sizeof(g));
+    int max_blocks = 0, max_r = 0;
+    for (; g.n < kActiveGroup && i0 + g.n < n; ++g.n) {
+      const flop_active_gather_t& a = pr[i0 + g.n];
+      if (a.r <= 0 || a.d_in <= 0 || a.d_out <= 0 || a.r > INT32_MAX / 2 || a.d_in > INT32_MAX || a.d_out > INT32_MAX / 2)
+        return FLOP_ERR_INVALID_ARG;
+      if (!a.z || !a.P || !a.Q || !a.idx || !a.pos || !a.k_dev || !a.z_c || !a.P_c || !a.Q_c || a.ldp < a.r || a.ldq < a.d_in ||
+          a.ldpc < a.r || a.ldqc < a.d_in || (a.dz_dla_c && !a.dz_dla))
+        return FLOP_ERR_INVALID_ARG;
+      if (!bf16_ok(a.P, a.ldp) || !bf16_ok(a.Q, a.ldq) || !bf16_ok(a.P_c, a.ldpc) || !bf16_ok(a.Q_c, a.ldqc)) return FLOP_ERR_UNSUPPORTED;
+      if ((size_t)a.r * 2 > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
+      ActiveGather& o = g.a[g.n];
+      o.z = a.z; o.dz_dla = a.dz_dla; o.P = (const bf16*)a.P; o.ldp = a.ldp; o.Q = (const bf16*)a.Q; o.ldq = a.ldq;
+      o.r = (int)a.r; o.d_in = (int)a.d_in; o.d_out = (int)a.d_out; o.idx = a.idx; o.pos = a.pos; o.k_dev = a.k_dev;
+      o.z_c = a.z_c; o.dz_dla_c = a.dz_dla_c; o.P_c = (bf16*)a.P_c; o.ldpc = a.ldpc; o.Q_c = (bf16*)a.Q_c; o.ldqc = a.ldqc;
+      max_blocks = std::max(max_blocks, o.r + o.d_out);
+      max_r = std::max(max_r, o.r);
+    }
+    launch_k(active_select_kernel, dim3(g.n), dim3(1024), (size_t)0, st, g);
+    const size_t smem = (size_t)max_r * 2;
+    if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(active_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    launch_k(active_gather_kernel, dim3(max_blocks, g.n), dim3(256), smem, st, g);
+    count_launch(2);
+    FLOP_CUDA(cudaGetLastError());
+  }
+  return FLOP_OK;
+}
+
+int flop_active_ranks_scatter(const flop_active_scatter_t* pr, int n, int accumulate, int wgrad_dt, void* stream) {
+  if (n < 0 || (n > 0 && !pr) || !valid_dt(wgrad_dt)) return FLOP_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int i0 = 0; i0 < n; i0 += kActiveGroup) {
+    ActiveScatterGroup g;
+    memset(&g, 0, sizeof(g));
+    g.accumulate = accumulate;
+    int max_blocks = 0;
+    for (; g.n < kActiveGroup && i0 + g.n < n; ++g.n) {
+      const flop_active_scatter_t& a = pr[i0 + g.n];
+      if (a.r <= 0 || a.d_in <= 0 || a.d_out <= 0 || a.r > INT32_MAX / 2 || a.d_in > INT32_MAX || a.d_out > INT32_MAX / 2 || !a.idx ||
+          !a.pos || !a.k_dev)
+        return FLOP_ERR_INVALID_ARG;
+      if ((a.dP && (!a.dP_c || a.lddp < a.r || a.lddpc < a.r)) || (a.dQ && (!a.dQ_c || a.lddq < a.d_in || a.lddqc < a.d_in)) ||
+          (a.dlog_alpha && !a.dlog_alpha_c))
+        return FLOP_ERR_INVALID_ARG;
+      ActiveScatter& o = g.a[g.n];
+      o.idx = a.idx; o.pos = a.pos; o.k_dev = a.k_dev; o.r = (int)a.r; o.d_in = (int)a.d_in; o.d_out = (int)a.d_out;
+      o.dP_c = a.dP_c; o.lddpc = a.lddpc; o.dQ_c = a.dQ_c; o.lddqc = a.lddqc; o.dla_c = a.dlog_alpha_c;
+      o.dP = a.dP; o.lddp = a.lddp; o.dQ = a.dQ; o.lddq = a.lddq; o.dla = a.dlog_alpha;
+      max_blocks = std::max(max_blocks, o.r + o.d_out);
+    }
+    if (wgrad_dt == FLOP_BF16) launch_k(active_scatter_kernel<bf16>, dim3(max_blocks, g.n), dim3(256), (size_t)0, st, g);
+    else                       launch_k(active_scatter_kernel<float>, dim3(max_blocks, g.n), dim3(256), (size_t)0, st, g);
+    count_launch();
+    FLOP_CUDA(cudaGetLastError());
+  }
   return FLOP_OK;
 }
 

@@ -58,6 +58,12 @@ struct Params {
   // EPI_WGRAD (splits == 1): wg_out[m*ldo + n] (=|+=) row_scale[m] * acc, bf16 or fp32; same fused row dot
   void* wg_out; int wg_f32; const float* row_scale; int accumulate;
   int tma_store;   // 1: bf16 output tiles leave through shared memory and a TMA store (tensor map given)
+  // Sizes known only on the device (nullable): the effective M, N, K are min(capacity, *ptr).  Used when the
+  // rank dimension is the number of active components of a sampled mask.  Tiles outside the effective
+  // extent are skipped by every role; the K loop stops at the 64-block that holds the last effective k, and
+  // the N extent is rounded up to 64, so operands must be zero between the effective size and the next
+  // multiple of 64.  An effective size of 0 is treated as 1 (an all-zero block).
+  const int* dyn_m; const int* dyn_n; const int* dyn_k;
 };
 
 enum { EPI_STORE = 0, EPI_SLICE = 1, EPI_WGRAD = 2 };
@@ -408,13 +414,13 @@ __device__ __forceinline__ void stage_chunk(const Params& p, const uint32_t (&v)
 // the ragged edges.  Otherwise (fp32 outputs, accumulate, split-K slices) each thread stores its row.
 template <int EPI, bool kClusterArrive>
 __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap* tmap_out, uint32_t store_buf, uint32_t t_acc,
-                                             int row0, int n_base, int split, int tn, int warp, int lane,
+                                             int row0, int n_base, int n_limit, int split, int tn, int warp, int lane,
                                              uint32_t release_bar) {
   const int q = warp & 3, h = (warp - 2) >> 2;
   const int row = row0 + q * 32 + lane;
   const bool row_ok = row < p.M;
   const uint32_t t_row = t_acc + ((uint32_t)(q * 32) << 16);
-  const int nchunks = (min(p.bn, p.N - n_base) + 31) >> 5;   // 32-column chunks that hold columns of D
+  const int nchunks = (min(p.bn, n_limit - n_base) + 31) >> 5;   // 32-column chunks that hold columns of D
   const int ngroups = (nchunks + 1) >> 1;                    // 64-column groups
   float dot = 0.f;
   bool released = false;

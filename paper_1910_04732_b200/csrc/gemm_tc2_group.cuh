@@ -62,7 +62,8 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t phase = 0;
       bool ok = true;
       for (int w = pair; w < total && ok; w += npairs) {
-        const GroupItem it = decode_group(gp, w);
+        const GroupItem it = decode_group(gp, w, BM2);
+        if (!it.active) continue;
         const GroupProblem& pr = gp.prob[it.g];
         const int half_n = pr.p.bn >> 1;
         const uint32_t tx = kATileBytes + (uint32_t)half_n * BK * 2;
@@ -105,7 +106,8 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int w = pair; w < total && ok; w += npairs) {
-        const GroupItem it = decode_group(gp, w);
+        const GroupItem it = decode_group(gp, w, BM2);
+        if (!it.active) continue;
         const uint32_t idesc = instr_desc2(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait2(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
@@ -134,13 +136,14 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int w = pair; w < total && ok; w += npairs) {
-      const GroupItem it = decode_group(gp, w);
+      const GroupItem it = decode_group(gp, w, BM2);
+        if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
       if (!mbar_wait2(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      run_epilogue<EPI, true>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.split, it.tn,
+      run_epilogue<EPI, true>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.n_limit, it.split, it.tn,
                               warp, lane, map_to_cta(tempty_bar(acc), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }

@@ -36,16 +36,28 @@ struct GroupParams {
   int bn_max;       // largest N tile: sizes the stages and the accumulator buffers
 };
 
-struct GroupItem { int g, tm, tn, split, kb0, kb1; };
+struct GroupItem { int g, tm, tn, split, kb0, kb1, n_limit; bool active; };
 
-__device__ __forceinline__ GroupItem decode_group(const GroupParams& gp, int w) {
+// Work item w of the group; bm = rows of D per tile (128, or 256 for a CTA pair).  When a problem
+// carries device-side sizes the item may lie outside the effective extent (active = false: every
+// role skips it, so stage and accumulator phases stay in step) or have a shorter K loop.
+__device__ __forceinline__ GroupItem decode_group(const GroupParams& gp, int w, int bm) {
   int g = 0;
 #pragma unroll
   for (int i = 1; i < kMaxGroup; ++i)
     if (i < gp.n && w >= gp.prob[i].work_begin) g = i;
   const Params& p = gp.prob[g].p;
   const WorkItem it = decode(p, w - gp.prob[g].work_begin);
-  return GroupItem{g, it.tm, it.tn, it.split, it.kb0, it.kb1};
+  GroupItem o{g, it.tm, it.tn, it.split, it.kb0, it.kb1, p.N, true};
+  if (p.dyn_m || p.dyn_n || p.dyn_k) {
+    const int m_eff = p.dyn_m ? max(1, min(p.M, __ldg(p.dyn_m))) : p.M;
+    const int n_eff = p.dyn_n ? max(1, min(p.N, __ldg(p.dyn_n))) : p.N;
+    const int k_eff = p.dyn_k ? max(1, min(p.K, __ldg(p.dyn_k))) : p.K;
+    if (p.dyn_n) o.n_limit = min(p.N, (n_eff + 63) & ~63);
+    o.kb1 = min(o.kb1, (k_eff + BK - 1) / BK);
+    o.active = o.tm * bm < m_eff && o.tn * p.bn < n_eff && o.kb0 < o.kb1;
+  }
+  return o;
 }
 
 template <bool A_MN, bool B_MN, int EPI>
@@ -94,7 +106,8 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       int armed = 0;
       bool ok = true;
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        const GroupItem it = decode_group(gp, w);
+        const GroupItem it = decode_group(gp, w, BM);
+        if (!it.active) continue;
         const GroupProblem& pr = gp.prob[it.g];
         const int bn = pr.p.bn;
         const uint32_t tx = kATileBytes + (uint32_t)bn * BK * 2;
@@ -140,7 +153,8 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        const GroupItem it = decode_group(gp, w);
+        const GroupItem it = decode_group(gp, w, BM);
+        if (!it.active) continue;
         const uint32_t idesc = instr_desc(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
@@ -169,13 +183,14 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-      const GroupItem it = decode_group(gp, w);
+      const GroupItem it = decode_group(gp, w, BM);
+        if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      run_epilogue<EPI, false>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM, it.tn * p.bn, it.split, it.tn, warp, lane,
+      run_epilogue<EPI, false>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM, it.tn * p.bn, it.n_limit, it.split, it.tn, warp, lane,
                                tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
