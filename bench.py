@@ -172,6 +172,47 @@ class Job:
         self.graph = None
         self.world = 1
 
+    def enable_active_ranks(self):
+        """Buffers and argument arrays for training on the active components only (z_k > 0): per layer one
+        gather, the grouped forward and backward with the rank read on the device, one scatter."""
+        torch, b = self.torch, self.b
+        bf = torch.bfloat16
+        dev = self.log_alpha.device
+        self.active_groups = []
+        for e in self.mats:
+            m = e["m"]
+            if "ws" not in e:
+                e["ws"] = b.alloc_workspace(b.workspace_bytes(b.OP_BWD, self.w.T, m.d_in, m.d_out, m.r, b.BF16), dev)
+            e["idx"] = torch.zeros(m.r, dtype=torch.int32, device=dev)
+            e["pos"] = torch.zeros(m.r, dtype=torch.int32, device=dev)
+            e["k"] = torch.zeros(1, dtype=torch.int32, device=dev)
+            e["zc"], e["dzc"], e["dlac"] = (torch.zeros(m.r, device=dev) for _ in range(3))
+            e["Pc"], e["Qc"] = b.padded(m.d_out, m.r, bf, dev), b.padded(m.r, m.d_in, bf, dev)
+            e["dPc"], e["dQc"] = b.padded(m.d_out, m.r, bf, dev), b.padded(m.r, m.d_in, bf, dev)
+        g = self.group if self.group > 0 else len(self.w.matrices)
+        for i in range(0, len(self.mats), g):
+            ch = self.mats[i:i + g]
+            z = lambda e: self.z[e["lo"]:e["hi"]]
+            gat = b.problem_array([b.active_gather_problem(z(e), self.dz_dla[e["lo"]:e["hi"]], e["P"], e["Q"], e["idx"], e["pos"],
+                                                           e["k"], e["zc"], e["dzc"], e["Pc"], e["Qc"]) for e in ch])
+            fwd = b.problem_array([b.fwd_problem(e["X"], e["Qc"], e["Pc"], e["zc"], e["Y"], e["H"], r_dev=e["k"]) for e in ch])
+            bwd = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Qc"], e["Pc"], e["zc"], e["dzc"], e["H"], e["dX"], e["dPc"],
+                                                 e["dQc"], e["dlac"], e["ws"], r_dev=e["k"]) for e in ch])
+            sca = b.problem_array([b.active_scatter_problem(e["idx"], e["pos"], e["k"], e["m"].d_in, e["m"].d_out, e["m"].r,
+                                                            e["dPc"], e["dQc"], e["dlac"], e["dP"], e["dQ"],
+                                                            self.dlog_alpha[e["lo"]:e["hi"]]) for e in ch])
+            self.active_groups.append((gat, fwd, bwd, sca))
+
+    def step_active(self):
+        b = self.b
+        self.sample_gates()
+        for gat, fwd, bwd, sca in self.active_groups:
+            b.active_ranks_gather(gat)
+            b.gated_lowrank_fwd_grouped(fwd)
+            b.gated_lowrank_bwd_grouped(bwd)
+            b.active_ranks_scatter(sca)
+        self.finish()
+
     def input_bytes(self) -> int:
         return sum(e["X"].numel() * 2 + e["dY"].numel() * 2 for e in self.mats)
 
@@ -221,21 +262,23 @@ class Job:
         self.finish()
 
 
-def capture_step(job: Job):
+def capture_step(job: Job, fn=None):
     """One whole step captured in a CUDA graph (the library's launches, programmatic dependent
     launch edges included); replays cost one host call instead of ~25."""
     import torch
     g = torch.cuda.CUDAGraph()
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
+    fn = job.step if fn is None else fn
     with torch.cuda.stream(side):
-        job.step()                      # every kernel configured before capture
+        fn()                            # every kernel configured before capture
         torch.cuda.synchronize()
         with torch.cuda.graph(g, stream=side):
-            job.step()
+            fn()
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     job.graph = g
+    return g
 
 
 def time_steps(job: Job, steps: int, world: int, use_graph: bool = False):
@@ -369,6 +412,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-active", action="store_true", help="skip the extra active-rank-training measurement")
     ap.add_argument("--no-graph", action="store_true", help="issue every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--group", type=int, default=-1, help="matrices per grouped call (0: one call per matrix; default: one layer)")
     ap.add_argument("--streams", type=int, default=1, help="streams over which independent matrices are issued")
@@ -424,6 +468,35 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     assert b.device_status() == b.OK
 
+    # Extra (not the headline): the same step computed on the active rank components only.
+    active = None
+    if world == 1 and not args.no_active:
+        job.enable_active_ranks()
+        for _ in range(3):
+            job.step_active()
+        torch.cuda.synchronize()
+        run = job.step_active
+        if use_graph:
+            g_act = capture_step(job, job.step_active)
+            run = g_act.replay
+            job.graph = None
+        k_steps = max(3, min(args.steps, 50))
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(k_steps):
+            run()
+        a1.record()
+        torch.cuda.synchronize()
+        act_ms = a0.elapsed_time(a1) / k_steps
+        frac = float(job.mask.float().mean().item())
+        active = {"ms_per_step": act_ms, "value": w.T / (act_ms / 1e3), "unit": "tokens/s",
+                  "active_fraction_last_step": frac,
+                  "note": "gather z>0 components, grouped fwd/bwd with device-side rank, scatter; same outputs as the dense step"}
+        assert b.device_status() == b.OK
+
     e2e = None
     if not args.no_e2e:
         e2e_ms, h2d, d2h = time_e2e(job, max(3, min(args.steps, 20)), world)
@@ -468,6 +541,8 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
+    if active is not None:
+        line["active_rank_training"] = active
     if world == 1 and not args.no_cpu_baseline:
         dt, sample, threads = oracle_sample(w)
         line["cpu_baseline"] = {"value": w.T / (dt * w.layers), "unit": "tokens/s", "cores": threads, "kind": "oracle",

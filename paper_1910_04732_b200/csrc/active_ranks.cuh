@@ -63,39 +63,43 @@ active_select_kernel(const __grid_constant__ ActiveGatherGroup g) {
 
 __device__ __forceinline__ int pad64(int k) { return (max(k, 1) + 63) & ~63; }
 
-// blockIdx.x < r: Q row task (compact row c = blockIdx.x); otherwise P row task (row i = blockIdx.x - r).
-__global__ void __launch_bounds__(256)
-active_gather_kernel(const __grid_constant__ ActiveGatherGroup g) {
+constexpr int kActiveWarps = 8;   // one row task per warp, eight per block
+
+// Row task t = blockIdx.x * 8 + warp: t < r is compact row t of Q_c, otherwise row t - r of P_c.
+__global__ void __launch_bounds__(32 * kActiveWarps)
+active_gather_kernel(const __grid_constant__ ActiveGatherGroup g, int smem_row_elems) {
   pdl_wait();
   pdl_launch_dependents();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const ActiveGather& a = g.a[blockIdx.y];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x * kActiveWarps + warp;
   const int k = *a.k_dev, kp = min(a.r, pad64(k));
-  if ((int)blockIdx.x < a.r) {
-    const int c = blockIdx.x;
+  if (t < a.r) {
+    const int c = t;
     if (c >= kp) return;
     __nv_bfloat16* o = a.Q_c + (int64_t)c * a.ldqc;
     if (c < k) {
       const __nv_bfloat16* q = a.Q + (int64_t)a.idx[c] * a.ldq;
-      for (int j = threadIdx.x * 8; j < a.d_in; j += blockDim.x * 8) {     // rows are 16-byte aligned (ld % 8 == 0)
+      for (int j = lane * 8; j < a.d_in; j += 32 * 8) {     // rows are 16-byte aligned (ld % 8 == 0)
         if (j + 8 <= a.d_in) *reinterpret_cast<uint4*>(o + j) = *reinterpret_cast<const uint4*>(q + j);
         else for (int e = j; e < a.d_in; ++e) o[e] = q[e];
       }
     } else {
-      for (int j = threadIdx.x; j < a.d_in; j += blockDim.x) o[j] = __float2bfloat16_rn(0.f);
+      for (int j = lane; j < a.d_in; j += 32) o[j] = __float2bfloat16_rn(0.f);
     }
   } else {
-    const int i = (int)blockIdx.x - a.r;
+    const int i = t - a.r;
     if (i >= a.d_out) return;
-    __nv_bfloat16* row = reinterpret_cast<__nv_bfloat16*>(smem_raw);
+    __nv_bfloat16* row = reinterpret_cast<__nv_bfloat16*>(smem_raw) + (size_t)warp * smem_row_elems;
     const __nv_bfloat16* p = a.P + (int64_t)i * a.ldp;
-    for (int j = threadIdx.x * 8; j < a.r; j += blockDim.x * 8) {
+    for (int j = lane * 8; j < a.r; j += 32 * 8) {
       if (j + 8 <= a.r) *reinterpret_cast<uint4*>(row + j) = *reinterpret_cast<const uint4*>(p + j);
       else for (int e = j; e < a.r; ++e) row[e] = p[e];
     }
-    __syncthreads();
+    __syncwarp();
     __nv_bfloat16* o = a.P_c + (int64_t)i * a.ldpc;
-    for (int c = threadIdx.x; c < kp; c += blockDim.x) o[c] = c < k ? row[a.idx[c]] : __float2bfloat16_rn(0.f);
+    for (int c = lane; c < kp; c += 32) o[c] = c < k ? row[a.idx[c]] : __float2bfloat16_rn(0.f);
   }
 }
 
@@ -107,39 +111,64 @@ struct ActiveScatter {
 };
 struct ActiveScatterGroup { ActiveScatter a[kActiveGroup]; int n; int accumulate; };
 
-// blockIdx.x < r: dQ row j = blockIdx.x (and dlog_alpha[j]); otherwise dP row i = blockIdx.x - r.
+// Row task t = blockIdx.x * 8 + warp: t < r is row t of dQ (and dlog_alpha[t]), otherwise row t - r of dP.
 template <typename TW>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(32 * kActiveWarps)
 active_scatter_kernel(const __grid_constant__ ActiveScatterGroup g) {
   pdl_wait();
   pdl_launch_dependents();
   const ActiveScatter& a = g.a[blockIdx.y];
   const int acc = g.accumulate;
-  if ((int)blockIdx.x < a.r) {
-    const int j = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = blockIdx.x * kActiveWarps + warp;
+  if (t < a.r) {
+    const int j = t;
     const int c = a.pos[j];
     if (a.dQ) {
       TW* o = reinterpret_cast<TW*>(a.dQ) + (int64_t)j * a.lddq;
-      if (c >= 0) {
-        const TW* s = reinterpret_cast<const TW*>(a.dQ_c) + (int64_t)c * a.lddqc;
-        for (int e = threadIdx.x; e < a.d_in; e += blockDim.x) o[e] = acc ? from_f32<TW>(to_f32<TW>(o[e]) + to_f32<TW>(s[e])) : s[e];
+      constexpr int V = 16 / (int)sizeof(TW);
+      const TW* s = c >= 0 ? reinterpret_cast<const TW*>(a.dQ_c) + (int64_t)c * a.lddqc : nullptr;
+      const bool vec = !acc && ((reinterpret_cast<uintptr_t>(o) | reinterpret_cast<uintptr_t>(s)) & 15) == 0;
+      if (vec) {       // plain copy or zero fill, 16 bytes per lane
+        for (int e = lane * V; e < a.d_in; e += 32 * V) {
+          if (e + V <= a.d_in) *reinterpret_cast<uint4*>(o + e) = s ? *reinterpret_cast<const uint4*>(s + e) : make_uint4(0, 0, 0, 0);
+          else for (int x = e; x < a.d_in; ++x) o[x] = s ? s[x] : from_f32<TW>(0.f);
+        }
+      } else if (c >= 0) {
+        for (int e = lane; e < a.d_in; e += 32) o[e] = acc ? from_f32<TW>(to_f32<TW>(o[e]) + to_f32<TW>(s[e])) : s[e];
       } else if (!acc) {
-        for (int e = threadIdx.x; e < a.d_in; e += blockDim.x) o[e] = from_f32<TW>(0.f);
+        for (int e = lane; e < a.d_in; e += 32) o[e] = from_f32<TW>(0.f);
       }
     }
-    if (a.dla && threadIdx.x == 0) {
+    if (a.dla && lane == 0) {
       const float v = c >= 0 ? a.dla_c[c] : 0.f;
       a.dla[j] = acc ? a.dla[j] + v : v;
     }
   } else {
-    const int i = (int)blockIdx.x - a.r;
+    const int i = t - a.r;
     if (i >= a.d_out || !a.dP) return;
     TW* o = reinterpret_cast<TW*>(a.dP) + (int64_t)i * a.lddp;
     const TW* s = reinterpret_cast<const TW*>(a.dP_c) + (int64_t)i * a.lddpc;
-    for (int j = threadIdx.x; j < a.r; j += blockDim.x) {      // coalesced row write; the read of dP_c is a gather
-      const int c = a.pos[j];
-      const float v = c >= 0 ? to_f32<TW>(s[c]) : 0.f;
-      o[j] = acc ? from_f32<TW>(to_f32<TW>(o[j]) + v) : from_f32<TW>(v);
+    // coalesced row write, 16 bytes per lane; the read of dP_c is a gather within one (cached) row
+    constexpr int V = 16 / (int)sizeof(TW);
+    const bool vec = !acc && (reinterpret_cast<uintptr_t>(o) & 15) == 0;
+    for (int j0 = lane * V; j0 < a.r; j0 += 32 * V) {
+      if (vec && j0 + V <= a.r) {
+        uint4 raw;
+        TW* e = reinterpret_cast<TW*>(&raw);
+#pragma unroll
+        for (int x = 0; x < V; ++x) {
+          const int c = __ldg(a.pos + j0 + x);
+          e[x] = c >= 0 ? s[c] : from_f32<TW>(0.f);
+        }
+        *reinterpret_cast<uint4*>(o + j0) = raw;
+      } else {
+        for (int j = j0; j < min(j0 + V, a.r); ++j) {
+          const int c = a.pos[j];
+          const float v = c >= 0 ? to_f32<TW>(s[c]) : 0.f;
+          o[j] = acc ? from_f32<TW>(to_f32<TW>(o[j]) + v) : from_f32<TW>(v);
+        }
+      }
     }
   }
 }

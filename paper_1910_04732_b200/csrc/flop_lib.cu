@@ -1099,7 +1099,7 @@ int flop_active_ranks_gather(const flop_active_gather_t* pr, int n, int dt, void
           a.ldpc < a.r || a.ldqc < a.d_in || (a.dz_dla_c && !a.dz_dla))
         return FLOP_ERR_INVALID_ARG;
       if (!bf16_ok(a.P, a.ldp) || !bf16_ok(a.Q, a.ldq) || !bf16_ok(a.P_c, a.ldpc) || !bf16_ok(a.Q_c, a.ldqc)) return FLOP_ERR_UNSUPPORTED;
-      if ((size_t)a.r * 2 > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
+      if ((size_t)a.r * 2 * kActiveWarps > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
       ActiveGather& o = g.a[g.n];
       o.z = a.z; o.dz_dla = a.dz_dla; o.P = (const bf16*)a.P; o.ldp = a.ldp; o.Q = (const bf16*)a.Q; o.ldq = a.ldq;
       o.r = (int)a.r; o.d_in = (int)a.d_in; o.d_out = (int)a.d_out; o.idx = a.idx; o.pos = a.pos; o.k_dev = a.k_dev;
@@ -1108,9 +1108,10 @@ int flop_active_ranks_gather(const flop_active_gather_t* pr, int n, int dt, void
       max_r = std::max(max_r, o.r);
     }
     launch_k(active_select_kernel, dim3(g.n), dim3(1024), (size_t)0, st, g);
-    const size_t smem = (size_t)max_r * 2;
+    const int row_elems = (max_r + 7) & ~7;   // per-warp staging row, 16-byte aligned
+    const size_t smem = (size_t)row_elems * 2 * kActiveWarps;
     if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(active_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    launch_k(active_gather_kernel, dim3(max_blocks, g.n), dim3(256), smem, st, g);
+    launch_k(active_gather_kernel, dim3((max_blocks + kActiveWarps - 1) / kActiveWarps, g.n), dim3(32 * kActiveWarps), smem, st, g, row_elems);
     count_launch(2);
     FLOP_CUDA(cudaGetLastError());
   }
@@ -1139,8 +1140,8 @@ int flop_active_ranks_scatter(const flop_active_scatter_t* pr, int n, int accumu
       o.dP = a.dP; o.lddp = a.lddp; o.dQ = a.dQ; o.lddq = a.lddq; o.dla = a.dlog_alpha;
       max_blocks = std::max(max_blocks, o.r + o.d_out);
     }
-    if (wgrad_dt == FLOP_BF16) launch_k(active_scatter_kernel<bf16>, dim3(max_blocks, g.n), dim3(256), (size_t)0, st, g);
-    else                       launch_k(active_scatter_kernel<float>, dim3(max_blocks, g.n), dim3(256), (size_t)0, st, g);
+    if (wgrad_dt == FLOP_BF16) launch_k(active_scatter_kernel<bf16>, dim3((max_blocks + kActiveWarps - 1) / kActiveWarps, g.n), dim3(32 * kActiveWarps), (size_t)0, st, g);
+    else                       launch_k(active_scatter_kernel<float>, dim3((max_blocks + kActiveWarps - 1) / kActiveWarps, g.n), dim3(32 * kActiveWarps), (size_t)0, st, g);
     count_launch();
     FLOP_CUDA(cudaGetLastError());
   }

@@ -10,6 +10,8 @@ bytes of each call (what must be read and written once), time is the mean of CUD
 event timings after warm-up.  The second table is the inference configuration:
 compaction once, then the compact forward against the uncompacted gated forward
 (both replayed from CUDA graphs so that host launch cost does not hide the kernels).
+The third table is one training step of a BERT-shaped layer on the active rank
+components only, against the dense gated step, for several fractions of open gates.
 """
 from __future__ import annotations
 
@@ -133,7 +135,61 @@ def main():
         flops = 2.0 * T * k * (mtx.d_in + mtx.d_out)
         wbytes = 2.0 * k * (mtx.d_in + mtx.d_out)
         print(f"{T:6d} {tc_ * 1e6:15.1f} {tg_ * 1e6:13.1f} {tg_ / tc_:9.2f} {flops / tc_ / 1e9:16.0f} {wbytes / tc_ / 1e9:12.0f}")
+    # ---- training on the active rank components: one BERT-shaped layer (six matrices, T = 4096)
+    for wl in ("bert", "sru"):
+        active_table(I.WORKLOADS[wl], g)
     assert b.device_status() == b.OK
+
+
+def active_table(w, g):
+    bf = torch.bfloat16
+    T = w.T
+    es = []
+    for mtx in w.matrices:
+        e = dict(m=mtx)
+        rn = lambda rows, cols, sc=1.0: (torch.randn(rows, cols, generator=g, device="cuda") * sc).to(bf)
+        e["X"], e["dY"] = rn(T, mtx.d_in), rn(T, mtx.d_out)
+        e["Q"], e["P"] = rn(mtx.r, mtx.d_in, mtx.d_in ** -0.5), rn(mtx.d_out, mtx.r, mtx.r ** -0.5)
+        e["z"], e["dzd"] = torch.zeros(mtx.r, device="cuda"), torch.ones(mtx.r, device="cuda")
+        for name, rows, cols in (("H", T, mtx.r), ("Y", T, mtx.d_out), ("dX", T, mtx.d_in), ("dP", mtx.d_out, mtx.r),
+                                 ("dQ", mtx.r, mtx.d_in), ("Pc", mtx.d_out, mtx.r), ("Qc", mtx.r, mtx.d_in),
+                                 ("dPc", mtx.d_out, mtx.r), ("dQc", mtx.r, mtx.d_in)):
+            e[name] = b.padded(rows, cols, bf)
+        for name in ("dla", "zc", "dzc", "dlac"):
+            e[name] = torch.zeros(mtx.r, device="cuda")
+        e["idx"], e["pos"] = (torch.zeros(mtx.r, dtype=torch.int32, device="cuda") for _ in range(2))
+        e["k"] = torch.zeros(1, dtype=torch.int32, device="cuda")
+        e["ws"] = b.alloc_workspace(b.workspace_bytes(b.OP_BWD, T, mtx.d_in, mtx.d_out, mtx.r, b.BF16))
+        es.append(e)
+    fwd_d = b.problem_array([b.fwd_problem(e["X"], e["Q"], e["P"], e["z"], e["Y"], e["H"]) for e in es])
+    bwd_d = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], e["z"], e["dzd"], e["H"], e["dX"], e["dP"], e["dQ"],
+                                           e["dla"], e["ws"]) for e in es])
+    gat = b.problem_array([b.active_gather_problem(e["z"], e["dzd"], e["P"], e["Q"], e["idx"], e["pos"], e["k"], e["zc"], e["dzc"],
+                                                   e["Pc"], e["Qc"]) for e in es])
+    fwd_a = b.problem_array([b.fwd_problem(e["X"], e["Qc"], e["Pc"], e["zc"], e["Y"], e["H"], r_dev=e["k"]) for e in es])
+    bwd_a = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Qc"], e["Pc"], e["zc"], e["dzc"], e["H"], e["dX"], e["dPc"], e["dQc"],
+                                           e["dlac"], e["ws"], r_dev=e["k"]) for e in es])
+    sca = b.problem_array([b.active_scatter_problem(e["idx"], e["pos"], e["k"], e["m"].d_in, e["m"].d_out, e["m"].r, e["dPc"],
+                                                    e["dQc"], e["dlac"], e["dP"], e["dQ"], e["dla"]) for e in es])
+
+    def dense():
+        b.gated_lowrank_fwd_grouped(fwd_d)
+        b.gated_lowrank_bwd_grouped(bwd_d)
+
+    def active_step():
+        b.active_ranks_gather(gat)
+        b.gated_lowrank_fwd_grouped(fwd_a)
+        b.gated_lowrank_bwd_grouped(bwd_a)
+        b.active_ranks_scatter(sca)
+
+    print(f"\ntraining on the active rank components, one {w.name}-shaped layer ({len(es)} matrices, T={T}), graph replay")
+    print(f"{'open gates':>11s} {'dense us':>9s} {'active us':>10s} {'speed-up':>9s}   (active = select + gather + fwd + bwd + scatter)")
+    for frac in (1.0, 0.6, 0.3, 0.15, 0.05):
+        for e in es:
+            e["z"].copy_((torch.rand(e["m"].r, generator=g, device="cuda") < frac).float() * 0.7)
+        td = timed(dense, iters=20, graph=True)
+        ta = timed(active_step, iters=20, graph=True)
+        print(f"{frac:11.2f} {td * 1e6:9.1f} {ta * 1e6:10.1f} {td / ta:9.2f}")
 
 
 if __name__ == "__main__":
