@@ -75,6 +75,11 @@ int flop_device_status(void* stream);
  * stream; _end waits for them and returns the summed kernel time (ms), the summed
  * algorithmic flops 2 M N K of those launches and their number (HOST out pointers,
  * nullable).  Not thread-safe with respect to concurrent launches. */
+/* Self-test of the bounded device-side wait (no counterpart in the paper): launches one thread that waits
+ * on a barrier nothing will ever signal, for at most limit_cycles SM cycles (<= 2e9), then records
+ * FLOP_ERR_TIMEOUT in the device status word and writes 1 to *gave_up_dev (DEVICE int).  The context stays
+ * usable; flop_device_status() returns and clears the code. */
+int flop_selftest_wait_timeout(int64_t limit_cycles, int* gave_up_dev, void* stream);
 unsigned long long flop_launch_count(void);
 int flop_gemm_timing_begin(void);
 int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launches);

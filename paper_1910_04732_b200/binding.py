@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 
-EXPORTS = ("flop_status_string", "flop_device_status", "flop_launch_count", "flop_gemm_timing_begin",
+EXPORTS = ("flop_status_string", "flop_device_status", "flop_selftest_wait_timeout", "flop_launch_count", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
@@ -92,6 +92,7 @@ def load_library() -> ctypes.CDLL:
     lib.flop_device_status.argtypes = [vp]
     lib.flop_workspace_bytes.argtypes = [ci, i64, i64, i64, i64, ci, ctypes.POINTER(sz)]
     lib.flop_launch_count.argtypes = []
+    lib.flop_selftest_wait_timeout.argtypes = [i64, vp, vp]
     lib.flop_gemm_timing_begin.argtypes = []
     lib.flop_gemm_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                          ctypes.POINTER(ctypes.c_int64)]
@@ -164,6 +165,12 @@ def workspace_bytes(op: int, T: int, d_in: int, d_out: int, r: int, dt: int) -> 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
     """A 256-byte aligned scratch buffer (torch's caching allocator aligns to 512)."""
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def selftest_wait_timeout(limit_cycles: int, gave_up: torch.Tensor) -> None:
+    """Launch the bounded-wait self-test: a wait that can never complete must give up after limit_cycles."""
+    _check(load_library().flop_selftest_wait_timeout(int(limit_cycles), _ptr(gave_up), _stream()),
+           "flop_selftest_wait_timeout")
 
 
 def launch_count() -> int:

@@ -591,6 +591,14 @@ int flop_device_status(void* stream) {
   return v;
 }
 
+int flop_selftest_wait_timeout(int64_t limit_cycles, int* gave_up_dev, void* stream) {
+  if (limit_cycles <= 0 || limit_cycles > 2000000000LL || !gave_up_dev) return FLOP_ERR_INVALID_ARG;
+  launch_k(tc::wait_selftest_kernel, dim3(1), dim3(32), (size_t)0, (cudaStream_t)stream, (long long)limit_cycles, gave_up_dev);
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
 unsigned long long flop_launch_count(void) { return g_launches; }
 
 int flop_gemm_timing_begin(void) {

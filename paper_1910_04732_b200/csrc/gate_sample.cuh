@@ -31,7 +31,7 @@ struct GateConsts {
   double beta_d, gamma_d, zeta_d;        // exact images of the fp32 parameters
 };
 
-constexpr float kBand = 1e-4f;  // |t - c| below this -> fp64; fp32 error of t is < 5e-6
+constexpr float kBand = 2.5e-5f;  // |t - c| below this -> fp64; fp32 error of t is < 5.3e-6 (see gate_one)
 
 __device__ __forceinline__ void gate_fp64(float alpha, float u, const GateConsts& g, float& z, int& m, float& d) {
   // The sampler exactly as printed, one rounded operation at a time.
@@ -49,7 +49,8 @@ __device__ __forceinline__ void gate_fp64(float alpha, float u, const GateConsts
 __device__ __forceinline__ void gate_one(float alpha, uint32_t bits, const GateConsts& g, float& z, int& m, float& d) {
   const float u = ((float)(bits >> 9) + 0.5f) * 1.1920928955078125e-7f;  // 2^-23; exact
   // logit(u) with the fast intrinsics: u / (1 - u) is within 2 ulp, __logf within 2 ulp of a value of
-  // magnitude <= 16.7, so t is off by < 5e-6, far inside the band that sends a gate to fp64
+  // magnitude <= 16.7 (4e-6), the sum with alpha rounds once more (1e-6): t is off by < 5.3e-6, a fifth
+  // of the band that sends a gate to fp64
   const float t = __logf(__fdividef(u, 1.0f - u)) + alpha;
   if (fabsf(t - g.c0) < kBand || fabsf(t - g.c1) < kBand || !(fabsf(t) < 1e30f)) {
     gate_fp64(alpha, u, g, z, m, d);

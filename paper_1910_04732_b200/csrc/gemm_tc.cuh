@@ -199,6 +199,31 @@ __device__ __forceinline__ WorkItem decode(const Params& p, int w) {
   return it;
 }
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on, with the
+// given cycle limit, and must come back with the timeout recorded (the status word is then read by
+// flop_device_status()).  Exercises the exact wait routine of the GEMM kernels without a GEMM.
+__global__ void wait_selftest_kernel(long long limit_cycles, int* gave_up) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int s_abort;
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const uint32_t b = smem_u32(&bar);
+    const long long t0 = clock64();
+    bool done = false;
+    while (!done) {                       // the body of mbar_wait with a caller-chosen limit
+      if (mbar_try_wait(b, 0)) break;
+      if (clock64() - t0 > limit_cycles) {
+        s_abort = 1;
+        report_timeout();
+        done = true;
+      }
+    }
+    *gave_up = s_abort;
+  }
+}
+
 // One 32-column chunk of one accumulator row (held by this thread) through the epilogue.
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32], int row, bool row_ok, int n0, int split,

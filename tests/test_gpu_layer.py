@@ -175,3 +175,16 @@ def test_degenerate_sizes(b):
         b.gated_lowrank_bwd(dY, X, Q, P, z, z, H, None, dP, dQ, dla, None)  # empty batch: zero gradients
         assert torch.count_nonzero(dP) == 0 and torch.count_nonzero(dQ) == 0 and torch.count_nonzero(dla) == 0
     assert b.device_status() == b.OK
+
+
+def test_bounded_wait_gives_up_and_reports_timeout(b):
+    """A device-side wait that nothing will ever satisfy: the kernel must return on its own, the status
+    word must say FLOP_ERR_TIMEOUT once, and the library must keep working afterwards."""
+    assert b.device_status() == b.OK
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.selftest_wait_timeout(2_000_000, flag)            # about a millisecond
+    assert b.device_status() == b.ERR_TIMEOUT
+    assert int(flag.item()) == 1
+    assert b.device_status() == b.OK                    # reading the status clears it
+    w = I.Workload("t", "bf16", 256, 1, (I.Matrix("w", 128, 128, 64),), ("normal", 0.5, 1.5), 0.5)
+    run_layer(b, I.layer_problem(w, 0, 0, seed=9), "bf16")
