@@ -697,7 +697,7 @@ static int gate_sample_impl(const float* log_alpha, int64_t n, flop_hc_params_t 
                      (!mask || (reinterpret_cast<uintptr_t>(mask) & 3) == 0);
   const int64_t nblk = (n + 3) / 4;
   const int64_t want = (nblk + 255) / 256;
-  const int grid = (int)std::min<int64_t>(want, (int64_t)num_sms() * 16);
+  const int grid = (int)std::min<int64_t>(want, (int64_t)num_sms() * 32);
   launch_k(gate_sample_kernel, dim3(grid), dim3(256), (size_t)(0), (cudaStream_t)stream, log_alpha, n, g, make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)),
                                                              offset, offset_dev, z, mask, dz_dla, vec_ok);
   count_launch();

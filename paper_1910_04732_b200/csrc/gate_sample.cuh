@@ -76,6 +76,7 @@ gate_sample_kernel(const float* __restrict__ log_alpha, int64_t n, GateConsts g,
   // the counter offset may also live in device memory, so that a captured launch can advance it
   const uint64_t offset = offset_host + (offset_dev ? *offset_dev : 0ull);
   const int64_t nblk = (n + 3) >> 2;
+#pragma unroll 2
   for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblk; b += (int64_t)gridDim.x * blockDim.x) {
     const uint64_t ctr = offset + (uint64_t)b;
     const uint4 x = philox4x32_10(make_uint4((uint32_t)ctr, (uint32_t)(ctr >> 32), 0u, 0u), key);
@@ -84,13 +85,13 @@ gate_sample_kernel(const float* __restrict__ log_alpha, int64_t n, GateConsts g,
     float zz[4], dd[4];
     int mm[4];
     if (vec_ok && j0 + 4 <= n) {
-      const float4 a = *reinterpret_cast<const float4*>(log_alpha + j0);
+      const float4 a = __ldcs(reinterpret_cast<const float4*>(log_alpha + j0));   // streamed once: do not keep in cache
       const float aa[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) gate_one(aa[i], bits[i], g, zz[i], mm[i], dd[i]);
-      *reinterpret_cast<float4*>(z + j0) = make_float4(zz[0], zz[1], zz[2], zz[3]);
-      if (mask) *reinterpret_cast<uchar4*>(mask + j0) = make_uchar4(mm[0], mm[1], mm[2], mm[3]);
-      if (dz_dla) *reinterpret_cast<float4*>(dz_dla + j0) = make_float4(dd[0], dd[1], dd[2], dd[3]);
+      __stcs(reinterpret_cast<float4*>(z + j0), make_float4(zz[0], zz[1], zz[2], zz[3]));
+      if (mask) __stcs(reinterpret_cast<uchar4*>(mask + j0), make_uchar4(mm[0], mm[1], mm[2], mm[3]));
+      if (dz_dla) __stcs(reinterpret_cast<float4*>(dz_dla + j0), make_float4(dd[0], dd[1], dd[2], dd[3]));
     } else {
       for (int i = 0; i < 4 && j0 + i < n; ++i) {
         gate_one(log_alpha[j0 + i], bits[i], g, zz[i], mm[i], dd[i]);

@@ -101,7 +101,7 @@ l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__
     float a[4];
     const bool full = j0 + 4 <= hi;
     if (full && al_a) {
-      const float4 t = *reinterpret_cast<const float4*>(log_alpha + j0);
+      const float4 t = __ldcs(reinterpret_cast<const float4*>(log_alpha + j0));
       a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
     } else {
 #pragma unroll
