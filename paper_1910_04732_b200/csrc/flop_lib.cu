@@ -26,6 +26,7 @@
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
 #include "active_ranks.cuh"
+#include "gemm_small_t.cuh"
 
 using namespace flop;
 typedef __nv_bfloat16 bf16;
@@ -434,6 +435,40 @@ bool wgrad_direct_ok(const void* out, int64_t ldo, int wgrad_dt) {
   return aligned16(out) && (ldo % (wgrad_dt == FLOP_F32 ? 4 : 8)) == 0;
 }
 
+// Few-token forward product C = (A B^T) * col_scale on the CUDA cores (see gemm_small_t.cuh).
+// Returns FLOP_ERR_UNSUPPORTED when the shape does not fit (the caller then uses the tensor-core path).
+template <int TT>
+int launch_small_t_inst(const bf16* A, int64_t lda, const bf16* B, int64_t ldb, bf16* C, int64_t ldc, const float* cs, int T,
+                        int N, int K, int k_pad, size_t smem, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    FLOP_CUDA(cudaFuncSetAttribute(small_t_gemm_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    configured = true;
+  }
+  const int grid = std::min((N + kSmallTWarps - 1) / kSmallTWarps, num_sms() * 4);
+  launch_k(small_t_gemm_kernel<TT>, dim3(grid), dim3(32 * kSmallTWarps), smem, st, A, lda, B, ldb, C, ldc, cs, T, N, K, k_pad);
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+int launch_small_t(const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc, const float* cs, int64_t T,
+                   int64_t N, int64_t K, cudaStream_t st) {
+  static const int off = env_int("FLOP_NO_SMALL_T");
+  if (off || T < 1 || T > kSmallTMax || N > INT32_MAX || K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  int tt = 1;
+  while (tt < T) tt *= 2;
+  const int k_pad = (int)round_up(K, 256);                 // every lane's 8-element step stays inside the row
+  const size_t smem = (size_t)tt * k_pad * 2;
+  if (smem > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
+  const bf16* a = (const bf16*)A; const bf16* b = (const bf16*)B; bf16* c = (bf16*)C;
+  switch (tt) {
+    case 1: return launch_small_t_inst<1>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
+    case 2: return launch_small_t_inst<2>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
+    case 4: return launch_small_t_inst<4>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
+    default: return launch_small_t_inst<8>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
+  }
+}
+
 int launch_simt(const float* A, int64_t a_sm, int64_t a_sk, const float* B, int64_t b_sn, int64_t b_sk, float* C,
                 int64_t ldc, int64_t M, int64_t N, int64_t K, const float* col_scale, const float* row_scale,
                 int accumulate, cudaStream_t st) {
@@ -725,6 +760,15 @@ static int fwd_impl(const void* X, int64_t ldx, const void* Q, int64_t ldq, cons
       if (r > 0) FLOP_TRY(zero_2d<bf16>(H, ldh, T, r, st));
       return FLOP_OK;
     }
+    if (T <= kSmallTMax) {   // a handful of tokens: stream the weights once on the CUDA cores
+      const int rc = launch_small_t(X, ldx, Q, ldq, H, ldh, z, T, r, d_in, st);
+      if (rc == FLOP_OK) {
+        const int rc2 = launch_small_t(H, ldh, P, ldp, Y, ldy, nullptr, T, d_out, r, st);
+        if (rc2 != FLOP_ERR_UNSUPPORTED) return rc2;
+      } else if (rc != FLOP_ERR_UNSUPPORTED) {
+        return rc;
+      }
+    }
     // GEMM1: H' = (X Q^T) * z, gate applied to column k in the epilogue
     const TcPlan p1 = plan_tc(T, r, d_in, false, false);
     FLOP_TRY(launch_tc({X, ldx, false}, {Q, ldq, false}, T, r, d_in, p1, store_epilogue(H, ldh, z), st));
@@ -782,6 +826,15 @@ int flop_compact_fwd(const void* X, int64_t ldx, const void* Qc, int64_t ldqc, c
   const FwdWs w = plan_fwd_ws(ar, T, k, dt);
   if (dt == FLOP_BF16) {
     if (!bf16_ok(Y, ldy) || !bf16_ok(X, ldx) || !bf16_ok(Qc, ldqc) || !bf16_ok(Pc, ldpc)) return FLOP_ERR_UNSUPPORTED;
+    if (T <= kSmallTMax) {
+      const int rc = launch_small_t(X, ldx, Qc, ldqc, w.H, w.ldh, nullptr, T, k, d_in, st);
+      if (rc == FLOP_OK) {
+        const int rc2 = launch_small_t(w.H, w.ldh, Pc, ldpc, Y, ldy, nullptr, T, d_out, k, st);
+        if (rc2 != FLOP_ERR_UNSUPPORTED) return rc2;
+      } else if (rc != FLOP_ERR_UNSUPPORTED) {
+        return rc;
+      }
+    }
     const TcPlan p1 = plan_tc(T, k, d_in, false, false);
     FLOP_TRY(launch_tc({X, ldx, false}, {Qc, ldqc, false}, T, k, d_in, p1, store_epilogue(w.H, w.ldh, nullptr), st));
     const TcPlan p2 = plan_tc(T, d_out, k, false, false);
