@@ -516,7 +516,7 @@ def main():
     tflops = w.flops_per_step() * world / (step_ms / 1e3) / 1e12
     gemm_tflops = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     # dram__bytes_read.sum + dram__bytes_write.sum of the GEMM launches of one bert layer, from the ncu capture
-    # summarised in profiles/gemm_group_kernel_bert_ncu_full.md (grouped calls of six matrices): mean per launch
+    # summarised under profiles/ (grouped calls of six matrices): mean per launch
     traffic = 102.8e6 if (w.name == "bert" and group == 6) else None
     line = {
         "metric": METRIC, "value": tokens_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
