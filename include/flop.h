@@ -84,6 +84,15 @@ unsigned long long flop_launch_count(void);
 int flop_gemm_timing_begin(void);
 int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launches);
 
+/* Device-side stamps (no counterpart in the paper): between _begin and _end, GEMM launch i is
+ * issued with a pointer to stamps_dev[2i..2i+1] (DEVICE, zero-initialised by the caller) and writes
+ * there the %globaltimer (ns) at which its first CTA passed the dependency wait and the latest
+ * time at which one of its CTAs finished.  The pointers stay in the launches, so a CUDA graph
+ * captured in between refreshes the stamps at every replay; this times kernels where host events
+ * cannot be placed.  _end returns the number of stamped launches and the sum of their 2 M N K. */
+int flop_gemm_stamps_begin(unsigned long long* stamps_dev, int capacity);
+int flop_gemm_stamps_end(int* launches, double* total_flops);
+
 /* Bytes of scratch the given call needs (HOST out pointer).  For FLOP_OP_L0
  * pass the total number of gates as T and the number of segments as r. */
 int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt,

@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
 
 EXPORTS = ("flop_status_string", "flop_device_status", "flop_selftest_wait_timeout", "flop_launch_count", "flop_gemm_timing_begin",
-           "flop_gemm_timing_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
+           "flop_gemm_timing_end", "flop_gemm_stamps_begin", "flop_gemm_stamps_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
            "flop_expected_l0_lagrangian",
@@ -98,6 +98,8 @@ def load_library() -> ctypes.CDLL:
                                          ctypes.POINTER(ctypes.c_int64)]
     lib.flop_tc_gemm.argtypes = [vp, i64, ci, vp, i64, ci, vp, i64, vp, vp, i64, i64, i64, ci, ci, ci,
                                  ctypes.POINTER(ctypes.c_int), vp]
+    lib.flop_gemm_stamps_begin.argtypes = [vp, ci]
+    lib.flop_gemm_stamps_end.argtypes = [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double)]
     lib.flop_gate_sample.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
     lib.flop_gate_sample_devoff.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp, vp]
     lib.flop_gated_lowrank_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
@@ -187,6 +189,19 @@ def gemm_timing_end():
     _check(load_library().flop_gemm_timing_end(ctypes.byref(ms), ctypes.byref(fl), ctypes.byref(n)),
            "flop_gemm_timing_end")
     return ms.value, fl.value, int(n.value)
+
+
+def gemm_stamps_begin(stamps: torch.Tensor) -> None:
+    """stamps: zeroed int64 device tensor of 2 * capacity elements (start, end ns per GEMM launch)."""
+    assert stamps.element_size() == 8
+    _check(load_library().flop_gemm_stamps_begin(_ptr(stamps), stamps.numel() // 2), "flop_gemm_stamps_begin")
+
+
+def gemm_stamps_end():
+    """(stamped launches, sum of their algorithmic flops)."""
+    n, fl = ctypes.c_int(0), ctypes.c_double(0)
+    _check(load_library().flop_gemm_stamps_end(ctypes.byref(n), ctypes.byref(fl)), "flop_gemm_stamps_end")
+    return int(n.value), fl.value
 
 
 def device_status() -> int:

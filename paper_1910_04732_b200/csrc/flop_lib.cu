@@ -110,6 +110,14 @@ std::mutex g_timing_mu;
 
 inline void count_launch(int n = 1) { g_launches += (unsigned long long)n; }
 
+// Device-side stamps (flop_gemm_stamps_begin/end): while on, GEMM launch i writes its start and end
+// %globaltimer to stamps[2i], stamps[2i+1] of a caller-provided device buffer.
+struct GemmStamps {
+  unsigned long long* buf = nullptr;
+  int capacity = 0, used = 0;
+  double flops = 0.0;
+} g_stamps;
+
 struct GemmTimer {
   cudaStream_t st;
   bool active;
@@ -357,6 +365,11 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     const int cta2 = first.pl.cta2;
     gp.stages = std::min(tc::kMaxStages, (kSmemBudget - kSmemFixed) /
                                              (int)(cta2 ? tc::stage_bytes2(gp.bn_max) : tc::stage_bytes(gp.bn_max)));
+    gp.stamp = nullptr;
+    if (g_stamps.buf && g_stamps.used < g_stamps.capacity) {
+      gp.stamp = g_stamps.buf + 2 * g_stamps.used++;
+      g_stamps.flops += flops;
+    }
     const bool a_mn = first.A.mn_major, b_mn = first.B.mn_major;
     int rc = FLOP_ERR_UNSUPPORTED;
     if (!a_mn && !b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, false, tc::EPI_STORE>(gp, cta2, flops, st);
@@ -635,6 +648,19 @@ int flop_selftest_wait_timeout(int64_t limit_cycles, int* gave_up_dev, void* str
 }
 
 unsigned long long flop_launch_count(void) { return g_launches; }
+
+int flop_gemm_stamps_begin(unsigned long long* stamps_dev, int capacity) {
+  if (!stamps_dev || capacity <= 0) return FLOP_ERR_INVALID_ARG;
+  g_stamps.buf = stamps_dev; g_stamps.capacity = capacity; g_stamps.used = 0; g_stamps.flops = 0.0;
+  return FLOP_OK;
+}
+
+int flop_gemm_stamps_end(int* launches, double* total_flops) {
+  if (launches) *launches = g_stamps.used;
+  if (total_flops) *total_flops = g_stamps.flops;
+  g_stamps.buf = nullptr; g_stamps.capacity = 0;
+  return FLOP_OK;
+}
 
 int flop_gemm_timing_begin(void) {
   std::lock_guard<std::mutex> lk(g_timing_mu);

@@ -54,6 +54,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
   volatile int* abort_flag = &s_abort;
   pdl_wait();
   pdl_launch_dependents();
+  if (gp.stamp && blockIdx.x == 0 && threadIdx.x == 0) gp.stamp[0] = global_ns();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -166,6 +167,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
     tcgen05_fence_after();
     tmem_dealloc2(tmem_base, kTmemCols);
   }
+  if (gp.stamp && threadIdx.x == 0) atomicMax(gp.stamp + 1, global_ns());
 }
 
 }  // namespace tc

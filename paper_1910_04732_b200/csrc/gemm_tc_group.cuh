@@ -34,7 +34,17 @@ struct GroupParams {
   int total_work;   // sum over problems of tiles_m * tiles_n * splits
   int stages;
   int bn_max;       // largest N tile: sizes the stages and the accumulator buffers
+  // Optional device-side stamp of this launch (nullable): [0] = %globaltimer when CTA 0 passes the
+  // dependency wait, [1] = the latest %globaltimer at which a CTA finished (atomic max).  Lets a
+  // caller time launches that run inside a replayed CUDA graph, where host events cannot be placed.
+  unsigned long long* stamp;
 };
+
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 
 struct GroupItem { int g, tm, tn, split, kb0, kb1, n_limit; bool active; };
 
@@ -97,6 +107,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
   volatile int* abort_flag = &s_abort;
   pdl_wait();
   pdl_launch_dependents();
+  if (gp.stamp && blockIdx.x == 0 && threadIdx.x == 0) gp.stamp[0] = global_ns();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -202,6 +213,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
     tcgen05_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
+  if (gp.stamp && threadIdx.x == 0) atomicMax(gp.stamp + 1, global_ns());
 }
 
 }  // namespace tc
