@@ -275,6 +275,17 @@ int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const
                                         const float* target, const float* lambda, float* out4,
                                         float* seg_expected, float* dlog_alpha, void* stream);
 
+/* FLOP-AGP variant (Section 5, baselines): magnitude-based pruning of the learnable diagonal mask
+ * G = diag(g) instead of hard-concrete gates.  Segment i (one weight matrix) owns
+ * g[seg_off[i]..seg_off[i+1]): its round(sparsity * r_i) entries of smallest |g| are pruned (ties at the
+ * cut keep the lower indices); z = g on kept entries and 0 elsewhere, mask = [kept] (nullable),
+ * dz_dg = [kept] (nullable), seg_l1[i] = sum |g| over the segment (nullable; the L1 term on the masks
+ * is l1 times their sum), dg (nullable) += l1 * sign(g).  sparsity[1] is a DEVICE scalar so that a
+ * schedule can advance it on the device.  The forward/backward calls then take z and dz_dg where they
+ * take the sampled gate and dz_dla; the dlog_alpha they return is the gradient with respect to g. */
+int flop_agp_gates(const float* g, int64_t n, const int64_t* seg_off, int32_t n_seg, const float* sparsity,
+                   float l1, float* z, uint8_t* mask, float* dz_dg, float* seg_l1, float* dg, void* stream);
+
 /* Deterministic gates and compaction of one weight matrix (Sections 4.4, 4.1).
  * mode 0: log_alpha_or_z holds log_alpha; k = floor(sum_j pi_j + 1/2); the k
  *         gates with the largest log_alpha are kept (ties: lower index) with

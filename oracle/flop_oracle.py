@@ -33,6 +33,8 @@ other than itself:
                           equal sizes -> mean), finite differences.
     deterministic_mask / compact_ranks / compact_fwd
                           brute-force masking of the uncompacted layer.
+    agp_gates             brute-force properties of the magnitude rule (counts, kept >= pruned,
+                          tie order), finite differences of the L1 term.
     The *choices* the paper leaves open (values of kept inference gates,
     top-k tie-break, which factor absorbs the gate) are "parity unpinned":
     several answers satisfy the paper, the oracle fixes one.
@@ -283,3 +285,34 @@ def compact_fwd(X, Qc, Pc):
     """Inference forward on the compact factors: Y = (X Q_c^T) P_c^T (Section 4.1)."""
     X = np.asarray(X, dtype=np.float64)
     return (X @ np.asarray(Qc, dtype=np.float64).T) @ np.asarray(Pc, dtype=np.float64).T
+
+
+# ----------------------------------------------------------------------------
+# FLOP-AGP variant (Section 5, baselines): magnitude pruning of the diagonal mask
+# ----------------------------------------------------------------------------
+def agp_gates(g, seg_off, sparsity, l1):
+    """Magnitude-based pruning of the learnable diagonal G = diag(g) of every matrix.
+
+    Per segment (weight matrix) with r_i components, the round(sparsity * r_i)
+    entries of smallest |g_k| are pruned (ties: the higher index goes first), the
+    others keep their value:  z_k = g_k if kept else 0,  dz_k/dg_k = [kept].
+    The L1 term on the masks is l1 * sum_k |g_k| with gradient l1 * sign(g_k)
+    (the paper: "l1 regularization on the masks to encourage sparsity").
+    Returns dict(z, mask, dz_dg, seg_l1 (sum |g| per segment), l1_grad).
+    """
+    g = np.asarray(g, dtype=np.float64)
+    seg_off = np.asarray(seg_off, dtype=np.int64)
+    z = np.zeros_like(g)
+    mask = np.zeros(len(g), dtype=np.uint8)
+    seg_l1 = np.zeros(len(seg_off) - 1)
+    for i in range(len(seg_off) - 1):
+        lo, hi = int(seg_off[i]), int(seg_off[i + 1])
+        r = hi - lo
+        n_pruned = int(np.floor(float(sparsity) * r + 0.5))
+        keep = max(0, min(r, r - n_pruned))
+        order = sorted(range(r), key=lambda k: (-abs(g[lo + k]), k))     # largest magnitude first, then lower index
+        for k in order[:keep]:
+            mask[lo + k] = 1
+            z[lo + k] = g[lo + k]
+        seg_l1[i] = np.sum(np.abs(g[lo:hi]))
+    return dict(z=z, mask=mask, dz_dg=mask.astype(np.float64), seg_l1=seg_l1, l1_grad=float(l1) * np.sign(g))

@@ -25,7 +25,7 @@ EXPORTS = ("flop_status_string", "flop_device_status", "flop_selftest_wait_timeo
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
            "flop_expected_l0_lagrangian",
-           "flop_expected_l0_lagrangian_noalloc",
+           "flop_expected_l0_lagrangian_noalloc", "flop_agp_gates",
            "flop_compact_ranks", "flop_compact_fwd")
 
 
@@ -114,6 +114,7 @@ def load_library() -> ctypes.CDLL:
     lib.flop_expected_l0_lagrangian.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp,
                                                 vp, sz, vp]
     lib.flop_expected_l0_lagrangian_noalloc.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp, vp]
+    lib.flop_agp_gates.argtypes = [vp, i64, vp, ctypes.c_int32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp]
     lib.flop_compact_ranks.argtypes = [vp, ci, HcParams, i64, vp, i64, vp, i64, i64, i64, ci,
                                        vp, vp, vp, vp, i64, vp, i64, vp, sz, vp]
     lib.flop_compact_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, i64, i64, i64, i64, ci, vp, sz, vp]
@@ -341,6 +342,13 @@ def expected_l0_lagrangian_noalloc(log_alpha, seg_off, seg_size, hc, target, lam
         _ptr(log_alpha), log_alpha.numel(), _ptr(seg_off), _ptr(seg_size), seg_size.numel(), _hc(hc),
         _ptr(target), _ptr(lam), _ptr(out4), _ptr(seg_expected), _ptr(dlog_alpha), _stream()),
         "flop_expected_l0_lagrangian_noalloc")
+
+
+def agp_gates(g, seg_off, sparsity, l1: float, z, mask=None, dz_dg=None, seg_l1=None, dg=None) -> None:
+    """flop_agp_gates: magnitude pruning of the diagonal mask per segment (sparsity: 1-element device tensor)."""
+    _check(load_library().flop_agp_gates(_ptr(g), g.numel(), _ptr(seg_off), seg_off.numel() - 1, _ptr(sparsity), float(l1),
+                                         _ptr(z), _ptr(mask), _ptr(dz_dg), _ptr(seg_l1), _ptr(dg), _stream()),
+           "flop_agp_gates")
 
 
 def compact_ranks(log_alpha_or_z, mode: int, hc, idx, k_dev, z_det=None, P=None, Q=None, Pc=None, Qc=None) -> None:

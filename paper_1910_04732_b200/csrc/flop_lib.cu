@@ -27,6 +27,7 @@
 #include "wgrad.cuh"
 #include "active_ranks.cuh"
 #include "gemm_small_t.cuh"
+#include "agp.cuh"
 
 using namespace flop;
 typedef __nv_bfloat16 bf16;
@@ -1295,6 +1296,18 @@ int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const
     launch_k(l0_chunk_kernel<true>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
     count_launch();
   }
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+int flop_agp_gates(const float* g, int64_t n, const int64_t* seg_off, int32_t n_seg, const float* sparsity, float l1,
+                   float* z, uint8_t* mask, float* dz_dg, float* seg_l1, float* dg, void* stream) {
+  if (n < 0 || n_seg < 0 || !sparsity) return FLOP_ERR_INVALID_ARG;
+  if (n_seg == 0 || n == 0) return FLOP_OK;
+  if (!g || !seg_off || !z) return FLOP_ERR_INVALID_ARG;
+  launch_k(agp_gates_kernel, dim3((unsigned)n_seg), dim3(kAgpThreads), (size_t)0, (cudaStream_t)stream, g, seg_off, sparsity, l1, z,
+           mask, dz_dg, seg_l1, dg);
+  count_launch();
   FLOP_CUDA(cudaGetLastError());
   return FLOP_OK;
 }
