@@ -60,7 +60,8 @@ typedef enum {
   FLOP_OP_BWD = 1,         /* flop_gated_lowrank_bwd                   */
   FLOP_OP_L0 = 2,          /* flop_expected_l0_lagrangian (T = gates n, r = n_seg) */
   FLOP_OP_COMPACT = 3,     /* flop_compact_ranks                       */
-  FLOP_OP_COMPACT_FWD = 4  /* flop_compact_fwd (r = k)                 */
+  FLOP_OP_COMPACT_FWD = 4, /* flop_compact_fwd (r = k)                 */
+  FLOP_OP_EMBEDDING_BWD = 5 /* flop_gated_embedding_bwd (r = d_i)       */
 } flop_op_t;
 
 const char* flop_status_string(int status);
@@ -274,6 +275,28 @@ int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const
                                         const float* seg_size, int32_t n_seg, flop_hc_params_t hc,
                                         const float* target, const float* lambda, float* out4,
                                         float* seg_expected, float* dlog_alpha, void* stream);
+
+/* Gated adaptive embedding of one word cluster (Section 4.2): E~ = E G O with E[n_rows, d_i] the
+ * reduced-dimension embeddings of the cluster's words, O[d_i, d] the projection to the model
+ * dimension and G = diag(z) pruning the d_i reduced dimensions.  ids[T] (int32, DEVICE) are row
+ * indices into E (values outside [0, n_rows) are clamped).  bf16 only.
+ *   forward : H_save[T, d_i] = E[ids, :] * z (required, it feeds the backward pass), Y[T, d] = H_save O
+ *   backward: dH' = dY O^T, dO = H_save^T dY (type wgrad_dt; overwritten or += with accumulate),
+ *             dE[ids[t], :] += dH'[t, :] * z  (fp32, ALWAYS accumulated with atomic adds because words
+ *             repeat across tokens: clear dE before the first call of a step; the order of the adds
+ *             is not fixed, so dE is reproducible only to fp32 rounding),
+ *             dlog_alpha = dz_dla * sum_t E[ids[t], :] dH'[t, :]  (fixed summation order).
+ *   Any of dE, dO, dlog_alpha may be NULL.  Workspace: flop_workspace_bytes(FLOP_OP_EMBEDDING_BWD, T,
+ *   0, 0, d_i, dt).  The tied softmax side of the same cluster, logits = ((h O^T) * z) E^T, is
+ *   flop_gated_lowrank_fwd/bwd with Q = O^T and P = E. */
+int flop_gated_embedding_fwd(const int32_t* ids, int64_t T, const void* E, int64_t lde, int64_t n_rows,
+                             const void* O, int64_t ldo, const float* z, void* Y, int64_t ldy, void* H_save,
+                             int64_t ldh, int64_t d_i, int64_t d, int dt, void* stream);
+int flop_gated_embedding_bwd(const void* dY, int64_t lddy, const int32_t* ids, int64_t T, const void* E,
+                             int64_t lde, int64_t n_rows, const void* O, int64_t ldo, const float* z,
+                             const float* dz_dla, const void* H_save, int64_t ldh, float* dE, int64_t ldde,
+                             void* dO, int64_t lddo, float* dlog_alpha, int accumulate, int64_t d_i, int64_t d,
+                             int dt, int wgrad_dt, void* ws, size_t ws_bytes, void* stream);
 
 /* FLOP-AGP variant (Section 5, baselines): magnitude-based pruning of the learnable diagonal mask
  * G = diag(g) instead of hard-concrete gates.  Segment i (one weight matrix) owns

@@ -35,6 +35,7 @@ other than itself:
                           brute-force masking of the uncompacted layer.
     agp_gates             brute-force properties of the magnitude rule (counts, kept >= pruned,
                           tie order), finite differences of the L1 term.
+    gated_embedding_fwd/bwd  equal to the (pinned) layer functions on one-hot inputs.
     The *choices* the paper leaves open (values of kept inference gates,
     top-k tie-break, which factor absorbs the gate) are "parity unpinned":
     several answers satisfy the paper, the oracle fixes one.
@@ -316,3 +317,44 @@ def agp_gates(g, seg_off, sparsity, l1):
             z[lo + k] = g[lo + k]
         seg_l1[i] = np.sum(np.abs(g[lo:hi]))
     return dict(z=z, mask=mask, dz_dg=mask.astype(np.float64), seg_l1=seg_l1, l1_grad=float(l1) * np.sign(g))
+
+
+# ----------------------------------------------------------------------------
+# Gated adaptive embedding of one word cluster (Section 4.2): E~ = E G O
+# ----------------------------------------------------------------------------
+def gated_embedding_fwd(ids, E, O, z):
+    """Embedding lookup through the gated factorization of one word cluster.
+
+    E [n, d_i] holds the reduced-dimension embeddings of the cluster's n words,
+    O [d_i, d] projects them back to the model dimension, G = diag(z) prunes
+    the d_i reduced dimensions:  row t of Y is (E[ids[t], :] * z) O.
+    Returns (H = E[ids], H' = H * z, Y).
+    """
+    E = np.asarray(E, dtype=np.float64)
+    O = np.asarray(O, dtype=np.float64)
+    z = np.asarray(z, dtype=np.float64)
+    H = E[np.asarray(ids, dtype=np.int64)]
+    Hp = H * z[None, :]
+    return H, Hp, Hp @ O
+
+
+def gated_embedding_bwd(dY, ids, E, O, z, dz_dla):
+    """Chain rule through gated_embedding_fwd:
+        dH' = dY O^T      dO = H'^T dY      dz_k = sum_t H[t,k] dH'[t,k]
+        dE[w, :] = sum over the tokens t with ids[t] = w of dH'[t, :] * z
+        dalpha = dz * dz/dalpha
+    """
+    dY = np.asarray(dY, dtype=np.float64)
+    E = np.asarray(E, dtype=np.float64)
+    O = np.asarray(O, dtype=np.float64)
+    z = np.asarray(z, dtype=np.float64)
+    ids = np.asarray(ids, dtype=np.int64)
+    H = E[ids]
+    Hp = H * z[None, :]
+    dHp = dY @ O.T
+    dO = Hp.T @ dY
+    dz = np.sum(H * dHp, axis=0)
+    dE = np.zeros_like(E)
+    for t in range(len(ids)):
+        dE[ids[t]] += dHp[t] * z
+    return dict(dE=dE, dO=dO, dz=dz, dlog_alpha=dz * np.asarray(dz_dla, dtype=np.float64))

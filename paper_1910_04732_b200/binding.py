@@ -18,14 +18,15 @@ LIB_PATH = os.path.join(_HERE, "libflop_b200.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 F32, BF16 = 0, 1
-OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD = range(5)
+OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD, OP_EMBEDDING_BWD = range(6)
 
 EXPORTS = ("flop_status_string", "flop_device_status", "flop_selftest_wait_timeout", "flop_launch_count", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_gemm_stamps_begin", "flop_gemm_stamps_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
            "flop_expected_l0_lagrangian",
-           "flop_expected_l0_lagrangian_noalloc", "flop_agp_gates",
+           "flop_expected_l0_lagrangian_noalloc", "flop_agp_gates", "flop_gated_embedding_fwd",
+           "flop_gated_embedding_bwd",
            "flop_compact_ranks", "flop_compact_fwd")
 
 
@@ -114,6 +115,9 @@ def load_library() -> ctypes.CDLL:
     lib.flop_expected_l0_lagrangian.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp,
                                                 vp, sz, vp]
     lib.flop_expected_l0_lagrangian_noalloc.argtypes = [vp, i64, vp, vp, ctypes.c_int32, HcParams, vp, vp, vp, vp, vp, vp]
+    lib.flop_gated_embedding_fwd.argtypes = [vp, i64, vp, i64, i64, vp, i64, vp, vp, i64, vp, i64, i64, i64, ci, vp]
+    lib.flop_gated_embedding_bwd.argtypes = [vp, i64, vp, i64, vp, i64, i64, vp, i64, vp, vp, vp, i64, vp, i64, vp, i64,
+                                             vp, ci, i64, i64, ci, ci, vp, sz, vp]
     lib.flop_agp_gates.argtypes = [vp, i64, vp, ctypes.c_int32, vp, ctypes.c_float, vp, vp, vp, vp, vp, vp]
     lib.flop_compact_ranks.argtypes = [vp, ci, HcParams, i64, vp, i64, vp, i64, i64, i64, ci,
                                        vp, vp, vp, vp, i64, vp, i64, vp, sz, vp]
@@ -342,6 +346,23 @@ def expected_l0_lagrangian_noalloc(log_alpha, seg_off, seg_size, hc, target, lam
         _ptr(log_alpha), log_alpha.numel(), _ptr(seg_off), _ptr(seg_size), seg_size.numel(), _hc(hc),
         _ptr(target), _ptr(lam), _ptr(out4), _ptr(seg_expected), _ptr(dlog_alpha), _stream()),
         "flop_expected_l0_lagrangian_noalloc")
+
+
+def gated_embedding_fwd(ids, E, O, z, Y, H_save) -> None:
+    T, (n_rows, d_i), d = ids.numel(), E.shape, O.shape[1]
+    _check(load_library().flop_gated_embedding_fwd(_ptr(ids), T, _ptr(E), _ld(E), n_rows, _ptr(O), _ld(O), _ptr(z), _ptr(Y),
+                                                   _ld(Y), _ptr(H_save), _ld(H_save), d_i, d, _dt(E), _stream()),
+           "flop_gated_embedding_fwd")
+
+
+def gated_embedding_bwd(dY, ids, E, O, z, dz_dla, H_save, dE, dO, dlog_alpha, ws, accumulate: bool = False) -> None:
+    T, (n_rows, d_i), d = ids.numel(), E.shape, O.shape[1]
+    wdt = _dt(dO) if dO is not None else BF16
+    _check(load_library().flop_gated_embedding_bwd(
+        _ptr(dY), _ld(dY), _ptr(ids), T, _ptr(E), _ld(E), n_rows, _ptr(O), _ld(O), _ptr(z), _ptr(dz_dla), _ptr(H_save),
+        _ld(H_save), _ptr(dE), _ld(dE) if dE is not None else 0, _ptr(dO), _ld(dO) if dO is not None else 0,
+        _ptr(dlog_alpha), int(accumulate), d_i, d, _dt(E), wdt, _ptr(ws), ws.numel() if ws is not None else 0, _stream()),
+        "flop_gated_embedding_bwd")
 
 
 def agp_gates(g, seg_off, sparsity, l1: float, z, mask=None, dz_dg=None, seg_l1=None, dg=None) -> None:

@@ -28,6 +28,7 @@
 #include "active_ranks.cuh"
 #include "gemm_small_t.cuh"
 #include "agp.cuh"
+#include "embedding.cuh"
 
 using namespace flop;
 typedef __nv_bfloat16 bf16;
@@ -724,6 +725,8 @@ int flop_tc_gemm(const void* A, int64_t lda, int a_mn_major, const void* B, int6
   return FLOP_OK;
 }
 
+static size_t embedding_ws_bytes(int64_t T, int64_t d_i);
+
 int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt, size_t* out_bytes) {
   if (!out_bytes || T < 0 || d_in < 0 || d_out < 0 || r < 0 || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
   Arena ar{nullptr, 0, 0};
@@ -739,6 +742,7 @@ int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t
     }
     case FLOP_OP_L0: ar.used = l0_ws_bytes(T, r); break;
     case FLOP_OP_COMPACT: ar.used = 0; break;
+    case FLOP_OP_EMBEDDING_BWD: ar.used = embedding_ws_bytes(T, r); break;
     default: return FLOP_ERR_INVALID_ARG;
   }
   *out_bytes = align_up(ar.used, 256);
@@ -1309,6 +1313,91 @@ int flop_agp_gates(const float* g, int64_t n, const int64_t* seg_off, int32_t n_
            mask, dz_dg, seg_l1, dg);
   count_launch();
   FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+// ---- gated adaptive embedding of one word cluster (Section 4.2): Y = (E[ids] * z) O
+static size_t embedding_ws_bytes(int64_t T, int64_t d_i) {
+  Arena ar{nullptr, 0, 0};
+  ar.take((size_t)T * round_up(std::max<int64_t>(d_i, 1), 8) * 2);                                   // dH'
+  const int64_t blocks = (T + kEmbWarps * kEmbTokensPerWarp - 1) / (kEmbWarps * kEmbTokensPerWarp);
+  ar.take((size_t)std::max<int64_t>(blocks, 1) * std::max<int64_t>(d_i, 1) * 4);                     // dz partials
+  return align_up(ar.used, 256);
+}
+
+int flop_gated_embedding_fwd(const int32_t* ids, int64_t T, const void* E, int64_t lde, int64_t n_rows, const void* O,
+                             int64_t ldo, const float* z, void* Y, int64_t ldy, void* H_save, int64_t ldh, int64_t d_i,
+                             int64_t d, int dt, void* stream) {
+  if (T < 0 || n_rows < 0 || d_i < 0 || d < 0 || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  if (dt != FLOP_BF16) return FLOP_ERR_UNSUPPORTED;
+  if (T == 0 || d == 0) return FLOP_OK;
+  if (d_i == 0 || n_rows == 0) return bf16_ok(Y, ldy) ? zero_2d<bf16>(Y, ldy, T, d, (cudaStream_t)stream) : FLOP_ERR_UNSUPPORTED;
+  if (!ids || !z || !check_mat(E, lde, d_i) || !check_mat(O, ldo, d) || !check_mat(Y, ldy, d) || !check_mat(H_save, ldh, d_i))
+    return FLOP_ERR_INVALID_ARG;
+  if (!bf16_ok(E, lde) || !bf16_ok(O, ldo) || !bf16_ok(Y, ldy) || !bf16_ok(H_save, ldh)) return FLOP_ERR_UNSUPPORTED;
+  if (T > INT32_MAX || n_rows > INT32_MAX || d_i > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  launch_k(embed_gather_kernel, dim3((unsigned)((T + kEmbWarps - 1) / kEmbWarps)), dim3(32 * kEmbWarps), (size_t)0, st, ids, (int)T,
+           (const bf16*)E, lde, (int)n_rows, z, (int)d_i, (bf16*)H_save, ldh);
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  // Y[T, d] = H'[T, d_i] O[d_i, d]: B(n, k) = O[k, n] is read "transposed" (MN-major)
+  const TcPlan pl = plan_tc(T, d, d_i, false, true);
+  return launch_tc({H_save, ldh, false}, {O, ldo, true}, T, d, d_i, pl, store_epilogue(Y, ldy, nullptr), st);
+}
+
+int flop_gated_embedding_bwd(const void* dY, int64_t lddy, const int32_t* ids, int64_t T, const void* E, int64_t lde,
+                             int64_t n_rows, const void* O, int64_t ldo, const float* z, const float* dz_dla,
+                             const void* H_save, int64_t ldh, float* dE, int64_t ldde, void* dO, int64_t lddo,
+                             float* dlog_alpha, int accumulate, int64_t d_i, int64_t d, int dt, int wgrad_dt, void* ws,
+                             size_t ws_bytes, void* stream) {
+  if (T < 0 || n_rows < 0 || d_i < 0 || d < 0 || !valid_dt(dt) || !valid_dt(wgrad_dt)) return FLOP_ERR_INVALID_ARG;
+  if (dt != FLOP_BF16) return FLOP_ERR_UNSUPPORTED;
+  if ((dE && ldde < d_i) || (dO && lddo < d) || (dlog_alpha && !dz_dla)) return FLOP_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (T == 0 || d == 0 || d_i == 0 || n_rows == 0) {      // empty batch or empty cluster: gradients are zero
+    if (!accumulate) {
+      if (dO) FLOP_TRY(wgrad_dt == FLOP_BF16 ? zero_2d<bf16>(dO, lddo, d_i, d, st) : zero_2d<float>(dO, lddo, d_i, d, st));
+      if (dlog_alpha) FLOP_TRY(zero_2d<float>(dlog_alpha, d_i, 1, d_i, st));
+    }
+    return FLOP_OK;
+  }
+  if (!ids || !z || !check_mat(dY, lddy, d) || !check_mat(E, lde, d_i) || !check_mat(O, ldo, d) || !check_mat(H_save, ldh, d_i))
+    return FLOP_ERR_INVALID_ARG;
+  if (!bf16_ok(dY, lddy) || !bf16_ok(E, lde) || !bf16_ok(O, ldo) || !bf16_ok(H_save, ldh)) return FLOP_ERR_UNSUPPORTED;
+  if (T > INT32_MAX || n_rows > INT32_MAX || d_i > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  if ((size_t)kEmbWarps * d_i * 4 > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
+  FLOP_TRY(check_ws(ws, ws_bytes, embedding_ws_bytes(T, d_i)));
+  Arena ar{(unsigned char*)ws, ws_bytes, 0};
+  const int64_t lddh = round_up(d_i, 8);
+  bf16* dH = (bf16*)ar.take((size_t)T * lddh * 2);
+  const int64_t blocks = (T + kEmbWarps * kEmbTokensPerWarp - 1) / (kEmbWarps * kEmbTokensPerWarp);
+  float* part = (float*)ar.take((size_t)blocks * d_i * 4);
+  // dH'[T, d_i] = dY[T, d] O^T: B(n = k_dim, k = j) = O[n, j] (K-major as stored)
+  FLOP_TRY(launch_tc({dY, lddy, false}, {O, ldo, false}, T, d_i, d, plan_tc(T, d_i, d, false, false),
+                     store_epilogue(dH, lddh, nullptr), st));
+  if (dO) {
+    // dO[d_i, d] = H'^T dY: contraction over tokens, written in place when the output allows 16-byte vectors
+    if (wgrad_direct_ok(dO, lddo, wgrad_dt)) {
+      TcPlan pl = plan_tc(d_i, d, T, false, true);
+      FLOP_TRY(launch_tc({H_save, ldh, true}, {dY, lddy, true}, d_i, d, T, pl, wgrad_epilogue(dO, lddo, wgrad_dt, nullptr, accumulate), st));
+    } else {
+      return FLOP_ERR_UNSUPPORTED;
+    }
+  }
+  if (dE || dlog_alpha) {
+    const size_t smem = (size_t)kEmbWarps * d_i * 4;
+    if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(embed_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    launch_k(embed_bwd_kernel, dim3((unsigned)blocks), dim3(32 * kEmbWarps), smem, st, ids, (int)T, (const bf16*)E, lde, (int)n_rows, z,
+             (int)d_i, (const bf16*)dH, lddh, dE, ldde, dlog_alpha ? part : nullptr);
+    count_launch();
+    if (dlog_alpha) {
+      launch_k(dalpha_kernel, dim3((unsigned)((d_i + 255) / 256)), dim3(256), (size_t)0, st, (const float*)part, (int)blocks, d_i, dz_dla,
+               (int)d_i, dlog_alpha, accumulate);
+      count_launch();
+    }
+    FLOP_CUDA(cudaGetLastError());
+  }
   return FLOP_OK;
 }
 

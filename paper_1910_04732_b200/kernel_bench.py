@@ -138,7 +138,32 @@ def main():
     # ---- training on the active rank components: one BERT-shaped layer (six matrices, T = 4096)
     for wl in ("bert", "sru"):
         active_table(I.WORKLOADS[wl], g)
+    embedding_table(g)
     assert b.device_status() == b.OK
+
+
+def embedding_table(g):
+    """Gated adaptive embedding: the three word clusters of the word-level model (reduced dimensions
+    1024 / 256 / 64 for the 20K most frequent, the next 40K and the remaining words; d = 1024),
+    T = 64 x 256 tokens drawn with a heavy-tailed frequency."""
+    bf = torch.bfloat16
+    T, d = 64 * 256, 1024
+    print(f"\ngated adaptive embedding, T={T} tokens, d={d} (lookup E[ids]*z, projection O; backward dO, dE, dlog_alpha)")
+    print(f"{'cluster':>22s} {'fwd us':>8s} {'bwd us':>8s} {'fwd+bwd TFLOP/s':>16s}")
+    for n_rows, d_i in ((20000, 1024), (40000, 256), (200000, 64)):
+        E = (torch.randn(n_rows, d_i, generator=g, device="cuda")).to(bf)
+        O_ = (torch.randn(d_i, d, generator=g, device="cuda") * d_i ** -0.5).to(bf)
+        dY = torch.randn(T, d, generator=g, device="cuda").to(bf)
+        ids = (torch.rand(T, generator=g, device="cuda") ** 4 * n_rows).to(torch.int32).clamp_(0, n_rows - 1)
+        z = (torch.rand(d_i, generator=g, device="cuda") < 0.6).float() * 0.8
+        dzd = torch.ones(d_i, device="cuda")
+        Y, H = b.padded(T, d, bf), b.padded(T, d_i, bf)
+        dE, dO, dla = torch.zeros(n_rows, d_i, device="cuda"), b.padded(d_i, d, bf), torch.zeros(d_i, device="cuda")
+        ws = b.alloc_workspace(b.workspace_bytes(b.OP_EMBEDDING_BWD, T, 0, 0, d_i, b.BF16))
+        tf = timed(lambda: b.gated_embedding_fwd(ids, E, O_, z, Y, H), iters=20, graph=True)
+        tb = timed(lambda: b.gated_embedding_bwd(dY, ids, E, O_, z, dzd, H, dE, dO, dla, ws), iters=20, graph=True)
+        flops = 6.0 * T * d_i * d          # one forward and two backward GEMMs
+        print(f"{f'n={n_rows}, d_i={d_i}':>22s} {tf * 1e6:8.1f} {tb * 1e6:8.1f} {flops / (tf + tb) / 1e12:16.0f}")
 
 
 def active_table(w, g):
