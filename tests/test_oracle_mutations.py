@@ -26,9 +26,9 @@ MUTANTS = [
      ["test_oracle_layer.test_sum_of_rank_one_components"]),
     ("forward_transposed_Q", "    H = X @ Q.T\n    Hp = H * z[None, :]\n    Y = Hp @ P.T", "    H = X @ Q[:, ::-1].T\n    Hp = H * z[None, :]\n    Y = Hp @ P.T",
      ["test_oracle_layer.test_sum_of_rank_one_components"]),
-    ("dP_uses_ungated_H", "dP = dY.T @ Hp", "dP = dY.T @ H",
+    ("dP_uses_ungated_H", "dP = dY.T @ Hp\n", "dP = dY.T @ H\n",
      ["test_oracle_layer.test_backward_matches_central_finite_differences"]),
-    ("dz_uses_gated_H", "dz = np.sum(H * dHp, axis=0)", "dz = np.sum(Hp * dHp, axis=0)",
+    ("dz_uses_gated_H", "dP = dY.T @ Hp\n    dz = np.sum(H * dHp, axis=0)", "dP = dY.T @ Hp\n    dz = np.sum(Hp * dHp, axis=0)",
      ["test_oracle_layer.test_three_forms_of_dz_agree"]),
     ("dQ_drops_gate", "dQ = dH.T @ X", "dQ = dHp.T @ X",
      ["test_oracle_layer.test_backward_matches_central_finite_differences"]),
@@ -49,6 +49,14 @@ MUTANTS = [
     ("compact_gathers_rows_of_P", "return P[:, idx].copy(), z[idx][:, None] * Q[idx, :]",
      "return P[:, np.sort(idx)[::-1]].copy(), z[idx][:, None] * Q[idx, :]",
      ["test_oracle_compact.test_compaction_equals_brute_force_masking"]),
+    ("embedding_drops_gate_in_dE", "dE[ids[t]] += dHp[t] * z", "dE[ids[t]] += dHp[t]",
+     ["test_oracle_embedding.test_embedding_equals_layer_on_one_hot_inputs"]),
+    ("embedding_overwrites_repeated_words", "dE[ids[t]] += dHp[t] * z", "dE[ids[t]] = dHp[t] * z",
+     ["test_oracle_embedding.test_embedding_equals_layer_on_one_hot_inputs"]),
+    ("agp_prunes_largest", "key=lambda k: (-abs(g[lo + k]), k))", "key=lambda k: (abs(g[lo + k]), k))",
+     ["test_oracle_agp.test_magnitude_rule_properties_and_brute_force"]),
+    ("agp_tie_order", "key=lambda k: (-abs(g[lo + k]), k))", "key=lambda k: (-abs(g[lo + k]), -k))",
+     ["test_oracle_agp.test_ties_and_l1_term"]),
     ("uniform_closed_at_zero", ".astype(np.float64) + 0.5) * 2.0 ** -23", ".astype(np.float64) + 0.0) * 2.0 ** -23",
      ["test_oracle_philox.test_uniform_mapping_open_interval_and_exact_in_fp32"]),
     ("philox_nine_rounds", "for _ in range(10):", "for _ in range(9):",
