@@ -4,7 +4,7 @@
 // 128 x BN tile, and gemm2_group_kernel in gemm_tc2_group.cuh, a CTA pair per 256 x BN tile)
 // serve all six GEMMs of the gated factorized layer W = P diag(z) Q (Section 4.1 of the paper).
 // Both are persistent and warp-specialised:
-//   warp 0      TMA producer: cp.async.bulk.tensor (no multicast) into a ring of
+//   warp 0      TMA producer: cp.async.bulk.tensor loads (every CTA fetches its own tiles) into a ring of
 //               128-byte-swizzled shared-memory stages, completion on mbarriers
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (K = 16 per instruction, bf16 in,
 //               fp32 accumulators in tensor memory), tcgen05.commit frees stages

@@ -16,7 +16,8 @@
 //   tfull[a]   one per CTA, signalled the same way when an accumulator is complete
 //   tempty[a]  lives in rank 0, expects the epilogue warps of both CTAs (remote arrivals)
 // The accumulator rows 0..127 sit in rank 0's tensor memory, rows 128..255 in rank 1's; each
-// CTA's epilogue warps drain their own half.  No TMA load uses multicast.
+// CTA's epilogue warps drain their own half.  Every CTA fetches its own operand tiles; the commit
+// above is the only instruction that signals both CTAs at once.
 // All mbarrier waits are bounded as in the one-CTA kernel; before tensor memory is freed the
 // two CTAs shake hands through an mbarrier (bounded) so that neither signals a peer that has
 // already left.
