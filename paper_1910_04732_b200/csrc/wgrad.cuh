@@ -153,7 +153,8 @@ __device__ __forceinline__ void reduce_unit(const float* __restrict__ slices, in
 // Number of work units (4 consecutive columns of one row, or one gate) of one problem.
 __host__ __device__ inline int64_t bwd_finish_units(const BwdFinishArgs& a) {
   const int64_t c4r = (a.r + 3) >> 2, c4d = (a.d_in + 3) >> 2;
-  return (a.dP ? (int64_t)a.d_out * c4r : 0) + ((a.dQ ? 1 : 0) + (a.Qz ? 1 : 0)) * (int64_t)a.r * c4d +
+  const int64_t c8d = (a.d_in + 7) >> 3;   // diag(z) Q moves 8 columns (16 bytes) per unit
+  return (a.dP ? (int64_t)a.d_out * c4r : 0) + (a.dQ ? (int64_t)a.r * c4d : 0) + (a.Qz ? (int64_t)a.r * c8d : 0) +
          (a.dlog_alpha ? (int64_t)a.r : 0);
 }
 
@@ -162,7 +163,8 @@ __device__ __forceinline__ void bwd_finish_unit(const BwdFinishArgs& a, int64_t 
   const int c4r = (a.r + 3) >> 2, c4d = (a.d_in + 3) >> 2;
   const int64_t n_p = a.dP ? (int64_t)a.d_out * c4r : 0;
   const int64_t n_q = a.dQ ? (int64_t)a.r * c4d : 0;
-  const int64_t n_qz = a.Qz ? (int64_t)a.r * c4d : 0;
+  const int c8d = (a.d_in + 7) >> 3;
+  const int64_t n_qz = a.Qz ? (int64_t)a.r * c8d : 0;
   constexpr int al = sizeof(TW) == 4 ? 15 : 7;   // 4 outputs: 16 B (fp32) or 8 B (bf16)
   if (u < n_p) {
     const bool vec_p = ((reinterpret_cast<uintptr_t>(a.dP) & al) == 0) && (a.lddp % 4 == 0);
@@ -176,21 +178,21 @@ __device__ __forceinline__ void bwd_finish_unit(const BwdFinishArgs& a, int64_t 
     reduce_unit<TW>(a.slices_q, a.n_slices_q, a.slice_elems_q, a.ld_slice_q, row, c0, a.d_in, a.z[row], (TW*)a.dQ, a.lddq,
                     a.accumulate, vec_q);
   } else if (u < n_p + n_q + n_qz) {
-    const int64_t v = u - n_p - n_q;
-    const int row = (int)(v / c4d), c0 = (int)(v % c4d) * 4;
-    const int valid = min(4, a.d_in - c0);
+    const int v = (int)(u - n_p - n_q);
+    const int row = v / c8d, c0 = (v - row * c8d) * 8;
+    const int valid = min(8, a.d_in - c0);
     const float g = a.z[row];
     const __nv_bfloat16* q = a.Q + (int64_t)row * a.ldq + c0;
     __nv_bfloat16* o = a.Qz + (int64_t)row * a.ldqz + c0;
-    if (valid == 4) {   // Q and Qz rows are 16-byte aligned with ld % 8 == 0: 8-byte accesses are aligned
-      const uint2 raw = *reinterpret_cast<const uint2*>(q);
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
-      const float2 x = __bfloat1622float2(h[0]), y = __bfloat1622float2(h[1]);
-      __nv_bfloat162 lo = __floats2bfloat162_rn(x.x * g, x.y * g), hi = __floats2bfloat162_rn(y.x * g, y.y * g);
-      uint2 out;
-      out.x = *reinterpret_cast<uint32_t*>(&lo);
-      out.y = *reinterpret_cast<uint32_t*>(&hi);
-      *reinterpret_cast<uint2*>(o) = out;
+    if (valid == 8) {   // Q and Qz rows are 16-byte aligned (ld % 8 == 0)
+      uint4 raw = *reinterpret_cast<const uint4*>(q);
+      __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 x = __bfloat1622float2(h[i]);
+        h[i] = __floats2bfloat162_rn(x.x * g, x.y * g);
+      }
+      *reinterpret_cast<uint4*>(o) = raw;
     } else {
       for (int i = 0; i < valid; ++i) o[i] = __float2bfloat16_rn(__bfloat162float(q[i]) * g);
     }
