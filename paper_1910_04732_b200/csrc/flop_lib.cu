@@ -100,7 +100,7 @@ int num_sms() {
 // ------------------------------------------------------------------ instrumentation
 // Host-side count of kernels launched by this library, and optional CUDA-event timing of
 // the tensor-core GEMM launches (flop_gemm_timing_begin/end): events are recorded on the
-// launching stream around every gemm_kernel launch and summed when timing ends.
+// launching stream around every tensor-core GEMM launch and summed when timing ends.
 unsigned long long g_launches = 0;
 struct GemmTiming {
   bool on = false;
@@ -157,7 +157,7 @@ struct Arena {
 // ------------------------------------------------------------------ tensor-core GEMM planning
 struct TcPlan {
   int bn, stages, tiles_m, tiles_n, splits, kb_per_split, num_kb;
-  int cta2;   // 1: pairs of CTAs compute 256 x bn tiles (gemm2_kernel); 0: one CTA per 128 x bn tile
+  int cta2;   // 1: pairs of CTAs compute 256 x bn tiles (gemm2_group_kernel); 0: one CTA per 128 x bn tile
 };
 
 constexpr int kSmemBudget = 227 * 1024 - 1024;   // opt-in maximum minus room for the static __shared__ variables

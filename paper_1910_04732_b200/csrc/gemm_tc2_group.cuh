@@ -1,4 +1,4 @@
-// Grouped form of the two-CTA tensor-core GEMM (gemm2_kernel): the 256 x BN tiles of up to
+// Grouped form of the two-CTA tensor-core GEMM (pieces in gemm_tc2.cuh): the 256 x BN tiles of up to
 // kMaxGroup independent problems in one persistent launch of CTA pairs.  It combines the two
 // measures that matter at BERT / Transformer-XL sizes: several tiles per CTA, so that pipeline
 // fill and epilogue drain overlap the next tile's main loop, and half a B tile per SM, so that the
