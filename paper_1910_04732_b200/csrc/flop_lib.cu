@@ -407,8 +407,11 @@ struct GroupShape { int bn, cta2; double items; };
 // of an SM (about 50 B/clk) is what usually decides, which favours CTA pairs and wide tiles;
 // padding waste and the number of rounds pull the other way.  FLOP_TC_GROUP_BN / FLOP_TC_GROUP_CTA2
 // (1 = force pairs, 2 = forbid) override for tuning.
-GroupShape plan_group(const std::vector<Mnk>& jobs, bool b_mn_major) {
-  static const int force_bn = env_int("FLOP_TC_GROUP_BN"), force_cta2 = env_int("FLOP_TC_GROUP_CTA2");
+GroupShape plan_group(const std::vector<Mnk>& jobs, bool b_mn_major, bool wgrad = false) {
+  static const int force_bn_all = env_int("FLOP_TC_GROUP_BN"), force_cta2_all = env_int("FLOP_TC_GROUP_CTA2");
+  static const int force_bn_w = env_int("FLOP_TC_WGRAD_BN"), force_cta2_w = env_int("FLOP_TC_WGRAD_CTA2");
+  const int force_bn = wgrad && force_bn_w ? force_bn_w : force_bn_all;
+  const int force_cta2 = wgrad && force_cta2_w ? force_cta2_w : force_cta2_all;
   const int sms = num_sms();
   GroupShape best{0, 0, 0.0};
   double best_cost = 1e300;
@@ -1089,7 +1092,7 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     if (a.dQ || a.dlog_alpha) mw.push_back({a.r, a.d_in, a.T});
     if (a.dX) m6.push_back({a.T, a.d_in, a.r});
   }
-  const GroupShape s3 = plan_group(m3, true), s6 = plan_group(m6, true), sw = plan_group(mw, true);
+  const GroupShape s3 = plan_group(m3, true), s6 = plan_group(m6, true), sw = plan_group(mw, true, true);
   if (sw.bn == 0 || sw.items < (sw.cta2 ? num_sms() / 2 : num_sms())) direct = false;
   auto direct_plan = [&](int64_t M, int64_t N, int64_t K) { return fixed_plan(M, N, K, sw.bn, sw.cta2); };
   for (int i = 0; i < n; ++i) {
