@@ -27,6 +27,7 @@
 #include "wgrad.cuh"
 #include "active_ranks.cuh"
 #include "gemm_small_t.cuh"
+#include "gemm_skinny.cuh"
 #include "agp.cuh"
 #include "embedding.cuh"
 
@@ -482,9 +483,45 @@ int launch_small_t(const void* A, int64_t lda, const void* B, int64_t ldb, void*
   switch (tt) {
     case 1: return launch_small_t_inst<1>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
     case 2: return launch_small_t_inst<2>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
-    case 4: return launch_small_t_inst<4>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
-    default: return launch_small_t_inst<8>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
+    default: return launch_small_t_inst<4>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
   }
+}
+
+// Forward product for 5..16 tokens with warp-level tensor-core instructions (see gemm_skinny.cuh).
+template <int MT>
+int launch_skinny_inst(const bf16* A, int64_t lda, const bf16* B, int64_t ldb, bf16* C, int64_t ldc, const float* cs, int T, int N,
+                       int K, int k_pad, size_t smem, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    FLOP_CUDA(cudaFuncSetAttribute(skinny_gemm_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    configured = true;
+  }
+  const int groups = (N + 7) / 8;
+  const int grid = std::min((groups + kSkinnyWarps - 1) / kSkinnyWarps, num_sms() * 2);
+  launch_k(skinny_gemm_kernel<MT>, dim3(grid), dim3(32 * kSkinnyWarps), smem, st, A, lda, B, ldb, C, ldc, cs, T, N, K, k_pad);
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+int launch_skinny(const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc, const float* cs, int64_t T, int64_t N,
+                  int64_t K, cudaStream_t st) {
+  static const int off = env_int("FLOP_NO_SKINNY");
+  if (off || T < 1 || T > kSkinnyMaxT || N > INT32_MAX || K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  const int mt = (int)((T + 15) / 16);
+  const int k_pad = (int)round_up(K, 32);
+  const size_t smem = (size_t)16 * mt * (k_pad + kSkinnyPad) * 2;
+  if (smem > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
+  const bf16* a = (const bf16*)A; const bf16* b = (const bf16*)B; bf16* c = (bf16*)C;
+  switch (mt) {
+    case 1: return launch_skinny_inst<1>(a, lda, b, ldb, c, ldc, cs, (int)T, (int)N, (int)K, k_pad, smem, st);
+    default: return FLOP_ERR_UNSUPPORTED;
+  }
+}
+// Few-token forward: CUDA-core streaming up to 4 tokens, warp-level tensor cores up to 16.
+int launch_few_tokens(const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc, const float* cs, int64_t T,
+                      int64_t N, int64_t K, cudaStream_t st) {
+  if (T <= kSmallTMax) return launch_small_t(A, lda, B, ldb, C, ldc, cs, T, N, K, st);
+  return launch_skinny(A, lda, B, ldb, C, ldc, cs, T, N, K, st);
 }
 
 int launch_simt(const float* A, int64_t a_sm, int64_t a_sk, const float* B, int64_t b_sn, int64_t b_sk, float* C,
@@ -794,10 +831,10 @@ static int fwd_impl(const void* X, int64_t ldx, const void* Q, int64_t ldq, cons
       if (r > 0) FLOP_TRY(zero_2d<bf16>(H, ldh, T, r, st));
       return FLOP_OK;
     }
-    if (T <= kSmallTMax) {   // a handful of tokens: stream the weights once on the CUDA cores
-      const int rc = launch_small_t(X, ldx, Q, ldq, H, ldh, z, T, r, d_in, st);
+    if (T <= kSkinnyMaxT) {   // a few tokens: the weights are streamed once (CUDA cores up to 4 tokens, warp-level MMA up to 16)
+      const int rc = launch_few_tokens(X, ldx, Q, ldq, H, ldh, z, T, r, d_in, st);
       if (rc == FLOP_OK) {
-        const int rc2 = launch_small_t(H, ldh, P, ldp, Y, ldy, nullptr, T, d_out, r, st);
+        const int rc2 = launch_few_tokens(H, ldh, P, ldp, Y, ldy, nullptr, T, d_out, r, st);
         if (rc2 != FLOP_ERR_UNSUPPORTED) return rc2;
       } else if (rc != FLOP_ERR_UNSUPPORTED) {
         return rc;
@@ -860,10 +897,10 @@ int flop_compact_fwd(const void* X, int64_t ldx, const void* Qc, int64_t ldqc, c
   const FwdWs w = plan_fwd_ws(ar, T, k, dt);
   if (dt == FLOP_BF16) {
     if (!bf16_ok(Y, ldy) || !bf16_ok(X, ldx) || !bf16_ok(Qc, ldqc) || !bf16_ok(Pc, ldpc)) return FLOP_ERR_UNSUPPORTED;
-    if (T <= kSmallTMax) {
-      const int rc = launch_small_t(X, ldx, Qc, ldqc, w.H, w.ldh, nullptr, T, k, d_in, st);
+    if (T <= kSkinnyMaxT) {
+      const int rc = launch_few_tokens(X, ldx, Qc, ldqc, w.H, w.ldh, nullptr, T, k, d_in, st);
       if (rc == FLOP_OK) {
-        const int rc2 = launch_small_t(w.H, w.ldh, Pc, ldpc, Y, ldy, nullptr, T, d_out, k, st);
+        const int rc2 = launch_few_tokens(w.H, w.ldh, Pc, ldpc, Y, ldy, nullptr, T, d_out, k, st);
         if (rc2 != FLOP_ERR_UNSUPPORTED) return rc2;
       } else if (rc != FLOP_ERR_UNSUPPORTED) {
         return rc;

@@ -1,23 +1,23 @@
-// Forward GEMM for a handful of tokens (T <= 8), bf16 in, fp32 accumulate, bf16 out:
+// Forward GEMM for a handful of tokens (T <= 4), bf16 in, fp32 accumulate, bf16 out:
 //     C[t, n] = col_scale[n] * sum_k A[t, k] B[n, k]          (A [T, K], B [N, K], both K-major)
 //
-// At T = 1..8 (pruned inference, batch x sequence of a few tokens) the product is a
+// At T = 1..4 (pruned inference, batch x sequence of a few tokens) the product is a
 // weight-streaming problem: every row of B is read once and used T times, a 128-row tensor-core
 // tile would be at most a quarter full, and a tensor-core launch costs ~9 us of pipeline set-up
 // against ~1 us of weight traffic.  Here one warp owns one output column n: its lanes stride over
 // K with 16-byte loads of B[n, :], multiply with the T rows of A held in shared memory, and a
 // shuffle tree adds the 32 partial sums per token.  Bound: HBM/L2 read of B.  Measured on the
-// 1024 -> 4096, k = 412 inference case: 6.3 / 8.3 / 10.3 / 14.4 us at T = 1 / 2 / 4 / 8 against a
-// flat 18.5 us for the tensor-core path, which takes over from T = 9.
+// 1024 -> 4096, k = 412 inference case: 6.3 / 8.3 / 10.3 / 14.4 us at T = 1 / 2 / 4 / 8; from T = 5 the
+// warp-level tensor-core kernel (gemm_skinny.cuh, 12 us) is faster.
 #pragma once
 #include "common.cuh"
 
 namespace flop {
 
-constexpr int kSmallTMax = 8;
+constexpr int kSmallTMax = 4;
 constexpr int kSmallTWarps = 8;
 
-template <int TT>   // TT = tokens rounded up to 1, 2, 4 or 8 (accumulators per lane)
+template <int TT>   // TT = tokens rounded up to 1, 2 or 4 (accumulators per lane)
 __global__ void __launch_bounds__(32 * kSmallTWarps)
 small_t_gemm_kernel(const __nv_bfloat16* __restrict__ A, int64_t lda, const __nv_bfloat16* __restrict__ B, int64_t ldb,
                     __nv_bfloat16* __restrict__ C, int64_t ldc, const float* __restrict__ col_scale, int T, int N, int K,

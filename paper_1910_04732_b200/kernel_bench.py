@@ -126,7 +126,7 @@ def main():
     k = int(kd.item())
     print(f"\npruned inference, d_in={mtx.d_in} d_out={mtx.d_out} r={mtx.r}: k = {k} survive; compaction (select + gather) {t_c * 1e6:.1f} us")
     print(f"{'T':>6s} {'compact fwd us':>15s} {'gated fwd us':>13s} {'speed-up':>9s} {'compact GFLOP/s':>16s} {'weight GB/s':>12s}")
-    for T in (1, 4, 16, 256, 4096):
+    for T in (1, 4, 8, 16, 64, 256, 4096):
         Xt = X[:T]
         Y, H = b.padded(T, mtx.d_out, bf), b.padded(T, mtx.r, bf)
         wsc = b.alloc_workspace(b.workspace_bytes(b.OP_COMPACT_FWD, T, mtx.d_in, mtx.d_out, k, b.BF16))

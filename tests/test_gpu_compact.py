@@ -85,7 +85,7 @@ def test_pruned_inference_config(b, dtype):
     assert np.all(np.isnan(host(Pc)[:, k:])) and np.all(np.isnan(host(Qc)[k:]))     # the rest is untouched
     assert rel_fro(host(Qc)[:k], Qco) < (4e-3 if dtype == "bf16" else 1e-6)
     tol = 2e-2 if dtype == "bf16" else 1e-5
-    for T in (1, 3, 8, 16, 256, 4096):          # 1..8: weight-streaming kernel, above: tensor cores
+    for T in (1, 3, 4, 5, 9, 16, 17, 64, 256, 4096):   # 1..4: CUDA-core streaming, 5..16: warp-level MMA, above: tcgen05
         X = to_dev(prob["X"][:T], dtype)
         Y = empty_dev(T, m.d_out, tdt)
         ws = b.alloc_workspace(b.workspace_bytes(b.OP_COMPACT_FWD, T, m.d_in, m.d_out, k, b.BF16 if dtype == "bf16" else b.F32))

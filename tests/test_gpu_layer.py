@@ -91,7 +91,7 @@ def test_f32_ragged_shapes(b, T, d_in, d_out, r):
     (1000, 410, 410, 410),     # Transformer-XL attention shape, K tail of 26
     (640, 410, 2100, 410),     # FFN1 shape
     (640, 2100, 410, 410),     # FFN2 shape
-    (1, 64, 64, 64), (16, 1024, 4096, 358),
+    (1, 64, 64, 64), (16, 1024, 4096, 358), (40, 200, 136, 72), (64, 410, 2100, 410),
     (2048, 768, 768, 768)])
 def test_bf16_shapes(b, T, d_in, d_out, r):
     w = I.Workload("t", "bf16", T, 1, (I.Matrix("w", d_in, d_out, r),), ("normal", 0.5, 1.5), 0.5)
