@@ -164,7 +164,21 @@ gather_p_kernel(const T* __restrict__ P, int64_t ldp, const int32_t* __restrict_
     }
     __syncthreads();
     T* o = Pc + (int64_t)i * ldpc;
-    for (int c = threadIdx.x; c < k; c += blockDim.x) o[c] = row[idx[c]];   // 2-byte stores, coalesced across the warp
+    // four surviving columns per thread and store where the element type and the alignment allow it
+    // (8-byte stores, 256 bytes per warp instruction), single elements otherwise
+    if (sizeof(T) == 2 && (reinterpret_cast<uintptr_t>(o) & 7) == 0 && (reinterpret_cast<uintptr_t>(idx) & 15) == 0) {
+      for (int c = threadIdx.x * 4; c < k; c += blockDim.x * 4) {
+        if (c + 3 < k) {
+          const int4 ii = *reinterpret_cast<const int4*>(idx + c);
+          T quad[4] = {row[ii.x], row[ii.y], row[ii.z], row[ii.w]};
+          *reinterpret_cast<uint2*>(o + c) = *reinterpret_cast<uint2*>(quad);
+        } else {
+          for (int e = c; e < k; ++e) o[e] = row[idx[e]];
+        }
+      }
+    } else {
+      for (int c = threadIdx.x; c < k; c += blockDim.x) o[c] = row[idx[c]];
+    }
     __syncthreads();
   }
 }
