@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD, OP_EMBEDDING_BWD = range(6)
 
-EXPORTS = ("flop_status_string", "flop_device_status", "flop_selftest_wait_timeout", "flop_launch_count", "flop_gemm_timing_begin",
+EXPORTS = ("flop_status_string", "flop_device_status", "flop_selftest_wait_timeout", "flop_launch_count", "flop_plan_tile_schedule", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_gemm_stamps_begin", "flop_gemm_stamps_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
@@ -93,6 +93,9 @@ def load_library() -> ctypes.CDLL:
     lib.flop_device_status.argtypes = [vp]
     lib.flop_workspace_bytes.argtypes = [ci, i64, i64, i64, i64, ci, ctypes.POINTER(sz)]
     lib.flop_launch_count.argtypes = []
+    lib.flop_plan_tile_schedule.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int32, ctypes.c_int32,
+                                            ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double),
+                                            ctypes.POINTER(ctypes.c_double)]
     lib.flop_selftest_wait_timeout.argtypes = [i64, vp, vp]
     lib.flop_gemm_timing_begin.argtypes = []
     lib.flop_gemm_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
@@ -127,6 +130,17 @@ def load_library() -> ctypes.CDLL:
     lib.flop_launch_count.restype = ctypes.c_ulonglong
     _lib = lib
     return lib
+
+
+def plan_tile_schedule(cost, units: int):
+    """Host-only: (unit of every work item, largest unit load, largest load of the round-robin deal)."""
+    n = len(cost)
+    c = (ctypes.c_double * max(n, 1))(*[float(v) for v in cost])
+    out = (ctypes.c_int32 * max(n, 1))()
+    ms, rr = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(load_library().flop_plan_tile_schedule(c, n, int(units), out, ctypes.byref(ms), ctypes.byref(rr)),
+           "flop_plan_tile_schedule")
+    return list(out)[:n], ms.value, rr.value
 
 
 def status_string(code: int) -> str:

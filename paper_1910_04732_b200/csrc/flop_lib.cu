@@ -304,10 +304,10 @@ int launch_group_inst(const tc::GroupParams& gp, int cta2, double flops, cudaStr
     GemmTimer timer(st, flops);
     if (!cta2) {
       const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes(gp.bn_max);
-      launch_k(kern1, dim3(std::min(gp.total_work, num_sms())), dim3(tc::kThreads), (size_t)smem, st, gp);
+      launch_k(kern1, dim3(gp.sched.n_units ? gp.sched.n_units : std::min(gp.total_work, num_sms())), dim3(tc::kThreads), (size_t)smem, st, gp);
     } else {
       const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes2(gp.bn_max);
-      const int pairs = std::min(gp.total_work, num_sms() / 2);
+      const int pairs = gp.sched.n_units ? gp.sched.n_units : std::min(gp.total_work, num_sms() / 2);
       cudaLaunchConfig_t cfg{};
       cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
       cudaLaunchAttribute attr[2];
@@ -332,6 +332,7 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     memset(&gp, 0, sizeof(gp));
     double flops = 0.0;
     const TcJob& first = jobs[i];
+    std::vector<double> item_cost;
     for (; i < jobs.size() && gp.n < tc::kMaxGroup; ++i) {
       const TcJob& j = jobs[i];
       if (j.M <= 0 || j.N <= 0 || j.K <= 0) continue;
@@ -360,6 +361,15 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       if (p.tma_store) FLOP_TRY(make_tmap(&pr.tout, tma_dst, j.M, j.N, j.ep.ldo, 64, 32));
       pr.work_begin = gp.total_work;
       gp.total_work += p.tiles_m * p.tiles_n * p.splits;
+      {   // cost of each work item of this problem in SM cycles (the model of plan_group), for the schedule
+        const double bytes = j.pl.cta2 ? (double)tc::stage_bytes2(p.bn) : (double)tc::stage_bytes(p.bn);
+        const double per_kb = std::max(2.0 * p.bn, bytes / 50.0), epi = 400.0 + 4.0 * p.bn;
+        if (item_cost.size() <= (size_t)tc::kMaxSched)
+          for (int sp = 0; sp < p.splits; ++sp) {
+            const int kbs = std::min(p.kb_per_split, p.num_kb - sp * p.kb_per_split);
+            item_cost.insert(item_cost.end(), (size_t)p.tiles_m * p.tiles_n, kbs * per_kb + epi);
+          }
+      }
       gp.bn_max = std::max(gp.bn_max, p.bn);
       flops += 2.0 * j.M * (double)j.N * j.K;
       ++gp.n;
@@ -372,6 +382,19 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     if (g_stamps.buf && g_stamps.used < g_stamps.capacity) {
       gp.stamp = g_stamps.buf + 2 * g_stamps.used++;
       g_stamps.flops += flops;
+    }
+    // Tiles of unequal length: deal them out by the longest-processing-time rule when that beats the
+    // round-robin order (FLOP_NO_SCHED=1 keeps round-robin, for comparison).
+    {
+      static const int no_sched = env_int("FLOP_NO_SCHED");
+      const int units = std::min(gp.total_work, cta2 ? num_sms() / 2 : num_sms());
+      double rr = 0.0;
+      if (no_sched || (int)item_cost.size() != gp.total_work) {
+        gp.sched.n_units = 0;
+      } else {
+        const double lpt = tc::build_schedule(item_cost, units, &gp.sched, &rr);
+        if (lpt < 0.0 || lpt > 0.97 * rr) gp.sched.n_units = 0;
+      }
     }
     const bool a_mn = first.A.mn_major, b_mn = first.B.mn_major;
     int rc = FLOP_ERR_UNSUPPORTED;
@@ -690,6 +713,23 @@ int flop_selftest_wait_timeout(int64_t limit_cycles, int* gave_up_dev, void* str
 }
 
 unsigned long long flop_launch_count(void) { return g_launches; }
+
+int flop_plan_tile_schedule(const double* cost, int32_t n, int32_t units, int32_t* unit_of_item, double* makespan,
+                            double* rr_makespan) {
+  if (n < 0 || (n > 0 && !cost) || n > tc::kMaxSched || units < 1 || units > tc::kMaxUnits) return FLOP_ERR_INVALID_ARG;
+  std::vector<double> c(cost, cost + n);
+  static tc::Schedule sched;   // 4 KB: kept off the stack
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  double rr = 0.0;
+  const double ms = tc::build_schedule(c, units, &sched, &rr);
+  if (makespan) *makespan = n > 0 ? ms : 0.0;
+  if (rr_makespan) *rr_makespan = rr;
+  if (unit_of_item && n > 0)
+    for (int u = 0; u < units; ++u)
+      for (int i = sched.begin[u]; i < sched.begin[u + 1]; ++i) unit_of_item[sched.item[i]] = u;
+  return FLOP_OK;
+}
 
 int flop_gemm_stamps_begin(unsigned long long* stamps_dev, int capacity) {
   if (!stamps_dev || capacity <= 0) return FLOP_ERR_INVALID_ARG;

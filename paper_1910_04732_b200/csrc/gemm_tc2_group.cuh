@@ -31,7 +31,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-  const int total = gp.total_work;
+  const WorkRange wr = work_range(gp, pair, npairs);
 
   if (threadIdx.x == 0) {
     s_abort = 0;
@@ -62,8 +62,8 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int w = pair; w < total && ok; w += npairs) {
-        const GroupItem it = decode_group(gp, w, BM2);
+      for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
+        const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
         if (!it.active) continue;
         const GroupProblem& pr = gp.prob[it.g];
         const int half_n = pr.p.bn >> 1;
@@ -106,8 +106,8 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int w = pair; w < total && ok; w += npairs) {
-        const GroupItem it = decode_group(gp, w, BM2);
+      for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
+        const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
         if (!it.active) continue;
         const uint32_t idesc = instr_desc2(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait2(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -136,8 +136,8 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int w = pair; w < total && ok; w += npairs) {
-      const GroupItem it = decode_group(gp, w, BM2);
+    for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
+      const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
         if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
       if (!mbar_wait2(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }

@@ -15,6 +15,7 @@
 // gemm_tc.cuh.  A single GEMM runs as a group of one.
 #pragma once
 #include "gemm_tc.cuh"
+#include "schedule.cuh"
 
 namespace flop {
 namespace tc {
@@ -38,7 +39,17 @@ struct GroupParams {
   // dependency wait, [1] = the latest %globaltimer at which a CTA finished (atomic max).  Lets a
   // caller time launches that run inside a replayed CUDA graph, where host events cannot be placed.
   unsigned long long* stamp;
+  // Which work items each persistent unit walks (schedule.cuh); n_units == 0: round-robin.
+  Schedule sched;
 };
+
+// The work items of persistent unit `unit` of `nunits`: for (i = first; i < last; i += step) item = work_at(gp, i).
+struct WorkRange { int first, last, step; };
+__device__ __forceinline__ WorkRange work_range(const GroupParams& gp, int unit, int nunits) {
+  if (gp.sched.n_units) return WorkRange{(int)gp.sched.begin[unit], (int)gp.sched.begin[unit + 1], 1};
+  return WorkRange{unit, gp.total_work, nunits};
+}
+__device__ __forceinline__ int work_at(const GroupParams& gp, int i) { return gp.sched.n_units ? (int)gp.sched.item[i] : i; }
 
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -86,7 +97,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
   __shared__ int s_abort;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total = gp.total_work;
+  const WorkRange wr = work_range(gp, (int)blockIdx.x, (int)gridDim.x);
 
   if (threadIdx.x == 0) {
     s_abort = 0;
@@ -116,8 +127,8 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t phase = 0;
       int armed = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        const GroupItem it = decode_group(gp, w, BM);
+      for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
+        const GroupItem it = decode_group(gp, work_at(gp, wi), BM);
         if (!it.active) continue;
         const GroupProblem& pr = gp.prob[it.g];
         const int bn = pr.p.bn;
@@ -163,8 +174,8 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-        const GroupItem it = decode_group(gp, w, BM);
+      for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
+        const GroupItem it = decode_group(gp, work_at(gp, wi), BM);
         if (!it.active) continue;
         const uint32_t idesc = instr_desc(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -193,8 +204,8 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-      const GroupItem it = decode_group(gp, w, BM);
+    for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
+      const GroupItem it = decode_group(gp, work_at(gp, wi), BM);
         if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }

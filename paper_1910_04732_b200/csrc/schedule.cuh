@@ -1,0 +1,76 @@
+// Static tile schedule of a grouped GEMM launch.
+//
+// A grouped launch walks one work list (the tiles of all its problems) with a fixed set of
+// persistent units (CTAs, or CTA pairs).  Dealing the list out round-robin gives every unit the
+// same NUMBER of tiles, which is only balanced when the tiles cost the same.  The launches of the
+// gated factorized layer mix tiles of different length: in H' = X Q^T and dH' = dY P the FFN
+// matrices contract over 3072 features (48 k-blocks) next to attention matrices that contract
+// over 768 (12 k-blocks).  The host therefore assigns tiles to units with the longest-processing-time rule (sort by cost,
+// always hand the next tile to the least loaded unit) and passes the per-unit lists to the kernel
+// as a table in its parameter block; every role of a unit (TMA producer, MMA issuer, epilogue
+// warps, and both CTAs of a pair) walks the same list, so no run-time hand-over is needed.
+// Launches with more work items than the table holds keep the round-robin order (with that many
+// tiles per unit the imbalance is small anyway).
+#pragma once
+#include <stdint.h>
+
+#ifndef __CUDACC_RTC__
+#include <algorithm>
+#include <functional>
+#include <queue>
+#include <utility>
+#include <vector>
+#endif
+
+namespace flop {
+namespace tc {
+
+constexpr int kMaxSched = 2048;   // work items a table can hold
+constexpr int kMaxUnits = 148;    // persistent CTAs (one-CTA kernel) or pairs (two-CTA kernel)
+
+struct Schedule {
+  int n_units;                       // 0: no table, round-robin over the work list
+  uint16_t begin[kMaxUnits + 1];     // unit u walks item[begin[u] .. begin[u+1])
+  uint16_t item[kMaxSched];          // work-list indices
+};
+
+// Longest-processing-time assignment of `cost.size()` work items to `units` units.  Items of equal
+// cost keep their work-list order (neighbouring tiles share operand tiles in L2).  Returns the
+// largest unit load; `rr_makespan` receives the largest load of the round-robin deal for comparison.
+inline double build_schedule(const std::vector<double>& cost, int units, Schedule* out, double* rr_makespan) {
+  const int n = (int)cost.size();
+  out->n_units = 0;
+  if (rr_makespan) {
+    std::vector<double> load((size_t)std::max(units, 1), 0.0);
+    for (int i = 0; i < n; ++i) load[(size_t)(i % std::max(units, 1))] += cost[(size_t)i];
+    *rr_makespan = load.empty() ? 0.0 : *std::max_element(load.begin(), load.end());
+  }
+  if (n == 0 || n > kMaxSched || units <= 0 || units > kMaxUnits) return -1.0;
+  std::vector<int> order((size_t)n);
+  for (int i = 0; i < n; ++i) order[(size_t)i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost[(size_t)a] > cost[(size_t)b]; });
+  typedef std::pair<double, int> LoadUnit;   // least loaded first, ties to the lower unit index
+  std::priority_queue<LoadUnit, std::vector<LoadUnit>, std::greater<LoadUnit>> heap;
+  for (int u = 0; u < units; ++u) heap.push(LoadUnit(0.0, u));
+  std::vector<std::vector<int>> lists((size_t)units);
+  double makespan = 0.0;
+  for (int i = 0; i < n; ++i) {
+    LoadUnit lu = heap.top();
+    heap.pop();
+    lists[(size_t)lu.second].push_back(order[(size_t)i]);
+    lu.first += cost[(size_t)order[(size_t)i]];
+    makespan = std::max(makespan, lu.first);
+    heap.push(lu);
+  }
+  int pos = 0;
+  for (int u = 0; u < units; ++u) {
+    out->begin[u] = (uint16_t)pos;
+    for (int w : lists[(size_t)u]) out->item[pos++] = (uint16_t)w;
+  }
+  for (int u = units; u <= kMaxUnits; ++u) out->begin[u] = (uint16_t)pos;
+  out->n_units = units;
+  return makespan;
+}
+
+}  // namespace tc
+}  // namespace flop

@@ -12,6 +12,12 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
 
 
+def pytest_sessionstart(session):
+    """The tests call the library through its C ABI: build it in-tree when it is missing or older than its sources."""
+    from paper_1910_04732_b200 import build
+    build.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
