@@ -836,7 +836,7 @@ static int gate_sample_impl(const float* log_alpha, int64_t n, flop_hc_params_t 
   if (!log_alpha || !z) return FLOP_ERR_INVALID_ARG;
   GateConsts g;
   g.beta_d = (double)hc.beta; g.gamma_d = (double)hc.gamma; g.zeta_d = (double)hc.zeta;
-  g.inv_beta = (float)(1.0 / g.beta_d); g.gamma = hc.gamma; g.zeta = hc.zeta;
+  g.inv_beta = (float)(1.0 / g.beta_d); g.neg_inv_beta_log2e = (float)(-1.4426950408889634 / g.beta_d); g.gamma = hc.gamma; g.zeta = hc.zeta;
   g.c0 = (float)(g.beta_d * log(-g.gamma_d / g.zeta_d));
   g.c1 = (float)(g.beta_d * log((1.0 - g.gamma_d) / (g.zeta_d - 1.0)));
   const int vec_ok = aligned16(log_alpha) && aligned16(z) && (!dz_dla || aligned16(dz_dla)) &&
