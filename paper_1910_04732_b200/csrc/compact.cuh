@@ -183,4 +183,123 @@ gather_p_kernel(const T* __restrict__ P, int64_t ldp, const int32_t* __restrict_
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// P gather with the rows staged by bulk asynchronous copies (bf16, rows of a multiple of 16 bytes).
+//
+// A block walks groups of `rows_per_stage` consecutive rows of P.  One thread hands the rows of the
+// next groups to the copy engine (cp.async.bulk global -> shared, completion counted in bytes on an
+// mbarrier per buffer) while all threads pick the surviving columns of the current group out of
+// shared memory and write them as 8-byte pieces, so the read of P is fully coalesced, needs no
+// registers or load instructions, and overlaps the select/store phase of the same block.  The
+// index list is kept in shared memory as 16-bit entries (r <= 65536).  Waits are bounded: when one
+// gives up, the block records FLOP_ERR_TIMEOUT, lets the copies in flight land (bounded) and returns.
+namespace gp {
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// 16-byte aligned source and destination, size a multiple of 16 bytes
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+constexpr long long kWaitCycles = 2000000000LL;   // ~1 s
+}  // namespace gp
+
+constexpr int kGatherMaxBuf = 4;
+
+__global__ void __launch_bounds__(256)
+gather_p_pipe_kernel(const __nv_bfloat16* __restrict__ P, int64_t ldp, const int32_t* __restrict__ idx,
+                     const int32_t* __restrict__ k_dev, int r, int d_out, __nv_bfloat16* __restrict__ Pc, int64_t ldpc,
+                     int rows_per_stage, int nbuf) {
+  pdl_wait();
+  pdl_launch_dependents();
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  __shared__ int s_abort;
+  const int k = min(*k_dev, r);
+  if (k <= 0) return;
+  const uint32_t row_bytes = (uint32_t)r * 2u;                     // multiple of 16 (checked by the host)
+  const uint32_t stage_bytes = row_bytes * (uint32_t)rows_per_stage;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw);            // nbuf barriers (64 bytes reserved)
+  unsigned short* sidx = reinterpret_cast<unsigned short*>(smem_raw + 64);               // r entries
+  unsigned char* bufs = smem_raw + 64 + (((size_t)r * 2 + 127) & ~(size_t)127);          // nbuf stages
+  const int n_groups = (d_out + rows_per_stage - 1) / rows_per_stage;
+  const int n_mine = (int)blockIdx.x < n_groups ? (n_groups - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  if (n_mine == 0) return;
+
+  auto issue = [&](int it) {   // thread 0: hand the rows of this block's it-th group to the copy engine
+    const int b = it % nbuf;
+    const int row0 = ((int)blockIdx.x + it * (int)gridDim.x) * rows_per_stage;
+    const int rows = min(rows_per_stage, d_out - row0);
+    const uint32_t bar = gp::smem_addr(&bars[b]);
+    gp::bar_expect_tx(bar, row_bytes * (uint32_t)rows);
+    for (int j = 0; j < rows; ++j)
+      gp::bulk_load(gp::smem_addr(bufs + (size_t)b * stage_bytes + (size_t)j * row_bytes), P + (int64_t)(row0 + j) * ldp, row_bytes, bar);
+  };
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int b = 0; b < nbuf; ++b) gp::bar_init(gp::smem_addr(&bars[b]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (int it = 0; it < min(nbuf, n_mine); ++it) issue(it);
+  }
+  for (int c = threadIdx.x; c < k; c += blockDim.x) sidx[c] = (unsigned short)idx[c];
+  __syncthreads();
+
+  const int kq = (k + 3) >> 2;   // 4-column pieces per row
+  const bool vec_out = (reinterpret_cast<uintptr_t>(Pc) & 7) == 0 && (ldpc & 3) == 0;
+  int issued = min(nbuf, n_mine);
+  for (int it = 0; it < n_mine; ++it) {
+    const int b = it % nbuf;
+    const uint32_t parity = (uint32_t)(it / nbuf) & 1u;
+    const uint32_t bar = gp::smem_addr(&bars[b]);
+    if (!gp::bar_try_wait(bar, parity)) {
+      const long long t0 = clock64();
+      while (!gp::bar_try_wait(bar, parity)) {
+        if (*(volatile int*)&s_abort) break;
+        if (clock64() - t0 > gp::kWaitCycles) { *(volatile int*)&s_abort = 1; report_timeout(); break; }
+      }
+    }
+    if (__syncthreads_or(s_abort)) break;   // every thread takes the same decision
+    const int row0 = ((int)blockIdx.x + it * (int)gridDim.x) * rows_per_stage;
+    const int rows = min(rows_per_stage, d_out - row0);
+    const __nv_bfloat16* stage = reinterpret_cast<const __nv_bfloat16*>(bufs + (size_t)b * stage_bytes);
+    for (int w = threadIdx.x; w < rows * kq; w += blockDim.x) {
+      const int j = w / kq, c = (w - j * kq) << 2;
+      const __nv_bfloat16* row = stage + (size_t)j * r;
+      __nv_bfloat16* o = Pc + (int64_t)(row0 + j) * ldpc + c;
+      if (c + 3 < k && vec_out) {
+        const uint2 ii = *reinterpret_cast<const uint2*>(sidx + c);   // four 16-bit indices
+        const unsigned short q0 = __bfloat16_as_ushort(row[ii.x & 0xFFFFu]), q1 = __bfloat16_as_ushort(row[ii.x >> 16]);
+        const unsigned short q2 = __bfloat16_as_ushort(row[ii.y & 0xFFFFu]), q3 = __bfloat16_as_ushort(row[ii.y >> 16]);
+        __stcs(reinterpret_cast<uint2*>(o), make_uint2((uint32_t)q0 | ((uint32_t)q1 << 16), (uint32_t)q2 | ((uint32_t)q3 << 16)));
+      } else {
+        for (int e = c; e < min(c + 4, k); ++e) o[e - c] = row[sidx[e]];
+      }
+    }
+    __syncthreads();   // the buffer has been read by everyone: it may be refilled
+    if (threadIdx.x == 0 && issued < n_mine) issue(issued);
+    if (issued < n_mine) ++issued;
+  }
+  if (s_abort && threadIdx.x == 0) {
+    // leaving early: give the copies already issued time to land so that nothing writes this block's
+    // shared memory after it has gone
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) {}
+  }
+}
+
 }  // namespace flop

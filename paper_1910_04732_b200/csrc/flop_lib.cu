@@ -1510,7 +1510,33 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
     if (smem > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
     if (dt == FLOP_BF16) {
       if (d_in > 0) launch_k(gather_q_kernel<bf16>, dim3((unsigned)r), dim3(256), (size_t)(0), st, (const bf16*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (bf16*)Qc, ldqc, vq);
-      if (d_out > 0) {
+      // rows staged by bulk asynchronous copies when they are 16-byte pieces; FLOP_GATHER_PIPE=0 keeps the plain kernel
+      static const char* pipe_env = getenv("FLOP_GATHER_PIPE");
+      static const int pipe_on = pipe_env ? atoi(pipe_env) : 1;
+      if (d_out > 0 && pipe_on && vp && r % 8 == 0) {
+        const size_t row_bytes = (size_t)r * 2, idx_bytes = (row_bytes + 127) & ~(size_t)127;
+        int rows_per_stage = (int)std::max<size_t>(1, std::min<size_t>(16, (16 * 1024) / row_bytes));
+        int nbuf = kGatherMaxBuf;
+        auto need = [&](int nb) { return 64 + idx_bytes + (size_t)nb * rows_per_stage * row_bytes; };
+        while (nbuf > 2 && need(nbuf) > 100 * 1024) --nbuf;   // two blocks per SM where the rows allow it
+        if (need(nbuf) <= (size_t)kSmemBudget) {
+          const size_t sm = need(nbuf);
+          static size_t configured = 0;
+          if (sm > 48 * 1024 && sm > configured) {
+            FLOP_CUDA(cudaFuncSetAttribute(gather_p_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
+            configured = (size_t)kSmemBudget;
+          }
+          const int64_t groups = (d_out + rows_per_stage - 1) / rows_per_stage;
+          const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (size_t)(224 * 1024) / sm));
+          const int grid = (int)std::min<int64_t>(groups, (int64_t)num_sms() * per_sm);
+          launch_k(gather_p_pipe_kernel, dim3((unsigned)grid), dim3(256), sm, st, (const bf16*)P, ldp, idx, k_dev, (int)r, (int)d_out,
+                   (bf16*)Pc, ldpc, rows_per_stage, nbuf);
+        } else {
+          if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(gather_p_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+          launch_k(gather_p_kernel<bf16>, dim3((unsigned)((d_out + rows_per_block - 1) / rows_per_block)), dim3(256), (size_t)(smem), st,
+              (const bf16*)P, ldp, idx, k_dev, (int)r, (int)d_out, (bf16*)Pc, ldpc, rows_per_block, vp);
+        }
+      } else if (d_out > 0) {
         if (smem > 48 * 1024) FLOP_CUDA(cudaFuncSetAttribute(gather_p_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         launch_k(gather_p_kernel<bf16>, dim3((unsigned)((d_out + rows_per_block - 1) / rows_per_block)), dim3(256), (size_t)(smem), st, 
             (const bf16*)P, ldp, idx, k_dev, (int)r, (int)d_out, (bf16*)Pc, ldpc, rows_per_block, vp);

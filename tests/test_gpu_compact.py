@@ -104,3 +104,39 @@ def test_compact_fwd_with_no_survivors(b):
     Y = torch.full((5, 24), float("nan"), dtype=torch.bfloat16, device="cuda")
     b.compact_fwd(X, X[:0], torch.zeros(24, 8, dtype=torch.bfloat16, device="cuda")[:, :0], Y, 0, None)
     assert torch.count_nonzero(Y) == 0
+
+
+@pytest.mark.parametrize("r,d_out,d_in,keep", [
+    (1024, 40003, 16, 0.35),    # 8 rows per stage, more groups than buffers per block (buffers reused, parity flips), ragged last group
+    (16384, 1003, 8, 0.40),     # one 32 KB row per stage, two buffers
+    (64, 777, 24, 0.5),         # 16 rows per stage, tiny rows
+    (1024, 517, 8, 0.001),      # one or two survivors: the scalar tail of a row
+    (1032, 300, 8, 1.0),        # every component survives
+    (1020, 300, 8, 0.35),       # rows that are not 16-byte multiples: the plain kernel
+])
+def test_gather_of_survivors_is_exact(b, r, d_out, d_in, keep):
+    """P_c = P[:, idx] and Q_c = diag(z) Q[idx, :] for a supplied gate vector (mode 1): a pure gather on the P side,
+    compared element by element with the oracle's indexing; columns from k on stay untouched."""
+    g = np.random.default_rng(r + d_out)
+    z = np.where(g.random(r) < keep, g.uniform(0.05, 1.0, r), 0.0).astype(np.float32)
+    if keep < 0.01:
+        z[:] = 0.0
+        z[[5, r - 3]] = (0.25, 0.75)
+    P = g.standard_normal((d_out, r)).astype(np.float32)
+    Q = g.standard_normal((r, d_in)).astype(np.float32)
+    Pd, Qd = to_dev(P, "bf16"), to_dev(Q, "bf16")
+    Pb, Qb = host(Pd), host(Qd)                      # the bf16-rounded values both sides use
+    zt = torch.from_numpy(z).cuda()
+    idx = torch.full((r,), -1, dtype=torch.int32, device="cuda")
+    kd = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Pc, Qc = empty_dev(d_out, r, torch.bfloat16), empty_dev(r, d_in, torch.bfloat16)
+    b.compact_ranks(zt, 1, HC, idx, kd, None, Pd, Qd, Pc, Qc)
+    k = int(kd.item())
+    ko, idxo = O.active_ranks(z)
+    assert k == ko and np.array_equal(idx.cpu().numpy()[:k], idxo)
+    Pco, Qco = O.compact_ranks(Pb, Qb, idxo, z.astype(np.float64))
+    got = host(Pc)
+    assert np.array_equal(got[:, :k], Pco)
+    assert np.all(np.isnan(got[:, k:]))
+    assert rel_fro(host(Qc)[:k], Qco) < 4e-3
+    assert b.device_status() == b.OK
