@@ -108,9 +108,12 @@ l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__
       for (int i = 0; i < 4; ++i) a[i] = (j0 + i < hi) ? log_alpha[j0 + i] : 0.f;
     }
     if (!kGrad) {
+      // the four probabilities of a vector are added in fp32 (each is in (0, 1): the group sum is exact to
+      // 2^-22), the groups in fp64: a quarter of the fp64 conversions and additions, which bound this pass
+      float p4[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (j0 + i < hi) sum += (double)l0_pi(a[i], thr);
+      for (int i = 0; i < 4; ++i) p4[i] = (j0 + i < hi) ? l0_pi(a[i], thr) : 0.f;
+      sum += (double)((p4[0] + p4[1]) + (p4[2] + p4[3]));
     } else {
       float gsum[4];
 #pragma unroll

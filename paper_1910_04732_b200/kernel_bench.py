@@ -56,6 +56,7 @@ def timed(fn, iters=10, warmup=3, graph=False):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--small", action="store_true", help="sizes for a profiler capture (a few hundred MB)")
+    ap.add_argument("--only-membound", action="store_true", help="stop after the table of memory-bound kernels")
     args = ap.parse_args()
     build.build()
     b.load_library()
@@ -69,7 +70,7 @@ def main():
     g = torch.Generator(device="cuda"); g.manual_seed(0)
 
     # ---- gate sampler: 4 B read + 4 + 4 + 1 B written per gate
-    n = 1 << (24 if args.small else 26)
+    n = 1 << (25 if args.small else 26)
     la = torch.randn(n, generator=g, device="cuda") * 1.5 + 1.0
     z, d, m = torch.empty(n, device="cuda"), torch.empty(n, device="cuda"), torch.empty(n, dtype=torch.uint8, device="cuda")
     t = timed(lambda: b.gate_sample(la, HC, 0, 0, z, m, d))
@@ -89,7 +90,7 @@ def main():
     del z, d, m, dla
 
     # ---- rank compaction and gather, ~35 % of the components survive
-    r, d_in, d_out = (4096, 4096, 16384) if args.small else (16384, 16384, 65536)
+    r, d_in, d_out = (16384, 4096, 8192) if args.small else (16384, 16384, 65536)
     a = torch.where(torch.rand(r, generator=g, device="cuda") < 0.35, 4.0, -4.0) + 0.1 * torch.randn(r, generator=g, device="cuda")
     P = torch.randn(d_out, r, generator=g, device="cuda", dtype=torch.float32).bfloat16()
     Q = torch.randn(r, d_in, generator=g, device="cuda", dtype=torch.float32).bfloat16()
@@ -99,7 +100,7 @@ def main():
     t_all = timed(lambda: b.compact_ranks(a, 0, HC, idx, kd, zd, P, Q, Pc, Qc))
     k = int(kd.item())
     rows.append(("compact_select_kernel", f"r = {r}", 4 * r * 6, t_sel))
-    rows.append(("gather_p_kernel + gather_q_kernel", f"r = {r}, d_in = {d_in}, d_out = {d_out}, k = {k}",
+    rows.append(("gather_p_pipe_kernel + gather_q_kernel", f"r = {r}, d_in = {d_in}, d_out = {d_out}, k = {k}",
                  2 * d_out * r + 2 * k * d_out + 4 * k * d_in + 4 * r, t_all - t_sel))
     del P, Q, Pc, Qc
 
@@ -107,6 +108,9 @@ def main():
     print(f"{'kernel(s)':44s} {'size':58s} {'MB':>9s} {'us':>9s} {'GB/s':>8s} {'of peak':>8s}")
     for name, what, nbytes, t in rows:
         print(f"{name:44s} {what:58s} {nbytes / 1e6:9.1f} {t * 1e6:9.1f} {nbytes / t / 1e9:8.0f} {nbytes / t / 1e9 / peak:8.2f}")
+
+    if args.only_membound:
+        return
 
     # ---- pruned inference: d_in = 1024, d_out = 4096, r = 1024, ~35 % survive
     w = I.WORKLOADS["infer"]
