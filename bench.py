@@ -167,6 +167,13 @@ class Job:
                                                      self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
                                                      self.dlog_alpha[e["lo"]:e["hi"]], e["ws"]) for e in chunk])
                 self.groups.append((fwd, bwd))
+        # data parallelism: one gradient bucket per grouped call (a layer), reduced while later layers compute
+        n_per = group if group > 0 else len(self.mats)
+        sizes_w = [e["dP"].shape[0] * r8(e["m"].r) + e["m"].r * r8(e["m"].d_in) for e in self.mats]
+        self.bucket_bounds = [0]
+        for i in range(0, len(sizes_w), n_per):
+            self.bucket_bounds.append(self.bucket_bounds[-1] + sum(sizes_w[i:i + n_per]))
+        self.reducer = None
         self.ws_l0 = b.alloc_workspace(b.workspace_bytes(b.OP_L0, self.n_gates, 0, 0, len(sizes), b.F32), device)
         self.offset_dev = torch.zeros(1, dtype=torch.int64, device=device)
         self.graph = None
@@ -235,15 +242,24 @@ class Job:
                                       self.out4, None, self.dlog_alpha, self.ws_l0)
         if self.world > 1:
             from paper_1910_04732_b200 import dp
-            dp.allreduce_gradients([self.wgrad, self.dlog_alpha])     # the one exchange step of the path
+            if self.reducer is not None and self.reducer.pending:
+                dp.allreduce_gradients([self.dlog_alpha])
+                self.reducer.wait()                                   # the layer buckets started during the step
+            else:
+                dp.allreduce_gradients([self.wgrad, self.dlog_alpha])     # the one exchange step of the path
 
     def step(self):
         torch = self.torch
         self.sample_gates()
         if self.group > 0:
-            for fwd, bwd in self.groups:
+            if self.world > 1 and self.reducer is None:
+                from paper_1910_04732_b200 import dp
+                self.reducer = dp.BucketedReducer(self.wgrad, self.bucket_bounds)
+            for i, (fwd, bwd) in enumerate(self.groups):
                 self.b.gated_lowrank_fwd_grouped(fwd)
                 self.b.gated_lowrank_bwd_grouped(bwd)
+                if self.reducer is not None:
+                    self.reducer.launch(i)                            # this layer's dP, dQ are final
         elif self.n_streams == 1:
             for e in self.mats:
                 self.run_matrix(e)

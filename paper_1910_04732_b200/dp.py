@@ -33,3 +33,35 @@ def allreduce_gradients(flat_buffers: Iterable[torch.Tensor], group=None) -> Non
         return
     for buf in flat_buffers:
         dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
+
+
+class BucketedReducer:
+    """Sums one flat gradient buffer over all ranks bucket by bucket, each bucket as soon as it is final.
+
+    The weight gradients of all matrices live in one flat buffer, layer after layer.  `launch(i)` starts the
+    all-reduce of bucket i (asynchronously: with NCCL it runs on the communicator's own stream, ordered after the
+    work already queued on the current stream) so that it overlaps the GEMMs of the layers still to come;
+    `wait()` makes the current stream wait for every bucket started since the last `wait()`.  At BERT sizes a
+    layer's bucket is 21 MB of bf16 against a backward pass of about 180 us per layer.
+    """
+
+    def __init__(self, flat: torch.Tensor, bounds, group=None):
+        self.flat, self.group = flat, group
+        self.bounds = [int(b) for b in bounds]
+        if self.bounds[0] != 0 or self.bounds[-1] != flat.numel() or any(a > b for a, b in zip(self.bounds, self.bounds[1:])):
+            raise ValueError("bucket bounds must run from 0 to flat.numel() without going back")
+        self.pending = []
+        self.active = dist.is_initialized() and dist.get_world_size(group) > 1
+
+    def n_buckets(self) -> int:
+        return len(self.bounds) - 1
+
+    def launch(self, i: int) -> None:
+        lo, hi = self.bounds[i], self.bounds[i + 1]
+        if self.active and hi > lo:
+            self.pending.append(dist.all_reduce(self.flat[lo:hi], op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+
+    def wait(self) -> None:
+        for work in self.pending:
+            work.wait()
+        self.pending = []

@@ -56,3 +56,42 @@ def test_token_shard_covers_every_token_once():
             assert s0 + c0 == s1
         assert max(c for _, c in spans) - min(c for _, c in spans) <= 1
     assert dp.gate_stream(3) == dp.gate_stream(3) and dp.gate_stream(3) != dp.gate_stream(4)
+
+
+def _bucket_worker(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    g = torch.Generator().manual_seed(100 + rank)
+    flat = torch.randn(1000, generator=g, dtype=torch.float64)
+    mine = flat.clone()
+    red = dp.BucketedReducer(flat, [0, 10, 10, 377, 1000])           # four buckets, one of them empty
+    for i in reversed(range(red.n_buckets())):                       # backward order, as the layers finish
+        red.launch(i)
+    red.wait()
+    parts = [torch.zeros(1000, dtype=torch.float64) for _ in range(world)]
+    dist.all_gather(parts, mine)
+    if rank == 0:
+        ok = torch.allclose(flat, sum(parts), rtol=0, atol=1e-12) and red.pending == []
+        with open(out, "w") as f:
+            f.write("ok" if ok else "mismatch")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_bucketed_reducer_sums_every_bucket(tmp_path):
+    out = str(tmp_path / "bucket.txt")
+    port = 31500 + (os.getpid() % 2000)
+    mp.spawn(_bucket_worker, args=(2, port, out), nprocs=2, join=True)
+    assert open(out).read() == "ok"
+
+
+def test_bucketed_reducer_checks_bounds_and_is_a_no_op_alone():
+    import pytest
+    flat = torch.ones(8)
+    for bad in ([1, 8], [0, 7], [0, 5, 3, 8]):
+        with pytest.raises(ValueError):
+            dp.BucketedReducer(flat, bad)
+    red = dp.BucketedReducer(flat, [0, 4, 8])       # no process group: nothing to exchange
+    red.launch(0); red.launch(1); red.wait()
+    assert torch.equal(flat, torch.ones(8))
