@@ -226,7 +226,7 @@ gather_p_pipe_kernel(const __nv_bfloat16* __restrict__ P, int64_t ldp, const int
                      int rows_per_stage, int nbuf) {
   pdl_wait();
   pdl_launch_dependents();
-  extern __shared__ __align__(128) unsigned char smem_raw[];
+  extern __shared__ __align__(16) unsigned char smem_raw[];   // every offset used below is a multiple of 16
   __shared__ int s_abort;
   const int k = min(*k_dev, r);
   if (k <= 0) return;

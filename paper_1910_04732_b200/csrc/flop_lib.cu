@@ -306,7 +306,7 @@ int launch_group_inst(const tc::GroupParams& gp, int cta2, double flops, cudaStr
       const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes(gp.bn_max);
       launch_k(kern1, dim3(gp.sched.n_units ? gp.sched.n_units : std::min(gp.total_work, num_sms())), dim3(tc::kThreads), (size_t)smem, st, gp);
     } else {
-      const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes2(gp.bn_max, gp.fused);
+      const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes2(gp.bn_max);
       const int pairs = gp.sched.n_units ? gp.sched.n_units : std::min(gp.total_work, num_sms() / 2);
       cudaLaunchConfig_t cfg{};
       cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
@@ -353,13 +353,6 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
       p.wg_out = j.ep.wg_out; p.wg_f32 = j.ep.wg_f32; p.row_scale = j.ep.row_scale; p.accumulate = j.ep.accumulate;
       p.dyn_m = j.dyn_m; p.dyn_n = j.dyn_n; p.dyn_k = j.dyn_k;
-      // CTA pairs with 256-wide tiles take two neighbouring N tiles per work item: the A k-block is fetched once
-      // for both, which brings the bytes an SM pulls from L2 per MMA cycle under what the L2 fabric delivers
-      // (FLOP_FUSE_N=0 switches it off, for comparison)
-      static const char* fuse_env = getenv("FLOP_FUSE_N");
-      static const int fuse_on = fuse_env ? atoi(fuse_env) : 1;
-      p.fuse_n = (fuse_on && j.pl.cta2 && p.bn == 256 && p.tiles_n >= 2) ? 1 : 0;
-      if (p.fuse_n) gp.fused = 1;
       // bf16 tiles that are plainly overwritten leave through a TMA store (64 x 32 boxes of the output)
       void* tma_dst = j.ep.kind == tc::EPI_STORE ? (void*)j.ep.out
                       : (j.ep.kind == tc::EPI_WGRAD && !j.ep.wg_f32 && !j.ep.accumulate) ? j.ep.wg_out : nullptr;
@@ -367,20 +360,14 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       p.tma_store = (tma_dst && !no_tma_store) ? 1 : 0;
       if (p.tma_store) FLOP_TRY(make_tmap(&pr.tout, tma_dst, j.M, j.N, j.ep.ldo, 64, 32));
       pr.work_begin = gp.total_work;
-      const int tn_items = tc::items_n(p.tiles_n, p.fuse_n);
-      gp.total_work += p.tiles_m * tn_items * p.splits;
+      gp.total_work += p.tiles_m * p.tiles_n * p.splits;
       {   // cost of each work item of this problem in SM cycles (the model of plan_group), for the schedule
         const double bytes = j.pl.cta2 ? (double)tc::stage_bytes2(p.bn) : (double)tc::stage_bytes(p.bn);
         const double per_kb = std::max(2.0 * p.bn, bytes / 50.0), epi = 400.0 + 4.0 * p.bn;
-        const double per_kb2 = std::max(4.0 * p.bn, (double)tc::stage_bytes2(p.bn, 1) / 50.0);   // two N tiles, one A block
         if (item_cost.size() <= (size_t)tc::kMaxSched)
           for (int sp = 0; sp < p.splits; ++sp) {
             const int kbs = std::min(p.kb_per_split, p.num_kb - sp * p.kb_per_split);
-            for (int tm = 0; tm < p.tiles_m; ++tm)
-              for (int ti = 0; ti < tn_items; ++ti) {
-                const bool two = p.fuse_n && 2 * ti + 1 < p.tiles_n;
-                item_cost.push_back(two ? kbs * per_kb2 + 2.0 * epi : kbs * per_kb + epi);
-              }
+            item_cost.insert(item_cost.end(), (size_t)p.tiles_m * p.tiles_n, kbs * per_kb + epi);
           }
       }
       gp.bn_max = std::max(gp.bn_max, p.bn);
@@ -390,7 +377,7 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     if (gp.n == 0) continue;
     const int cta2 = first.pl.cta2;
     gp.stages = std::min(tc::kMaxStages, (kSmemBudget - kSmemFixed) /
-                                             (int)(cta2 ? tc::stage_bytes2(gp.bn_max, gp.fused) : tc::stage_bytes(gp.bn_max)));
+                                             (int)(cta2 ? tc::stage_bytes2(gp.bn_max) : tc::stage_bytes(gp.bn_max)));
     gp.stamp = nullptr;
     if (g_stamps.buf && g_stamps.used < g_stamps.capacity) {
       gp.stamp = g_stamps.buf + 2 * g_stamps.used++;

@@ -64,10 +64,6 @@ struct Params {
   // the N extent is rounded up to 64, so operands must be zero between the effective size and the next
   // multiple of 64.  An effective size of 0 is treated as 1 (an all-zero block).
   const int* dyn_m; const int* dyn_n; const int* dyn_k;
-  // 1: a work item covers TWO neighbouring N tiles (tn, tn + 1) of one M tile (the last item of a row of
-  // an odd tile count covers one).  The CTA-pair kernel loads the A k-block once for both and keeps one
-  // accumulator buffer per tile (see gemm2_group_kernel); the one-CTA kernel never sets it.
-  int fuse_n;
 };
 
 enum { EPI_STORE = 0, EPI_SLICE = 1, EPI_WGRAD = 2 };
@@ -190,18 +186,14 @@ __host__ __device__ inline uint32_t stage_bytes(int bn) { return kATileBytes + (
 // shared memory after the stage ring: the epilogue warps' staging tiles, then the barriers
 constexpr uint32_t kStoreBufTotal = kEpiWarps * kStoreBufBytes;
 
-struct WorkItem { int tm, tn, split, kb0, kb1; bool two; };
-__host__ __device__ inline int items_n(int tiles_n, int fuse_n) { return fuse_n ? (tiles_n + 1) >> 1 : tiles_n; }
+struct WorkItem { int tm, tn, split, kb0, kb1; };
 __device__ __forceinline__ WorkItem decode(const Params& p, int w) {
   WorkItem it;
-  const int tn_items = items_n(p.tiles_n, p.fuse_n);
-  const int tiles = p.tiles_m * tn_items;
+  const int tiles = p.tiles_m * p.tiles_n;
   it.split = w / tiles;
   const int t = w - it.split * tiles;
-  it.tm = t / tn_items;
-  const int ti = t - it.tm * tn_items;
-  it.tn = p.fuse_n ? 2 * ti : ti;
-  it.two = p.fuse_n && it.tn + 1 < p.tiles_n;
+  it.tm = t / p.tiles_n;
+  it.tn = t - it.tm * p.tiles_n;
   it.kb0 = it.split * p.kb_per_split;
   it.kb1 = min(it.kb0 + p.kb_per_split, p.num_kb);
   return it;

@@ -98,11 +98,8 @@ __device__ __forceinline__ uint32_t instr_desc2(bool a_mn, bool b_mn, int n) {
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM2 >> 4) << 24);
 }
 
-// bytes one CTA of the pair loads per stage: its 128 rows of A and half of the B tile; with two N tiles
-// per work item (fused) the halves of both B tiles
-__host__ __device__ inline uint32_t stage_bytes2(int bn, int fused = 0) {
-  return kATileBytes + (uint32_t)(bn / 2) * BK * 2 * (fused ? 2u : 1u);
-}
+// bytes one CTA of the pair loads per stage: its 128 rows of A and half of the B tile
+__host__ __device__ inline uint32_t stage_bytes2(int bn) { return kATileBytes + (uint32_t)(bn / 2) * BK * 2; }
 
 }  // namespace tc
 }  // namespace flop

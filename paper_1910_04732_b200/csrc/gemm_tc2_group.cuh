@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sbytes = stage_bytes2(gp.bn_max, gp.fused);
+  const uint32_t sbytes = stage_bytes2(gp.bn_max);
   const uint32_t store_base = smem_base + (uint32_t)gp.stages * sbytes;   // 1024-byte aligned: stages are multiples of 1 KB
   const uint32_t bar_base = store_base + kStoreBufTotal;
   auto full_bar = [&](int s) { return bar_base + 8u * (uint32_t)s; };
@@ -67,10 +67,9 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
         if (!it.active) continue;
         const GroupProblem& pr = gp.prob[it.g];
         const int half_n = pr.p.bn >> 1;
-        const uint32_t half_bytes = (uint32_t)half_n * BK * 2;
-        const int nb = it.two ? 2 : 1;                       // B tiles of this work item
-        const uint32_t tx = kATileBytes + half_bytes * (uint32_t)nb;
+        const uint32_t tx = kATileBytes + (uint32_t)half_n * BK * 2;
         const int m_base = it.tm * BM2 + (int)rank * BM;
+        const int n_base = it.tn * pr.p.bn + (int)rank * half_n;
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait2(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t sa = smem_base + (uint32_t)stage * sbytes, sb = sa + kATileBytes;
@@ -83,15 +82,11 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
             for (int i = 0; i < BM / (int)kBoxMN; ++i)
               tma_load_2d_pair(sa + i * kBoxBytes, &pr.ta, m_base + i * (int)kBoxMN, kb * BK, fb);
           }
-          for (int j = 0; j < nb; ++j) {
-            const int n_base = (it.tn + j) * pr.p.bn + (int)rank * half_n;
-            const uint32_t sbj = sb + (uint32_t)j * half_bytes;
-            if (!B_MN) {
-              tma_load_2d_pair(sbj, &pr.tb, kb * BK, n_base, fb);
-            } else {
-              for (int i = 0; i < half_n / (int)kBoxMN; ++i)
-                tma_load_2d_pair(sbj + i * kBoxBytes, &pr.tb, n_base + i * (int)kBoxMN, kb * BK, fb);
-            }
+          if (!B_MN) {
+            tma_load_2d_pair(sb, &pr.tb, kb * BK, n_base, fb);
+          } else {
+            for (int i = 0; i < half_n / (int)kBoxMN; ++i)
+              tma_load_2d_pair(sb + i * kBoxBytes, &pr.tb, n_base + i * (int)kBoxMN, kb * BK, fb);
           }
           if (++stage == gp.stages) { stage = 0; phase ^= 1u; }
         }
@@ -115,15 +110,9 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
         const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
         if (!it.active) continue;
         const uint32_t idesc = instr_desc2(A_MN, B_MN, gp.prob[it.g].p.bn);
-        const uint32_t half_bytes = (uint32_t)(gp.prob[it.g].p.bn >> 1) * BK * 2;
         if (!mbar_wait2(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
-        // a fused item accumulates its second tile in the other buffer (whose phase has flipped if acc wraps)
-        const int acc2 = acc ^ 1;
-        const uint32_t acc2_phase = acc == 1 ? acc_phase ^ 1u : acc_phase;
-        if (it.two && !mbar_wait2(tempty_bar(acc2), acc2_phase ^ 1u, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * gp.bn_max);
-        const uint32_t d_tmem2 = tmem_base + (uint32_t)(acc2 * gp.bn_max);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait2(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tcgen05_fence_after();
@@ -133,10 +122,6 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
             const uint64_t ad = smem_desc(sa + (A_MN ? k * (UMMA_K * 128) : k * (UMMA_K * 2)), A_MN);
             const uint64_t bd = smem_desc(sb + (B_MN ? k * (UMMA_K * 128) : k * (UMMA_K * 2)), B_MN);
             umma2_bf16(d_tmem, ad, bd, idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
-            if (it.two) {
-              const uint64_t bd2 = smem_desc(sb + half_bytes + (B_MN ? k * (UMMA_K * 128) : k * (UMMA_K * 2)), B_MN);
-              umma2_bf16(d_tmem2, ad, bd2, idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
-            }
           }
           umma2_commit_mc(empty_bar(stage), 3);    // frees the stage in both CTAs
           if (++stage == gp.stages) { stage = 0; phase ^= 1u; }
@@ -144,10 +129,6 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
         if (!ok) break;
         umma2_commit_mc(tfull_bar(acc), 3);        // accumulator halves complete in both CTAs
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-        if (it.two) {
-          umma2_commit_mc(tfull_bar(acc), 3);
-          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-        }
       }
     }
   } else {
@@ -159,16 +140,13 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
         if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
-      for (int j = 0; j < (it.two ? 2 : 1) && ok; ++j) {   // the tiles of a fused item are drained one after the other
-        if (!mbar_wait2(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tcgen05_fence_after();
-        const int tn = it.tn + j;
-        run_epilogue<EPI, true>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM2 + (int)rank * BM, tn * p.bn, it.n_limit, it.split, tn,
-                                warp, lane, map_to_cta(tempty_bar(acc), 0));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-      }
+      if (!mbar_wait2(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tcgen05_fence_after();
+      run_epilogue<EPI, true>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.n_limit, it.split, it.tn,
+                              warp, lane, map_to_cta(tempty_bar(acc), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
     if (lane == 0) tma_store_wait_all();
   }

@@ -41,7 +41,6 @@ struct GroupParams {
   unsigned long long* stamp;
   // Which work items each persistent unit walks (schedule.cuh); n_units == 0: round-robin.
   Schedule sched;
-  int fused;   // some problem has fuse_n set: stages hold the A block and two B half-tiles (CTA-pair kernel only)
 };
 
 // The work items of persistent unit `unit` of `nunits`: for (i = first; i < last; i += step) item = work_at(gp, i).
@@ -58,7 +57,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 
-struct GroupItem { int g, tm, tn, split, kb0, kb1, n_limit; bool active, two; };
+struct GroupItem { int g, tm, tn, split, kb0, kb1, n_limit; bool active; };
 
 // Work item w of the group; bm = rows of D per tile (128, or 256 for a CTA pair).  When a problem
 // carries device-side sizes the item may lie outside the effective extent (active = false: every
@@ -70,7 +69,7 @@ __device__ __forceinline__ GroupItem decode_group(const GroupParams& gp, int w, 
     if (i < gp.n && w >= gp.prob[i].work_begin) g = i;
   const Params& p = gp.prob[g].p;
   const WorkItem it = decode(p, w - gp.prob[g].work_begin);
-  GroupItem o{g, it.tm, it.tn, it.split, it.kb0, it.kb1, p.N, true, it.two};
+  GroupItem o{g, it.tm, it.tn, it.split, it.kb0, it.kb1, p.N, true};
   if (p.dyn_m || p.dyn_n || p.dyn_k) {
     const int m_eff = p.dyn_m ? max(1, min(p.M, __ldg(p.dyn_m))) : p.M;
     const int n_eff = p.dyn_n ? max(1, min(p.N, __ldg(p.dyn_n))) : p.N;
@@ -78,7 +77,6 @@ __device__ __forceinline__ GroupItem decode_group(const GroupParams& gp, int w, 
     if (p.dyn_n) o.n_limit = min(p.N, (n_eff + 63) & ~63);
     o.kb1 = min(o.kb1, (k_eff + BK - 1) / BK);
     o.active = o.tm * bm < m_eff && o.tn * p.bn < n_eff && o.kb0 < o.kb1;
-    o.two = o.two && (o.tn + 1) * p.bn < n_eff;
   }
   return o;
 }
