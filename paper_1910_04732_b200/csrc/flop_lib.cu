@@ -23,6 +23,7 @@
 #include "gemm_tc2.cuh"
 #include "gemm_tc_group.cuh"
 #include "gemm_tc2_group.cuh"
+#include "gemm_tc2_dual.cuh"
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
 #include "active_ranks.cuh"
@@ -325,6 +326,35 @@ int launch_group_inst(const tc::GroupParams& gp, int cta2, double flops, cudaStr
   return FLOP_OK;
 }
 
+// A launch whose problems are of two kinds: bf16 stores with (K-major A, MN-major B) and in-place weight
+// gradients with both operands MN-major (the two steps of the grouped backward pass).  CTA pairs only.
+int launch_dual_inst(const tc::GroupParams& gp, double flops, cudaStream_t st) {
+  static bool configured = false;
+  auto kern = tc::gemm2_dual_kernel<false, true, tc::EPI_STORE, true, true, tc::EPI_WGRAD>;
+  if (!configured) {
+    FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    configured = true;
+  }
+  {
+    GemmTimer timer(st, flops);
+    const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes2(gp.bn_max);
+    const int pairs = gp.sched.n_units ? gp.sched.n_units : std::min(gp.total_work, num_sms() / 2);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_on() ? 2 : 1;
+    cudaLaunchKernelEx(&cfg, kern, gp);
+  }
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
 int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
   size_t i = 0;
   while (i < jobs.size()) {
@@ -332,14 +362,19 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     memset(&gp, 0, sizeof(gp));
     double flops = 0.0;
     const TcJob& first = jobs[i];
+    bool uniform = true, dual_ok = true;   // one kind of problem / the two kinds gemm2_dual_kernel is built for
     std::vector<double> item_cost;
     for (; i < jobs.size() && gp.n < tc::kMaxGroup; ++i) {
       const TcJob& j = jobs[i];
       if (j.M <= 0 || j.N <= 0 || j.K <= 0) continue;
       if (j.M > INT32_MAX || j.N > INT32_MAX || j.K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
       if (j.pl.cta2 != first.pl.cta2) return FLOP_ERR_INVALID_ARG;
-      if (j.A.mn_major != first.A.mn_major || j.B.mn_major != first.B.mn_major || j.ep.kind != first.ep.kind) return FLOP_ERR_INVALID_ARG;
+      if (j.A.mn_major != first.A.mn_major || j.B.mn_major != first.B.mn_major || j.ep.kind != first.ep.kind) uniform = false;
+      const bool kind0 = !j.A.mn_major && j.B.mn_major && j.ep.kind == tc::EPI_STORE;
+      const bool kind1 = j.A.mn_major && j.B.mn_major && j.ep.kind == tc::EPI_WGRAD;
+      if (!(kind0 || kind1) || !j.pl.cta2) dual_ok = false;
       tc::GroupProblem& pr = gp.prob[gp.n];
+      pr.p.kind = kind1 ? 1 : 0;
       if (!j.A.mn_major) FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.M, j.K, j.A.ld, tc::BK, tc::BM));
       else               FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.K, j.M, j.A.ld, tc::kBoxMN, tc::BK));
       if (!j.B.mn_major) FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.N, j.K, j.B.ld, tc::BK, (uint32_t)(j.pl.cta2 ? j.pl.bn / 2 : j.pl.bn)));
@@ -398,7 +433,8 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     }
     const bool a_mn = first.A.mn_major, b_mn = first.B.mn_major;
     int rc = FLOP_ERR_UNSUPPORTED;
-    if (!a_mn && !b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, false, tc::EPI_STORE>(gp, cta2, flops, st);
+    if (!uniform) rc = dual_ok ? launch_dual_inst(gp, flops, st) : FLOP_ERR_INVALID_ARG;
+    else if (!a_mn && !b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, false, tc::EPI_STORE>(gp, cta2, flops, st);
     else if (!a_mn && b_mn && first.ep.kind == tc::EPI_STORE) rc = launch_group_inst<false, true, tc::EPI_STORE>(gp, cta2, flops, st);
     else if (a_mn && b_mn && first.ep.kind == tc::EPI_SLICE) rc = launch_group_inst<true, true, tc::EPI_SLICE>(gp, cta2, flops, st);
     else if (a_mn && b_mn && first.ep.kind == tc::EPI_WGRAD) rc = launch_group_inst<true, true, tc::EPI_WGRAD>(gp, cta2, flops, st);
@@ -1228,6 +1264,46 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
       g6.push_back(j6);
     }
   }
+  auto run_finish = [&](const std::vector<BwdFinishArgs>& list) -> int {
+    for (size_t i = 0; i < list.size(); i += kFinishGroup) {
+      BwdFinishGroup g;
+      memset(&g, 0, sizeof(g));
+      for (; g.n < kFinishGroup && i + g.n < list.size(); ++g.n) {
+        g.a[g.n] = list[i + g.n];
+        g.unit_begin[g.n + 1] = g.unit_begin[g.n] + bwd_finish_units(g.a[g.n]);
+      }
+      const int64_t units = g.unit_begin[g.n];
+      if (units > 0) {
+        const int grid = (int)std::min<int64_t>((units + 255) / 256, (int64_t)num_sms() * 8);
+        if (wgrad_dt == FLOP_BF16) launch_k(bwd_finish_group_kernel<bf16>, dim3(grid), dim3(256), (size_t)0, st, g);
+        else                       launch_k(bwd_finish_group_kernel<float>, dim3(grid), dim3(256), (size_t)0, st, g);
+        count_launch();
+        FLOP_CUDA(cudaGetLastError());
+      }
+    }
+    return FLOP_OK;
+  };
+  // Two balanced launches instead of three uneven ones (gemm_tc2_dual.cuh): the products that need only saved
+  // tensors (dH' = dY P and dP = dY^T H') share the first work list, those that need dH' (dQ with the fused
+  // <Q, .> row dots, and dX) the second.  diag(z) Q depends on nothing computed here and is formed first; the
+  // ordered second stage of dlog_alpha comes last.  FLOP_STAGE_MERGE=0 keeps the three-launch order.
+  static const char* merge_env = getenv("FLOP_STAGE_MERGE");
+  static const int merge_on = merge_env ? atoi(merge_env) : 1;
+  const bool pairs_everywhere = !g3.empty() && g3[0].pl.cta2 && (g4.empty() || g4[0].pl.cta2) && (g5.empty() || g5[0].pl.cta2) &&
+                                (g6.empty() || g6[0].pl.cta2);
+  if (direct && merge_on && pairs_everywhere && g3.size() + g4.size() <= (size_t)tc::kMaxGroup &&
+      g5.size() + g6.size() <= (size_t)tc::kMaxGroup) {
+    std::vector<BwdFinishArgs> pre = fin, post = fin;
+    for (auto& f : pre) f.dlog_alpha = nullptr;
+    for (auto& f : post) f.Qz = nullptr;
+    FLOP_TRY(run_finish(pre));
+    g3.insert(g3.end(), g4.begin(), g4.end());
+    FLOP_TRY(launch_tc_group(g3, st));
+    g5.insert(g5.end(), g6.begin(), g6.end());
+    FLOP_TRY(launch_tc_group(g5, st));
+    FLOP_TRY(run_finish(post));
+    return FLOP_OK;
+  }
   if (direct) {   // both weight-gradient products of every matrix in one work list
     g4.insert(g4.end(), g5.begin(), g5.end());
     g5.clear();
@@ -1235,22 +1311,7 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
   FLOP_TRY(launch_tc_group(g3, st));   // dH' = dY P
   FLOP_TRY(launch_tc_group(g4, st));   // dY^T H' slices
   FLOP_TRY(launch_tc_group(g5, st));   // dH'^T X slices + fused <Q, .> row dots
-  for (size_t i = 0; i < fin.size(); i += kFinishGroup) {
-    BwdFinishGroup g;
-    memset(&g, 0, sizeof(g));
-    for (; g.n < kFinishGroup && i + g.n < fin.size(); ++g.n) {
-      g.a[g.n] = fin[i + g.n];
-      g.unit_begin[g.n + 1] = g.unit_begin[g.n] + bwd_finish_units(g.a[g.n]);
-    }
-    const int64_t units = g.unit_begin[g.n];
-    if (units > 0) {
-      const int grid = (int)std::min<int64_t>((units + 255) / 256, (int64_t)num_sms() * 8);
-      if (wgrad_dt == FLOP_BF16) launch_k(bwd_finish_group_kernel<bf16>, dim3(grid), dim3(256), (size_t)0, st, g);
-      else                       launch_k(bwd_finish_group_kernel<float>, dim3(grid), dim3(256), (size_t)0, st, g);
-      count_launch();
-      FLOP_CUDA(cudaGetLastError());
-    }
-  }
+  FLOP_TRY(run_finish(fin));
   FLOP_TRY(launch_tc_group(g6, st));   // dX = dH' (diag(z) Q)
   return FLOP_OK;
 }

@@ -64,6 +64,7 @@ struct Params {
   // the N extent is rounded up to 64, so operands must be zero between the effective size and the next
   // multiple of 64.  An effective size of 0 is treated as 1 (an all-zero block).
   const int* dyn_m; const int* dyn_n; const int* dyn_k;
+  int kind;   // 0 or 1: which of the two compile-time configurations of gemm2_dual_kernel serves this problem
 };
 
 enum { EPI_STORE = 0, EPI_SLICE = 1, EPI_WGRAD = 2 };
