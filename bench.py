@@ -4,7 +4,7 @@
 One step = one pass of the whole hot path over one batch of synthetic input:
 sample every gate of every layer (one launch), then for every factorized matrix
 of every layer the gated forward (2 GEMMs) and backward (4 GEMMs + the fused
-dlog_alpha reduction), then the expected-L0 / Lagrangian term over all gates.
+dlog_alpha reduction; grouped per layer into two forward and two backward launches), then the expected-L0 / Lagrangian term over all gates.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload bert|sru|txl] [--impl ours|reference]
 
@@ -546,7 +546,7 @@ def main():
     gemm_tflops = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     # dram__bytes_read.sum + dram__bytes_write.sum of the GEMM launches of one bert layer, from the ncu capture
     # summarised under profiles/ (grouped calls of six matrices): mean per launch
-    traffic = 100.9e6 if (w.name == "bert" and group == 6) else None
+    traffic = 118.6e6 if (w.name == "bert" and group == 6) else None
     line = {
         "metric": METRIC, "value": tokens_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
@@ -560,9 +560,9 @@ def main():
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": peaks["bf16_tflops_sustained"],
                      "unit": "TFLOP/s", "frac": gemm_tflops / peaks["bf16_tflops_sustained"], "traffic": traffic,
-                     "traffic_note": "DRAM read+write bytes per GEMM launch, mean of the five launches of one layer (ncu capture in profiles/)" if traffic else None,
+                     "traffic_note": "DRAM read+write bytes per GEMM launch, mean of the four launches of one layer (ncu capture in profiles/)" if traffic else None,
                      "peak_kind": f"{peak_kind} (sustained; burst {peaks['bf16_tflops']})",
-                     "kernel": "tc::gemm_group_kernel / tc::gemm2_group_kernel (every GEMM stage of the step)",
+                     "kernel": "tc::gemm2_group_kernel (forward) / tc::gemm2_dual_kernel (backward): every GEMM launch of the step",
                      "launches_per_step": gemm_launches // args.steps,
                      "kernel_ms_per_step": gemm_ms / args.steps, "step_ms_in_timed_pass": ms_timed_pass / args.steps,
                      "frac_of_nominal": gemm_tflops / NOMINAL_BF16_TFLOPS,
