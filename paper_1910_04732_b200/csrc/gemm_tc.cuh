@@ -1,7 +1,8 @@
 // bf16 tensor-core GEMM for sm_100a, shared pieces: D[M,N] = sum_k A(m,k) B(n,k), fp32 accumulate.
 //
 // The kernels built from this header (gemm_group_kernel in gemm_tc_group.cuh, one CTA per
-// 128 x BN tile, and gemm2_group_kernel in gemm_tc2_group.cuh, a CTA pair per 256 x BN tile)
+// 128 x BN tile; gemm2_group_kernel in gemm_tc2_group.cuh, a CTA pair per 256 x BN tile; and
+// gemm2_dual_kernel in gemm_tc2_dual.cuh, the pair kernel for a launch that holds two kinds of problem)
 // serve all six GEMMs of the gated factorized layer W = P diag(z) Q (Section 4.1 of the paper).
 // Both are persistent and warp-specialised:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads (every CTA fetches its own tiles) into a ring of
