@@ -139,3 +139,39 @@ def test_grouped_full_size_layer_as_the_benchmark_issues_it(b, name):
         _check_against_oracle(e, "g")
         dead = e["z_np"] == 0
         assert dead.any() and np.all(host(e["dQg"])[dead] == 0)          # closed gates: exact zeros in dQ
+
+
+def test_two_launch_backward_with_optional_outputs(b):
+    """Eight 768-wide matrices at T = 512: the weight gradients fill the machine, so the backward call runs as the
+    two shared launches (dH' with dP, then dX with dQ) plus the two small ones; some problems leave out dX, dP or
+    dlog_alpha, one launch list or the other may then hold fewer problems."""
+    mats = tuple(I.Matrix(f"m{i}", 768, 768, 768) for i in range(8))
+    w = I.Workload("g", "bf16", 512, 1, mats, ("bimodal", 3.0, 0.5), 0.5)
+    es = _setup(b, w, 0, 11)
+    b.gated_lowrank_fwd_grouped([b.fwd_problem(e["X"], e["Q"], e["P"], e["z"], e["Yg"], e["Hg"]) for e in es])
+    probs = []
+    for i, e in enumerate(es):
+        dX = None if i in (1, 5) else e["dXg"]
+        dP = None if i in (2, 5) else e["dPg"]
+        dla = None if i == 3 else e["dlag"]
+        probs.append(b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], e["z"], e["dzd"], e["Hg"], dX, dP, e["dQg"], dla, e["wsg"]))
+    n0 = b.launch_count()
+    b.gated_lowrank_bwd_grouped(probs)
+    assert b.launch_count() - n0 == 4          # diag(z) Q, two GEMM launches, dlog_alpha
+    assert b.device_status() == b.OK
+    for i, e in enumerate(es):
+        p = e["prob"]
+        G = O.gated_lowrank_bwd(p["dY"], p["X"], p["Q"], p["P"], e["z_np"], e["dzd_np"])
+        if i in (1, 5):
+            assert torch.isnan(e["dXg"]).all()
+        else:
+            assert rel_fro(host(e["dXg"]), G["dX"]) < 2e-2
+        if i in (2, 5):
+            assert torch.isnan(e["dPg"]).all()
+        else:
+            assert rel_fro(host(e["dPg"]), G["dP"]) < 2e-2
+        assert rel_fro(host(e["dQg"]), G["dQ"]) < 2e-2
+        if i == 3:
+            assert torch.isnan(e["dlag"]).all()
+        else:
+            assert rel_fro(host(e["dlag"]), G["dlog_alpha"]) < 2e-2
