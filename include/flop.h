@@ -85,7 +85,8 @@ unsigned long long flop_launch_count(void);
 /* Host-only planning helper (no counterpart in the paper; no GPU needed): the static tile schedule a grouped
  * GEMM launch uses.  cost[n] (HOST) = cost of each work item in work-list order, units = persistent CTAs or CTA
  * pairs (1..148), n <= 2048.  Items are assigned by the longest-processing-time rule (sorted by cost, ties keep
- * list order, each to the least loaded unit, ties to the lower unit).  unit_of_item[n] (HOST, nullable) receives
+ * list order, each to the least loaded unit, ties to the lower unit); when the round-robin deal is already within
+ * 3 % of the lower bound max(mean load, longest item) it is kept.  unit_of_item[n] (HOST, nullable) receives
  * the unit of every item, *makespan the largest unit load, *rr_makespan the largest load of the round-robin deal
  * (item i to unit i % units) for comparison (both HOST, nullable).  FLOP_ERR_INVALID_ARG on bad sizes. */
 int flop_plan_tile_schedule(const double* cost, int32_t n, int32_t units, int32_t* unit_of_item, double* makespan,

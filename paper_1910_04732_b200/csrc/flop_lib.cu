@@ -760,11 +760,17 @@ int flop_plan_tile_schedule(const double* cost, int32_t n, int32_t units, int32_
   std::lock_guard<std::mutex> lock(mu);
   double rr = 0.0;
   const double ms = tc::build_schedule(c, units, &sched, &rr);
-  if (makespan) *makespan = n > 0 ? ms : 0.0;
+  const bool table = sched.n_units > 0;   // otherwise the launch keeps the round-robin deal (it is within 3 % of the bound)
+  if (makespan) *makespan = n > 0 ? (table ? ms : rr) : 0.0;
   if (rr_makespan) *rr_makespan = rr;
-  if (unit_of_item && n > 0)
-    for (int u = 0; u < units; ++u)
-      for (int i = sched.begin[u]; i < sched.begin[u + 1]; ++i) unit_of_item[sched.item[i]] = u;
+  if (unit_of_item && n > 0) {
+    if (table) {
+      for (int u = 0; u < units; ++u)
+        for (int i = sched.begin[u]; i < sched.begin[u + 1]; ++i) unit_of_item[sched.item[i]] = u;
+    } else {
+      for (int i = 0; i < n; ++i) unit_of_item[i] = i % units;
+    }
+  }
   return FLOP_OK;
 }
 

@@ -46,6 +46,13 @@ inline double build_schedule(const std::vector<double>& cost, int units, Schedul
     *rr_makespan = load.empty() ? 0.0 : *std::max_element(load.begin(), load.end());
   }
   if (n == 0 || n > kMaxSched || units <= 0 || units > kMaxUnits) return -1.0;
+  if (rr_makespan) {
+    // Nothing to gain when round-robin is already within 3 % of the lower bound max(mean load, longest item):
+    // skip the sort (this keeps the host cost of the common equal-tile launches at one pass over the list).
+    double total = 0.0, longest = 0.0;
+    for (int i = 0; i < n; ++i) { total += cost[(size_t)i]; longest = std::max(longest, cost[(size_t)i]); }
+    if (*rr_makespan <= 1.03 * std::max(total / units, longest)) return -1.0;
+  }
   std::vector<int> order((size_t)n);
   for (int i = 0; i < n; ++i) order[(size_t)i] = i;
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost[(size_t)a] > cost[(size_t)b]; });

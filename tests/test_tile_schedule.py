@@ -63,3 +63,11 @@ def test_edges_and_argument_checks(b):
     assert lib.flop_plan_tile_schedule(one, 2049, 4, None, None, None) == b.ERR_INVALID_ARG
     assert lib.flop_plan_tile_schedule(None, 1, 4, None, None, None) == b.ERR_INVALID_ARG
     assert lib.flop_plan_tile_schedule(one, 1, 4, None, None, None) == b.OK
+
+
+def test_round_robin_is_kept_when_it_is_within_three_per_cent_of_the_bound(b):
+    # 740 equal tiles and 74 slightly longer ones on 74 units: round-robin gives 10 short + 1 long each, the optimum
+    cost = [10.0] * 740 + [10.2] * 74
+    unit_of, ms, rr = b.plan_tile_schedule(cost, 74)
+    assert unit_of == [i % 74 for i in range(len(cost))]
+    assert ms == rr
