@@ -83,7 +83,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         self.thread.join(timeout=2)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in self.lines:
             parts = [p.strip() for p in line.split(",")]
@@ -93,10 +93,15 @@ class ClockSampler:
                 sm.append(float(parts[0])); mx.append(float(parts[1]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(parts[2]))
+            except ValueError:
+                pass
             for n, v in zip(names, parts[3:7]):
                 if v.lower() == "active":
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "sm_mhz_min": min(sm) if sm else None, "power_w": float(np.median(pw)) if pw else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
@@ -159,14 +164,19 @@ class Job:
         if group > 0:
             for e in self.mats:
                 e["ws"] = b.alloc_workspace(b.workspace_bytes(b.OP_BWD, w.T, e["m"].d_in, e["m"].d_out, e["m"].r, b.BF16), device)
+                e["Qz"] = b.padded(e["m"].r, e["m"].d_in, bf, device)      # diag(z) Q, formed once per step
+            self.scale = b.problem_array([b.scale_rows_problem(e["Q"], self.z[e["lo"]:e["hi"]], e["Qz"]) for e in self.mats])
             for i in range(0, len(self.mats), group):
                 chunk = self.mats[i:i + group]
                 fwd = b.problem_array([b.fwd_problem(e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]], e["Y"], e["H"])
                                        for e in chunk])
                 bwd = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]],
                                                      self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
-                                                     self.dlog_alpha[e["lo"]:e["hi"]], e["ws"]) for e in chunk])
-                self.groups.append((fwd, bwd))
+                                                     self.dlog_alpha[e["lo"]:e["hi"]], e["ws"], Qz=e["Qz"]) for e in chunk])
+                bwd_plain = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]],
+                                                           self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
+                                                           self.dlog_alpha[e["lo"]:e["hi"]], e["ws"]) for e in chunk])
+                self.groups.append((fwd, bwd, bwd_plain))
         # data parallelism: one gradient bucket per grouped call (a layer), reduced while later layers compute
         n_per = group if group > 0 else len(self.mats)
         sizes_w = [e["dP"].shape[0] * r8(e["m"].r) + e["m"].r * r8(e["m"].d_in) for e in self.mats]
@@ -178,6 +188,9 @@ class Job:
         self.offset_dev = torch.zeros(1, dtype=torch.int64, device=device)
         self.graph = None
         self.world = 1
+        # chained calls: one launch for the two forward products, one for the whole backward pass of a layer
+        self.chain = False
+        self.sync = b.alloc_sync(device)
 
     def enable_active_ranks(self):
         """Buffers and argument arrays for training on the active components only (z_k > 0): per layer one
@@ -255,9 +268,15 @@ class Job:
             if self.world > 1 and self.reducer is None:
                 from paper_1910_04732_b200 import dp
                 self.reducer = dp.BucketedReducer(self.wgrad, self.bucket_bounds)
-            for i, (fwd, bwd) in enumerate(self.groups):
-                self.b.gated_lowrank_fwd_grouped(fwd)
-                self.b.gated_lowrank_bwd_grouped(bwd)
+            if self.chain:
+                self.b.scale_rows_grouped(self.scale)                 # diag(z) Q of every matrix: one launch per step
+            for i, (fwd, bwd, bwd_plain) in enumerate(self.groups):
+                if self.chain:
+                    self.b.gated_lowrank_fwd_chained(fwd, self.sync)
+                    self.b.gated_lowrank_bwd_chained(bwd, self.sync)
+                else:
+                    self.b.gated_lowrank_fwd_grouped(fwd)
+                    self.b.gated_lowrank_bwd_grouped(bwd_plain)
                 if self.reducer is not None:
                     self.reducer.launch(i)                            # this layer's dP, dQ are final
         elif self.n_streams == 1:
@@ -434,6 +453,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-active", action="store_true", help="skip the extra active-rank-training measurement")
     ap.add_argument("--no-graph", action="store_true", help="issue every step from the host instead of replaying a CUDA graph")
+    ap.add_argument("--chain", action="store_true", help="chained calls (one launch for the forward products, one for the backward pass of a layer, "
+                    "ordered on the device) instead of the grouped calls (a launch per GEMM stage); measured slower on B200, see profiles/")
+    ap.add_argument("--no-chain", action="store_true", help="(default) grouped calls")
     ap.add_argument("--group", type=int, default=-1, help="matrices per grouped call (0: one call per matrix; default: one layer)")
     ap.add_argument("--streams", type=int, default=1, help="streams over which independent matrices are issued")
     args = ap.parse_args()
@@ -463,6 +485,7 @@ def main():
     group = len(w.matrices) if args.group < 0 else args.group
     job = Job(w, torch.device("cuda", local), seed=1234 + rank, n_streams=args.streams, group=group)
     job.world = world
+    job.chain = bool(args.chain) and not args.no_chain
     for _ in range(args.warmup):
         job.step()
     torch.cuda.synchronize()
@@ -490,6 +513,9 @@ def main():
         dur_ns = float((st[:, 1] - st[:, 0]).clip(min=0).sum())
         if n_st > 0 and dur_ns > 0:
             graph_gemm = {"launches": n_st, "kernel_ms_per_step": dur_ns / 1e6, "tflops": fl_st / dur_ns / 1e3}
+            if os.environ.get("FLOP_BENCH_DUMP_STAMPS"):
+                rel = (st - st[0, 0]) / 1e3
+                print("stamps_us " + " ".join(f"[{a:.1f},{b:.1f}]" for a, b in rel[:16]), file=sys.stderr)
     # second pass of the same steps with CUDA events around every tensor-core GEMM launch
     b.gemm_timing_begin()
     ms_timed_pass = time_steps(job, args.steps, world)

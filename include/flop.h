@@ -23,7 +23,9 @@
  *   - Errors are return codes.  Arguments are checked on the host before
  *     anything is launched.  A device-side wait that runs out (a pipeline
  *     barrier that never completes) makes the kernel stop cleanly and record
- *     FLOP_ERR_TIMEOUT in a device status word read by flop_device_status().
+ *     FLOP_ERR_TIMEOUT in a device status word read by flop_last_async_status().
+ *   - The only environment variable the library reads is FLOP_DEBUG (1: print the failing CUDA call to
+ *     stderr).  Variant switches for tuning exist only in a build with -DFLOP_TUNING (listed in flop_lib.cu).
  *   - Sizes of zero (T == 0, r == 0, k == 0, n == 0) are legal: outputs that
  *     exist are zero-filled where the mathematics says so, nothing else runs.
  */
@@ -66,22 +68,22 @@ typedef enum {
 
 const char* flop_status_string(int status);
 
-/* Synchronises `stream`, returns the device status word (FLOP_OK or
- * FLOP_ERR_TIMEOUT) and clears it. */
+/* Synchronises `stream`, returns the device status word (FLOP_OK, or FLOP_ERR_TIMEOUT when a bounded
+ * device-side wait of an earlier call gave up) and clears it.  flop_device_status is the same call
+ * under its older name. */
+int flop_last_async_status(void* stream);
 int flop_device_status(void* stream);
 
-/* Instrumentation (no counterpart in the paper).  flop_launch_count: kernels this
- * library has launched so far in this process.  flop_gemm_timing_begin/end: while
- * timing is on, every tensor-core GEMM launch is bracketed by CUDA events on its
- * stream; _end waits for them and returns the summed kernel time (ms), the summed
- * algorithmic flops 2 M N K of those launches and their number (HOST out pointers,
- * nullable).  Not thread-safe with respect to concurrent launches. */
 /* Self-test of the bounded device-side wait (no counterpart in the paper): launches one thread that waits
  * on a barrier nothing will ever signal, for at most limit_cycles SM cycles (<= 2e9), then records
  * FLOP_ERR_TIMEOUT in the device status word and writes 1 to *gave_up_dev (DEVICE int).  The context stays
- * usable; flop_device_status() returns and clears the code. */
+ * usable; flop_last_async_status() returns and clears the code. */
 int flop_selftest_wait_timeout(int64_t limit_cycles, int* gave_up_dev, void* stream);
+
+/* Instrumentation (no counterpart in the paper): kernels this library has launched so far in this
+ * process.  Not synchronised with concurrent launches from other threads. */
 unsigned long long flop_launch_count(void);
+
 /* Host-only planning helper (no counterpart in the paper; no GPU needed): the static tile schedule a grouped
  * GEMM launch uses.  cost[n] (HOST) = cost of each work item in work-list order, units = persistent CTAs or CTA
  * pairs (1..148), n <= 2048.  Items are assigned by the longest-processing-time rule (sorted by cost, ties keep
@@ -91,6 +93,18 @@ unsigned long long flop_launch_count(void);
  * (item i to unit i % units) for comparison (both HOST, nullable).  FLOP_ERR_INVALID_ARG on bad sizes. */
 int flop_plan_tile_schedule(const double* cost, int32_t n, int32_t units, int32_t* unit_of_item, double* makespan,
                             double* rr_makespan);
+
+/* The queue of a chained launch (flop_gated_lowrank_*_chained; host only): stage[n] (HOST) is 0 for tiles that
+ * wait for nothing and 1 for tiles that read a stage-0 output; key[n] (HOST) orders the tiles inside a stage (lower
+ * first, ties keep list order).  queue_pos[n] (HOST, nullable) receives every item's position in the queue the
+ * persistent CTA pairs draw from.  All stage-0 items come before all stage-1 items, which is what makes the
+ * device-side waits free of cycles.  n <= 2048. */
+int flop_plan_chain_queue(const int32_t* stage, const int64_t* key, int32_t n, int32_t* queue_pos);
+
+/* Instrumentation (no counterpart in the paper).  While timing is on, every tensor-core GEMM launch is
+ * bracketed by CUDA events on its stream; _end waits for them and returns the summed kernel time (ms), the
+ * summed algorithmic flops 2 M N K of those launches and their number (HOST out pointers, nullable).
+ * Single-threaded use only: the event list and the counters are not guarded against concurrent launches. */
 int flop_gemm_timing_begin(void);
 int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launches);
 
@@ -99,7 +113,8 @@ int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launche
  * there the %globaltimer (ns) at which its first CTA passed the dependency wait and the latest
  * time at which one of its CTAs finished.  The pointers stay in the launches, so a CUDA graph
  * captured in between refreshes the stamps at every replay; this times kernels where host events
- * cannot be placed.  _end returns the number of stamped launches and the sum of their 2 M N K. */
+ * cannot be placed.  _end returns the number of stamped launches and the sum of their 2 M N K.
+ * Single-threaded use only, like the event timing above. */
 int flop_gemm_stamps_begin(unsigned long long* stamps_dev, int capacity);
 int flop_gemm_stamps_end(int* launches, double* total_flops);
 
@@ -199,11 +214,45 @@ typedef struct {
   int64_t T, d_in, d_out, r;
   void* ws; size_t ws_bytes;
   const int32_t* r_dev; /* nullable */
+  const void* Qz; int64_t ldqz; /* nullable: diag(z) Q formed beforehand by flop_scale_rows_grouped (same z, same Q) */
 } flop_bwd_problem_t;
+
+/* diag(z) Q for n matrices in one launch: Qz[k, :] = z[k] * Q[k, :] (r x d_in, bf16, rounded once).  The
+ * backward pass multiplies by it (dX = dH' (diag(z) Q), chain rule on Section 4.1); it depends only on the gate
+ * sample and the weights, so a training step may form it once, right after flop_gate_sample, for all
+ * matrices of the model, and pass it to the grouped / chained backward calls (flop_bwd_problem_t.Qz).
+ * Problems that leave Qz NULL have it formed inside the backward call, in their workspace.  HOST array. */
+typedef struct {
+  const void* Q; int64_t ldq; const float* z; void* Qz; int64_t ldqz; int64_t r, d_in;
+} flop_scale_rows_t;
+int flop_scale_rows_grouped(const flop_scale_rows_t* problems, int n, int dt, void* stream);
 
 int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* problems, int n, int dt, void* stream);
 int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* problems, int n, int accumulate, int dt,
                                    int wgrad_dt, void* stream);
+
+/* Chained forms: the same results as the grouped calls, with the dependent products of the call in ONE
+ * persistent launch (Section 4.1: y = P G Q x is two products that feed each other; its chain rule is two
+ * products, dH' = dY P and dP, followed by two that read dH').  The tiles of H' = (X Q^T) * z and of
+ * Y = H' P^T share one work list; a tile of the second product waits, on the device, for the 256-row block
+ * of H' it reads (counters in `sync`), instead of the whole first launch draining before the second fills.
+ * The backward call likewise runs {dH', dP} and {dX, dQ} in one launch, forms diag(z) Q inside it and
+ * finishes dlog_alpha inside it (no small kernels before or after).
+ *   sync       DEVICE, 16-byte aligned, at least flop_sync_bytes() bytes.  The CALLER zero-fills it once
+ *              (e.g. cudaMemsetAsync) before its first use; every call leaves it zero-filled again, also
+ *              inside a replayed CUDA graph.  Calls that share a sync area must be ordered on the GPU
+ *              (same stream, or events); concurrent calls need separate areas.  If a call ever reports
+ *              FLOP_ERR_TIMEOUT through flop_last_async_status(), zero-fill the area again.
+ *   Fallback   When the shapes do not allow one launch (fp32 storage, a product that needs split-K or
+ *              one-CTA tiles, more than 24 products, more counters than the area holds) the call runs the
+ *              grouped sequence of launches; results are the same.
+ *   Every wait on a counter is bounded like the pipeline waits (FLOP_ERR_TIMEOUT in the status word).
+ * flop_sync_bytes: HOST out pointer. */
+int flop_sync_bytes(size_t* out_bytes);
+int flop_gated_lowrank_fwd_chained(const flop_fwd_problem_t* problems, int n, int dt, void* sync,
+                                   size_t sync_bytes, void* stream);
+int flop_gated_lowrank_bwd_chained(const flop_bwd_problem_t* problems, int n, int accumulate, int dt,
+                                   int wgrad_dt, void* sync, size_t sync_bytes, void* stream);
 
 /* Training on the active rank components only (Section 4.3, last paragraph: the
  * mask is shared by the batch, so "parameters that are only active for the current

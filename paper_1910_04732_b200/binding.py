@@ -20,7 +20,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD, OP_EMBEDDING_BWD = range(6)
 
-EXPORTS = ("flop_status_string", "flop_device_status", "flop_selftest_wait_timeout", "flop_launch_count", "flop_plan_tile_schedule", "flop_gemm_timing_begin",
+EXPORTS = ("flop_status_string", "flop_last_async_status", "flop_device_status", "flop_sync_bytes",
+           "flop_gated_lowrank_fwd_chained", "flop_gated_lowrank_bwd_chained", "flop_selftest_wait_timeout", "flop_launch_count", "flop_plan_tile_schedule", "flop_plan_chain_queue", "flop_scale_rows_grouped", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_gemm_stamps_begin", "flop_gemm_stamps_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
@@ -49,7 +50,13 @@ class BwdProblem(ctypes.Structure):
                 ("dX", ctypes.c_void_p), ("lddx", ctypes.c_int64), ("dP", ctypes.c_void_p), ("lddp", ctypes.c_int64),
                 ("dQ", ctypes.c_void_p), ("lddq", ctypes.c_int64), ("dlog_alpha", ctypes.c_void_p),
                 ("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
-                ("ws", ctypes.c_void_p), ("ws_bytes", ctypes.c_size_t), ("r_dev", ctypes.c_void_p)]
+                ("ws", ctypes.c_void_p), ("ws_bytes", ctypes.c_size_t), ("r_dev", ctypes.c_void_p),
+                ("Qz", ctypes.c_void_p), ("ldqz", ctypes.c_int64)]
+
+
+class ScaleRows(ctypes.Structure):
+    _fields_ = [("Q", ctypes.c_void_p), ("ldq", ctypes.c_int64), ("z", ctypes.c_void_p), ("Qz", ctypes.c_void_p),
+                ("ldqz", ctypes.c_int64), ("r", ctypes.c_int64), ("d_in", ctypes.c_int64)]
 
 
 class ActiveGather(ctypes.Structure):
@@ -91,11 +98,18 @@ def load_library() -> ctypes.CDLL:
     lib.flop_status_string.restype = ctypes.c_char_p
     lib.flop_status_string.argtypes = [ci]
     lib.flop_device_status.argtypes = [vp]
+    lib.flop_last_async_status.argtypes = [vp]
+    lib.flop_sync_bytes.argtypes = [ctypes.POINTER(sz)]
+    lib.flop_gated_lowrank_fwd_chained.argtypes = [ctypes.POINTER(FwdProblem), ci, ci, vp, sz, vp]
+    lib.flop_gated_lowrank_bwd_chained.argtypes = [ctypes.POINTER(BwdProblem), ci, ci, ci, ci, vp, sz, vp]
     lib.flop_workspace_bytes.argtypes = [ci, i64, i64, i64, i64, ci, ctypes.POINTER(sz)]
     lib.flop_launch_count.argtypes = []
     lib.flop_plan_tile_schedule.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.c_int32, ctypes.c_int32,
                                             ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double),
                                             ctypes.POINTER(ctypes.c_double)]
+    lib.flop_plan_chain_queue.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32,
+                                          ctypes.POINTER(ctypes.c_int32)]
+    lib.flop_scale_rows_grouped.argtypes = [ctypes.POINTER(ScaleRows), ci, ci, vp]
     lib.flop_selftest_wait_timeout.argtypes = [i64, vp, vp]
     lib.flop_gemm_timing_begin.argtypes = []
     lib.flop_gemm_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
@@ -141,6 +155,16 @@ def plan_tile_schedule(cost, units: int):
     _check(load_library().flop_plan_tile_schedule(c, n, int(units), out, ctypes.byref(ms), ctypes.byref(rr)),
            "flop_plan_tile_schedule")
     return list(out)[:n], ms.value, rr.value
+
+
+def plan_chain_queue(stage, key):
+    """Host-only: the position of every work item in the queue of a chained launch."""
+    n = len(stage)
+    st = (ctypes.c_int32 * max(n, 1))(*[int(v) for v in stage])
+    k = (ctypes.c_int64 * max(n, 1))(*[int(v) for v in key])
+    pos = (ctypes.c_int32 * max(n, 1))()
+    _check(load_library().flop_plan_chain_queue(st, k, n, pos), "flop_plan_chain_queue")
+    return list(pos)[:n]
 
 
 def status_string(code: int) -> str:
@@ -293,13 +317,24 @@ def fwd_problem(X, Q, P, z, Y, H_save, r_dev=None) -> FwdProblem:
                       T, d_in, d_out, r, _p(r_dev))
 
 
-def bwd_problem(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws, r_dev=None) -> BwdProblem:
+def bwd_problem(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws, r_dev=None, Qz=None) -> BwdProblem:
     T, d_in = X.shape
     d_out, r = P.shape
     ld = lambda t: _ld(t) if t is not None else 0
     return BwdProblem(_p(dY), _ld(dY), _p(X), _ld(X), _p(Q), _ld(Q), _p(P), _ld(P), _p(z), _p(dz_dla), _p(H_save),
                       _ld(H_save), _p(dX), ld(dX), _p(dP), ld(dP), _p(dQ), ld(dQ), _p(dlog_alpha), T, d_in, d_out, r,
-                      _p(ws), ws.numel() if ws is not None else 0, _p(r_dev))
+                      _p(ws), ws.numel() if ws is not None else 0, _p(r_dev), _p(Qz), ld(Qz))
+
+
+def scale_rows_problem(Q, z, Qz) -> ScaleRows:
+    r, d_in = Q.shape
+    return ScaleRows(_p(Q), _ld(Q), _p(z), _p(Qz), _ld(Qz), r, d_in)
+
+
+def scale_rows_grouped(problems, dt: int = BF16) -> None:
+    """Qz = diag(z) Q for every problem, one launch (per 96 matrices)."""
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_scale_rows_grouped(arr, len(arr), dt, _stream()), "flop_scale_rows_grouped")
 
 
 def active_gather_problem(z, dz_dla, P, Q, idx, pos, k_dev, z_c, dz_dla_c, P_c, Q_c) -> ActiveGather:
@@ -340,6 +375,30 @@ def gated_lowrank_bwd_grouped(problems, accumulate: bool = False, dt: int = BF16
     arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
     _check(load_library().flop_gated_lowrank_bwd_grouped(arr, len(arr), int(accumulate), dt, wgrad_dt, _stream()),
            "flop_gated_lowrank_bwd_grouped")
+
+
+def sync_bytes() -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().flop_sync_bytes(ctypes.byref(out)), "flop_sync_bytes")
+    return int(out.value)
+
+
+def alloc_sync(device="cuda") -> torch.Tensor:
+    """A zero-filled sync area for the chained calls (they leave it zero-filled)."""
+    return torch.zeros(sync_bytes(), dtype=torch.uint8, device=device)
+
+
+def gated_lowrank_fwd_chained(problems, sync: torch.Tensor, dt: int = BF16) -> None:
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_gated_lowrank_fwd_chained(arr, len(arr), dt, _ptr(sync), sync.numel(), _stream()),
+           "flop_gated_lowrank_fwd_chained")
+
+
+def gated_lowrank_bwd_chained(problems, sync: torch.Tensor, accumulate: bool = False, dt: int = BF16,
+                              wgrad_dt: int = BF16) -> None:
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_gated_lowrank_bwd_chained(arr, len(arr), int(accumulate), dt, wgrad_dt, _ptr(sync),
+                                                         sync.numel(), _stream()), "flop_gated_lowrank_bwd_chained")
 
 
 def expected_l0_lagrangian(log_alpha, seg_off, seg_size, hc, target, lam, out4, seg_expected=None,

@@ -24,6 +24,7 @@
 #include "gemm_tc_group.cuh"
 #include "gemm_tc2_group.cuh"
 #include "gemm_tc2_dual.cuh"
+#include "gemm_tc2_chain.cuh"
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
 #include "active_ranks.cuh"
@@ -59,14 +60,39 @@ inline bool debug_on() {
   } while (0)
 
 
+// Tuning switches.  A library built with -DFLOP_TUNING reads them once from the environment (they exist to
+// compare variants on one machine); the normal build takes the defaults below and reads nothing but FLOP_DEBUG.
+//   FLOP_NO_PDL=1          launch without programmatic dependent launch
+//   FLOP_TC_BN / FLOP_TC_STAGES / FLOP_TC_CTA2 (1 force pairs, 2 forbid)     tile shape of single GEMMs
+//   FLOP_TC_GROUP_BN / FLOP_TC_GROUP_CTA2, FLOP_TC_WGRAD_BN / FLOP_TC_WGRAD_CTA2   tile shape of grouped launches
+//   FLOP_NO_TMA_STORE=1    bf16 output tiles by per-thread stores    FLOP_NO_SCHED=1   round-robin tile order
+//   FLOP_NO_SMALL_T=1, FLOP_NO_SKINNY=1   few-token forward kernels off
+//   FLOP_STAGE_MERGE=0     backward in three launches per stage instead of two shared ones
+//   FLOP_GATHER_PIPE=0     plain P gather kernel                     FLOP_NO_CHAIN=1   chained calls run unchained
+struct Tuning {
+  int no_pdl = 0, tc_bn = 0, tc_stages = 0, tc_cta2 = 0, no_tma_store = 0, no_sched = 0, group_bn = 0, group_cta2 = 0,
+      wgrad_bn = 0, wgrad_cta2 = 0, no_small_t = 0, no_skinny = 0, stage_merge = 1, gather_pipe = 1, no_chain = 0;
+};
+inline const Tuning& tuning() {
+  static const Tuning t = [] {
+    Tuning v;
+#ifdef FLOP_TUNING
+    auto get = [](const char* name, int dflt) { const char* e = getenv(name); return e ? atoi(e) : dflt; };
+    v.no_pdl = get("FLOP_NO_PDL", 0); v.tc_bn = get("FLOP_TC_BN", 0); v.tc_stages = get("FLOP_TC_STAGES", 0);
+    v.tc_cta2 = get("FLOP_TC_CTA2", 0); v.no_tma_store = get("FLOP_NO_TMA_STORE", 0); v.no_sched = get("FLOP_NO_SCHED", 0);
+    v.group_bn = get("FLOP_TC_GROUP_BN", 0); v.group_cta2 = get("FLOP_TC_GROUP_CTA2", 0); v.wgrad_bn = get("FLOP_TC_WGRAD_BN", 0);
+    v.wgrad_cta2 = get("FLOP_TC_WGRAD_CTA2", 0); v.no_small_t = get("FLOP_NO_SMALL_T", 0); v.no_skinny = get("FLOP_NO_SKINNY", 0);
+    v.stage_merge = get("FLOP_STAGE_MERGE", 1); v.gather_pipe = get("FLOP_GATHER_PIPE", 1); v.no_chain = get("FLOP_NO_CHAIN", 0);
+#endif
+    return v;
+  }();
+  return t;
+}
+
 // Every kernel goes through here: programmatic dependent launch lets a kernel's prologue overlap
 // the tail of its predecessor on the stream (the kernels call griddepcontrol.wait before they
-// touch global memory).  FLOP_NO_PDL=1 in the environment turns the attribute off.
-inline bool pdl_on() {
-  static int v = -1;
-  if (v < 0) { const char* e = getenv("FLOP_NO_PDL"); v = (e && e[0] && e[0] != '0') ? 0 : 1; }
-  return v == 1;
-}
+// touch global memory).
+inline bool pdl_on() { return !tuning().no_pdl; }
 template <typename... KArgs, typename... Args>
 inline void launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
   cudaLaunchConfig_t cfg{};
@@ -86,15 +112,33 @@ inline bool valid_dt(int dt) { return dt == FLOP_F32 || dt == FLOP_BF16; }
 inline size_t elt(int dt) { return dt == FLOP_BF16 ? 2 : 4; }
 inline bool valid_hc(const flop_hc_params_t& hc) { return hc.beta > 0.f && hc.gamma < 0.f && hc.zeta > 1.f; }
 
+// Per-device state (function attributes already set, SM count, built-in scratch address) is indexed by the
+// current device, so that a process that drives several GPUs configures each of them.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
+  return (dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
+// True the first time it is called for (flag array, current device): the caller then sets its function attributes.
+inline bool first_use_on_device(bool (&done)[kMaxDevices]) {
+  const int dev = current_device();
+  if (dev < 0) return true;            // unknown device: configure every time
+  if (done[dev]) return false;
+  done[dev] = true;
+  return true;
+}
+
 int num_sms() {
-  static int cached = 0;
-  if (cached) return cached;
-  int dev = 0, n = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+  static int cached[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev >= 0 && cached[dev]) return cached[dev];
+  int n = 0;
+  if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
     cudaGetLastError();
     return 148;   // B200; used only for planning when no device is visible
   }
-  cached = n;
+  cached[dev] = n;
   return n;
 }
 
@@ -163,20 +207,18 @@ struct TcPlan {
 };
 
 constexpr int kSmemBudget = 227 * 1024 - 1024;   // opt-in maximum minus room for the static __shared__ variables
-constexpr int kSmemBarrierBytes = 8 * (2 * tc::kMaxStages + 5);
+constexpr int kSmemBarrierBytes = 384;   // pipeline barriers (8 x (2 x 8 + 5) bytes) and the chained kernel's queue ring (160 bytes)
 constexpr int kSmemFixed = 1024 + (int)tc::kStoreBufTotal + kSmemBarrierBytes;   // alignment slack + epilogue staging + barriers
 
-inline int env_int(const char* name) { const char* e = getenv(name); return e ? atoi(e) : 0; }
 
 // Picks the tile shape (one CTA: 128 x bn; CTA pair: 256 x bn), and the split-K factor, by a small
 // cost model in SM cycles: waves over the machine x (k-blocks per work item x the slower of MMA
 // issue and shared-memory fill, plus the epilogue).  The fill rate of one SM's shared memory was
 // measured at about 54 bytes per cycle; a 128 x bn x 64 MMA block takes 2*bn cycles.
-// FLOP_TC_BN, FLOP_TC_STAGES, FLOP_TC_CTA2 (1 = force pairs, 2 = forbid pairs) override for tuning.
 TcPlan plan_tc(int64_t M, int64_t N, int64_t K, bool allow_split, bool b_mn_major, bool allow_cta2 = true) {
   const int sms = num_sms();
   const int num_kb = (int)((K + tc::BK - 1) / tc::BK);
-  static const int force_bn = env_int("FLOP_TC_BN"), force_stages = env_int("FLOP_TC_STAGES"), force_cta2 = env_int("FLOP_TC_CTA2");
+  const int force_bn = tuning().tc_bn, force_stages = tuning().tc_stages, force_cta2 = tuning().tc_cta2;
   TcPlan best{};
   double best_cost = 1e300;
   const int bns[4] = {256, 192, 128, 64};
@@ -289,17 +331,20 @@ struct TcJob {
   const int* dyn_m = nullptr;   // effective sizes on the device (see tc::Params), nullable
   const int* dyn_n = nullptr;
   const int* dyn_k = nullptr;
+  // chained launches (gemm_tc2_chain.cuh): stage 0 waits for nothing, stage 1 reads a stage-0 output; inside a
+  // stage a unit walks lower classes first; link holds the counters and the folded-in side work
+  int stage = 0, order_class = 0;
+  tc::ChainLink link{};
 };
 
 template <bool A_MN, bool B_MN, int EPI>
 int launch_group_inst(const tc::GroupParams& gp, int cta2, double flops, cudaStream_t st) {
-  static bool configured = false;
+  static bool configured[kMaxDevices] = {};
   auto kern1 = tc::gemm_group_kernel<A_MN, B_MN, EPI>;
   auto kern2 = tc::gemm2_group_kernel<A_MN, B_MN, EPI>;
-  if (!configured) {
+  if (first_use_on_device(configured)) {
     FLOP_CUDA(cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     FLOP_CUDA(cudaFuncSetAttribute(kern2, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    configured = true;
   }
   {
     GemmTimer timer(st, flops);
@@ -329,12 +374,9 @@ int launch_group_inst(const tc::GroupParams& gp, int cta2, double flops, cudaStr
 // A launch whose problems are of two kinds: bf16 stores with (K-major A, MN-major B) and in-place weight
 // gradients with both operands MN-major (the two steps of the grouped backward pass).  CTA pairs only.
 int launch_dual_inst(const tc::GroupParams& gp, double flops, cudaStream_t st) {
-  static bool configured = false;
+  static bool configured[kMaxDevices] = {};
   auto kern = tc::gemm2_dual_kernel<false, true, tc::EPI_STORE, true, true, tc::EPI_WGRAD>;
-  if (!configured) {
-    FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    configured = true;
-  }
+  if (first_use_on_device(configured)) FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
   {
     GemmTimer timer(st, flops);
     const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes2(gp.bn_max);
@@ -355,6 +397,55 @@ int launch_dual_inst(const tc::GroupParams& gp, double flops, cudaStream_t st) {
   return FLOP_OK;
 }
 
+// Fills the next problem slot of a launch from a job: tensor maps, sizes, epilogue, work-list position; appends
+// the cost of each of its work items (SM cycles, the model of plan_group) for the schedule.
+int add_problem(tc::GroupParams& gp, const TcJob& j, std::vector<double>& item_cost, double& flops) {
+  if (j.M > INT32_MAX || j.N > INT32_MAX || j.K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
+  const bool kind1 = j.A.mn_major && j.B.mn_major && j.ep.kind == tc::EPI_WGRAD;
+  tc::GroupProblem& pr = gp.prob[gp.n];
+  pr.p.kind = kind1 ? 1 : 0;
+  if (!j.A.mn_major) FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.M, j.K, j.A.ld, tc::BK, tc::BM));
+  else               FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.K, j.M, j.A.ld, tc::kBoxMN, tc::BK));
+  if (!j.B.mn_major) FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.N, j.K, j.B.ld, tc::BK, (uint32_t)(j.pl.cta2 ? j.pl.bn / 2 : j.pl.bn)));
+  else               FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.K, j.N, j.B.ld, tc::kBoxMN, tc::BK));
+  tc::Params& p = pr.p;
+  p.M = (int)j.M; p.N = (int)j.N; p.K = (int)j.K;
+  p.bn = j.pl.bn; p.stages = 0; p.tiles_m = j.pl.tiles_m; p.tiles_n = j.pl.tiles_n;
+  p.splits = j.pl.splits; p.kb_per_split = j.pl.kb_per_split; p.num_kb = j.pl.num_kb;
+  p.out = j.ep.out; p.ldo = j.ep.ldo; p.col_scale = j.ep.col_scale;
+  p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
+  p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
+  p.wg_out = j.ep.wg_out; p.wg_f32 = j.ep.wg_f32; p.row_scale = j.ep.row_scale; p.accumulate = j.ep.accumulate;
+  p.dyn_m = j.dyn_m; p.dyn_n = j.dyn_n; p.dyn_k = j.dyn_k;
+  p.link = j.link;
+  // bf16 tiles that are plainly overwritten leave through a TMA store (64 x 32 boxes of the output)
+  void* tma_dst = j.ep.kind == tc::EPI_STORE ? (void*)j.ep.out
+                  : (j.ep.kind == tc::EPI_WGRAD && !j.ep.wg_f32 && !j.ep.accumulate) ? j.ep.wg_out : nullptr;
+  p.tma_store = (tma_dst && !tuning().no_tma_store) ? 1 : 0;
+  if (p.tma_store) FLOP_TRY(make_tmap(&pr.tout, tma_dst, j.M, j.N, j.ep.ldo, 64, 32));
+  pr.work_begin = gp.total_work;
+  gp.total_work += p.tiles_m * p.tiles_n * p.splits;
+  const double bytes = j.pl.cta2 ? (double)tc::stage_bytes2(p.bn) : (double)tc::stage_bytes(p.bn);
+  const double per_kb = std::max(2.0 * p.bn, bytes / 50.0), epi = 400.0 + 4.0 * p.bn;
+  if (item_cost.size() <= (size_t)tc::kMaxSched)
+    for (int sp = 0; sp < p.splits; ++sp) {
+      const int kbs = std::min(p.kb_per_split, p.num_kb - sp * p.kb_per_split);
+      item_cost.insert(item_cost.end(), (size_t)p.tiles_m * p.tiles_n, kbs * per_kb + epi);
+    }
+  gp.bn_max = std::max(gp.bn_max, p.bn);
+  flops += 2.0 * j.M * (double)j.N * j.K;
+  ++gp.n;
+  return FLOP_OK;
+}
+
+inline void attach_stamp(tc::GroupParams& gp, double flops) {
+  gp.stamp = nullptr;
+  if (g_stamps.buf && g_stamps.used < g_stamps.capacity) {
+    gp.stamp = g_stamps.buf + 2 * g_stamps.used++;
+    g_stamps.flops += flops;
+  }
+}
+
 int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
   size_t i = 0;
   while (i < jobs.size()) {
@@ -367,64 +458,24 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     for (; i < jobs.size() && gp.n < tc::kMaxGroup; ++i) {
       const TcJob& j = jobs[i];
       if (j.M <= 0 || j.N <= 0 || j.K <= 0) continue;
-      if (j.M > INT32_MAX || j.N > INT32_MAX || j.K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
       if (j.pl.cta2 != first.pl.cta2) return FLOP_ERR_INVALID_ARG;
       if (j.A.mn_major != first.A.mn_major || j.B.mn_major != first.B.mn_major || j.ep.kind != first.ep.kind) uniform = false;
       const bool kind0 = !j.A.mn_major && j.B.mn_major && j.ep.kind == tc::EPI_STORE;
       const bool kind1 = j.A.mn_major && j.B.mn_major && j.ep.kind == tc::EPI_WGRAD;
       if (!(kind0 || kind1) || !j.pl.cta2) dual_ok = false;
-      tc::GroupProblem& pr = gp.prob[gp.n];
-      pr.p.kind = kind1 ? 1 : 0;
-      if (!j.A.mn_major) FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.M, j.K, j.A.ld, tc::BK, tc::BM));
-      else               FLOP_TRY(make_tmap(&pr.ta, j.A.ptr, j.K, j.M, j.A.ld, tc::kBoxMN, tc::BK));
-      if (!j.B.mn_major) FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.N, j.K, j.B.ld, tc::BK, (uint32_t)(j.pl.cta2 ? j.pl.bn / 2 : j.pl.bn)));
-      else               FLOP_TRY(make_tmap(&pr.tb, j.B.ptr, j.K, j.N, j.B.ld, tc::kBoxMN, tc::BK));
-      tc::Params& p = pr.p;
-      p.M = (int)j.M; p.N = (int)j.N; p.K = (int)j.K;
-      p.bn = j.pl.bn; p.stages = 0; p.tiles_m = j.pl.tiles_m; p.tiles_n = j.pl.tiles_n;
-      p.splits = j.pl.splits; p.kb_per_split = j.pl.kb_per_split; p.num_kb = j.pl.num_kb;
-      p.out = j.ep.out; p.ldo = j.ep.ldo; p.col_scale = j.ep.col_scale;
-      p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
-      p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
-      p.wg_out = j.ep.wg_out; p.wg_f32 = j.ep.wg_f32; p.row_scale = j.ep.row_scale; p.accumulate = j.ep.accumulate;
-      p.dyn_m = j.dyn_m; p.dyn_n = j.dyn_n; p.dyn_k = j.dyn_k;
-      // bf16 tiles that are plainly overwritten leave through a TMA store (64 x 32 boxes of the output)
-      void* tma_dst = j.ep.kind == tc::EPI_STORE ? (void*)j.ep.out
-                      : (j.ep.kind == tc::EPI_WGRAD && !j.ep.wg_f32 && !j.ep.accumulate) ? j.ep.wg_out : nullptr;
-      static const int no_tma_store = env_int("FLOP_NO_TMA_STORE");
-      p.tma_store = (tma_dst && !no_tma_store) ? 1 : 0;
-      if (p.tma_store) FLOP_TRY(make_tmap(&pr.tout, tma_dst, j.M, j.N, j.ep.ldo, 64, 32));
-      pr.work_begin = gp.total_work;
-      gp.total_work += p.tiles_m * p.tiles_n * p.splits;
-      {   // cost of each work item of this problem in SM cycles (the model of plan_group), for the schedule
-        const double bytes = j.pl.cta2 ? (double)tc::stage_bytes2(p.bn) : (double)tc::stage_bytes(p.bn);
-        const double per_kb = std::max(2.0 * p.bn, bytes / 50.0), epi = 400.0 + 4.0 * p.bn;
-        if (item_cost.size() <= (size_t)tc::kMaxSched)
-          for (int sp = 0; sp < p.splits; ++sp) {
-            const int kbs = std::min(p.kb_per_split, p.num_kb - sp * p.kb_per_split);
-            item_cost.insert(item_cost.end(), (size_t)p.tiles_m * p.tiles_n, kbs * per_kb + epi);
-          }
-      }
-      gp.bn_max = std::max(gp.bn_max, p.bn);
-      flops += 2.0 * j.M * (double)j.N * j.K;
-      ++gp.n;
+      FLOP_TRY(add_problem(gp, j, item_cost, flops));
     }
     if (gp.n == 0) continue;
     const int cta2 = first.pl.cta2;
     gp.stages = std::min(tc::kMaxStages, (kSmemBudget - kSmemFixed) /
                                              (int)(cta2 ? tc::stage_bytes2(gp.bn_max) : tc::stage_bytes(gp.bn_max)));
-    gp.stamp = nullptr;
-    if (g_stamps.buf && g_stamps.used < g_stamps.capacity) {
-      gp.stamp = g_stamps.buf + 2 * g_stamps.used++;
-      g_stamps.flops += flops;
-    }
+    attach_stamp(gp, flops);
     // Tiles of unequal length: deal them out by the longest-processing-time rule when that beats the
-    // round-robin order (FLOP_NO_SCHED=1 keeps round-robin, for comparison).
+    // round-robin order.
     {
-      static const int no_sched = env_int("FLOP_NO_SCHED");
       const int units = std::min(gp.total_work, cta2 ? num_sms() / 2 : num_sms());
       double rr = 0.0;
-      if (no_sched || (int)item_cost.size() != gp.total_work) {
+      if (tuning().no_sched || (int)item_cost.size() != gp.total_work) {
         gp.sched.n_units = 0;
       } else {
         const double lpt = tc::build_schedule(item_cost, units, &gp.sched, &rr);
@@ -441,6 +492,113 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
     FLOP_TRY(rc);
   }
   return FLOP_OK;
+}
+
+// ---- chained launch: the tiles of two dependent GEMM stages in ONE persistent CTA-pair launch (gemm_tc2_chain.cuh)
+constexpr size_t kSyncBytes = 64 * 1024;   // size of a sync area (flop_sync_bytes)
+
+template <bool A0, bool B0, int E0, bool A1, bool B1, int E1>
+int launch_chain_inst(const tc::GroupParams& gp, int pairs, double flops, cudaStream_t st) {
+  static bool configured[kMaxDevices] = {};
+  auto kern = tc::gemm2_chain_kernel<A0, B0, E0, A1, B1, E1>;
+  if (first_use_on_device(configured)) FLOP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+  {
+    GemmTimer timer(st, flops);
+    const int smem = kSmemFixed + gp.stages * (int)tc::stage_bytes2(gp.bn_max);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(tc::kChainThreads); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_on() ? 2 : 1;
+    cudaLaunchKernelEx(&cfg, kern, gp);
+  }
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
+// Whether a set of jobs can run as one chained launch: CTA-pair tiles throughout, no split-K, at most
+// kMaxGroup problems, and a sync area that holds `sync_words` counters.
+bool chain_ok(const std::vector<TcJob>& jobs, const void* sync, size_t sync_bytes, size_t sync_words) {
+  if (!sync || tuning().no_chain || jobs.empty() || jobs.size() > (size_t)tc::kMaxGroup) return false;
+  if (sync_words * 4 > std::min(sync_bytes, kSyncBytes)) return false;
+  for (const TcJob& j : jobs)
+    if (!j.pl.cta2 || j.pl.splits != 1 || j.M <= 0 || j.N <= 0 || j.K <= 0) return false;
+  return true;
+}
+
+// jobs: stage-0 jobs first (when the queue table cannot hold the launch the kernel walks the work list in order).
+// backward = the two kinds of the backward pass (bf16 store with MN-major B / in-place weight gradient), else bf16
+// stores with both operands K-major.  dep_job[i] = index of the job whose output job i reads (-1: none).
+int launch_tc_chain(const std::vector<TcJob>& jobs, const std::vector<int>& dep_job, unsigned* sync, int sync_words, bool backward,
+                    cudaStream_t st) {
+  tc::GroupParams gp;
+  memset(&gp, 0, sizeof(gp));
+  double flops = 0.0;
+  std::vector<double> item_cost;
+  struct Item { int job, tm; };
+  std::vector<Item> items;
+  bool side = false;
+  for (size_t i = 0; i < jobs.size(); ++i) {
+    const TcJob& j = jobs[i];
+    if (i > 0 && j.stage < jobs[i - 1].stage) return FLOP_ERR_INVALID_ARG;
+    FLOP_TRY(add_problem(gp, j, item_cost, flops));
+    for (int tm = 0; tm < j.pl.tiles_m; ++tm)
+      for (int tn = 0; tn < j.pl.tiles_n; ++tn) items.push_back(Item{(int)i, tm});
+    if (j.link.sw_qz) side = true;
+  }
+  gp.stages = std::min(tc::kMaxStages, (kSmemBudget - kSmemFixed) / (int)tc::stage_bytes2(gp.bn_max));
+  attach_stamp(gp, flops);
+  const int pairs = std::max(1, std::min(gp.total_work, num_sms() / 2));
+  // Queue order.  First stage: by class (tiles that others wait for first), long tiles before short ones, then by
+  // row block and problem.  Second stage: by class, then in the order in which the tiles they wait for leave the
+  // queue, long before short.
+  gp.sched.n_units = 0;
+  const int n = (int)items.size();
+  if ((int)item_cost.size() == n && n == gp.total_work && n <= tc::kMaxSched) {
+    const int64_t kCostMax = (int64_t)1 << 30;
+    auto inv_cost = [&](int i) { return kCostMax - std::min<int64_t>(kCostMax - 1, (int64_t)item_cost[(size_t)i]); };
+    std::vector<int> stage((size_t)n);
+    std::vector<int64_t> key((size_t)n, 0);
+    std::vector<int> first;   // stage-0 items
+    for (int i = 0; i < n; ++i) {
+      const TcJob& j = jobs[(size_t)items[(size_t)i].job];
+      stage[(size_t)i] = j.stage;
+      if (j.stage == 0) {
+        key[(size_t)i] = ((int64_t)j.order_class << 60) | (inv_cost(i) << 28) | ((int64_t)items[(size_t)i].tm << 8) | (int64_t)items[(size_t)i].job;
+        first.push_back(i);
+      }
+    }
+    std::stable_sort(first.begin(), first.end(), [&](int a, int b) { return key[(size_t)a] < key[(size_t)b]; });
+    // position in the queue at which the last tile of (job, row block) is drawn, and of the whole job
+    std::vector<std::vector<int>> ready(jobs.size());
+    std::vector<int> ready_all(jobs.size(), 0);
+    for (size_t q = 0; q < jobs.size(); ++q) ready[q].assign((size_t)std::max(1, jobs[q].pl.tiles_m), 0);
+    for (size_t pos = 0; pos < first.size(); ++pos) {
+      const Item& it = items[(size_t)first[pos]];
+      ready[(size_t)it.job][(size_t)it.tm] = (int)pos;
+      ready_all[(size_t)it.job] = (int)pos;
+    }
+    for (int i = 0; i < n; ++i) {
+      const Item& it = items[(size_t)i];
+      const TcJob& j = jobs[(size_t)it.job];
+      if (j.stage == 0) continue;
+      const int d = dep_job[(size_t)it.job];
+      int r = 0;
+      if (d >= 0) r = j.link.dep_mode == 1 ? ready[(size_t)d][(size_t)std::min<int>(it.tm, (int)ready[(size_t)d].size() - 1)] : ready_all[(size_t)d];
+      key[(size_t)i] = ((int64_t)j.order_class << 60) | ((int64_t)r << 40) | (inv_cost(i) << 8) | (int64_t)it.job;
+    }
+    tc::build_chain_queue(stage, key, &gp.sched);
+  }
+  gp.sync = sync;
+  gp.sync_words = sync_words;
+  gp.side_need = side ? (unsigned)(2 * pairs * tc::kSideWarps) : 0u;
+  if (backward) return launch_chain_inst<false, true, tc::EPI_STORE, true, true, tc::EPI_WGRAD>(gp, pairs, flops, st);
+  return launch_chain_inst<false, false, tc::EPI_STORE, false, false, tc::EPI_STORE>(gp, pairs, flops, st);
 }
 
 
@@ -465,11 +623,10 @@ struct GroupShape { int bn, cta2; double items; };
 // Cost in SM cycles of running all jobs with one tile shape: rounds over the machine x (average
 // k-blocks per tile x the slower of MMA issue and shared-memory fill) + epilogues.  The fill rate
 // of an SM (about 50 B/clk) is what usually decides, which favours CTA pairs and wide tiles;
-// padding waste and the number of rounds pull the other way.  FLOP_TC_GROUP_BN / FLOP_TC_GROUP_CTA2
-// (1 = force pairs, 2 = forbid) override for tuning.
+// padding waste and the number of rounds pull the other way.
 GroupShape plan_group(const std::vector<Mnk>& jobs, bool b_mn_major, bool wgrad = false, bool pairs_only = false) {
-  static const int force_bn_all = env_int("FLOP_TC_GROUP_BN"), force_cta2_all = env_int("FLOP_TC_GROUP_CTA2");
-  static const int force_bn_w = env_int("FLOP_TC_WGRAD_BN"), force_cta2_w = env_int("FLOP_TC_WGRAD_CTA2");
+  const int force_bn_all = tuning().group_bn, force_cta2_all = tuning().group_cta2;
+  const int force_bn_w = tuning().wgrad_bn, force_cta2_w = tuning().wgrad_cta2;
   const int force_bn = wgrad && force_bn_w ? force_bn_w : force_bn_all;
   const int force_cta2 = wgrad && force_cta2_w ? force_cta2_w : force_cta2_all;
   const int sms = num_sms();
@@ -519,11 +676,8 @@ bool wgrad_direct_ok(const void* out, int64_t ldo, int wgrad_dt) {
 template <int TT>
 int launch_small_t_inst(const bf16* A, int64_t lda, const bf16* B, int64_t ldb, bf16* C, int64_t ldc, const float* cs, int T,
                         int N, int K, int k_pad, size_t smem, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    FLOP_CUDA(cudaFuncSetAttribute(small_t_gemm_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    configured = true;
-  }
+  static bool configured[kMaxDevices] = {};
+  if (first_use_on_device(configured)) FLOP_CUDA(cudaFuncSetAttribute(small_t_gemm_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
   const int grid = std::min((N + kSmallTWarps - 1) / kSmallTWarps, num_sms() * 4);
   launch_k(small_t_gemm_kernel<TT>, dim3(grid), dim3(32 * kSmallTWarps), smem, st, A, lda, B, ldb, C, ldc, cs, T, N, K, k_pad);
   count_launch();
@@ -532,7 +686,7 @@ int launch_small_t_inst(const bf16* A, int64_t lda, const bf16* B, int64_t ldb, 
 }
 int launch_small_t(const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc, const float* cs, int64_t T,
                    int64_t N, int64_t K, cudaStream_t st) {
-  static const int off = env_int("FLOP_NO_SMALL_T");
+  const int off = tuning().no_small_t;
   if (off || T < 1 || T > kSmallTMax || N > INT32_MAX || K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
   int tt = 1;
   while (tt < T) tt *= 2;
@@ -551,11 +705,8 @@ int launch_small_t(const void* A, int64_t lda, const void* B, int64_t ldb, void*
 template <int MT>
 int launch_skinny_inst(const bf16* A, int64_t lda, const bf16* B, int64_t ldb, bf16* C, int64_t ldc, const float* cs, int T, int N,
                        int K, int k_pad, size_t smem, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    FLOP_CUDA(cudaFuncSetAttribute(skinny_gemm_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    configured = true;
-  }
+  static bool configured[kMaxDevices] = {};
+  if (first_use_on_device(configured)) FLOP_CUDA(cudaFuncSetAttribute(skinny_gemm_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
   const int groups = (N + 7) / 8;
   const int grid = std::min((groups + kSkinnyWarps - 1) / kSkinnyWarps, num_sms() * 2);
   launch_k(skinny_gemm_kernel<MT>, dim3(grid), dim3(32 * kSkinnyWarps), smem, st, A, lda, B, ldb, C, ldc, cs, T, N, K, k_pad);
@@ -565,7 +716,7 @@ int launch_skinny_inst(const bf16* A, int64_t lda, const bf16* B, int64_t ldb, b
 }
 int launch_skinny(const void* A, int64_t lda, const void* B, int64_t ldb, void* C, int64_t ldc, const float* cs, int64_t T, int64_t N,
                   int64_t K, cudaStream_t st) {
-  static const int off = env_int("FLOP_NO_SKINNY");
+  const int off = tuning().no_skinny;
   if (off || T < 1 || T > kSkinnyMaxT || N > INT32_MAX || K > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
   const int mt = (int)((T + 15) / 16);
   const int k_pad = (int)round_up(K, 32);
@@ -682,7 +833,6 @@ static __device__ __align__(256) unsigned char g_l0_builtin_scratch[kNoAllocScra
 
 // In host code the array's name is only a handle; the device address comes from the runtime,
 // asked once per device with that device current.
-constexpr int kMaxDevices = 64;
 void* g_l0_builtin_ptr[kMaxDevices] = {};
 std::mutex g_l0_builtin_mu;
 
@@ -730,7 +880,7 @@ const char* flop_status_string(int status) {
   }
 }
 
-int flop_device_status(void* stream) {
+int flop_last_async_status(void* stream) {
   FLOP_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
   int v = 0;
   FLOP_CUDA(cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)));
@@ -740,6 +890,8 @@ int flop_device_status(void* stream) {
   }
   return v;
 }
+
+int flop_device_status(void* stream) { return flop_last_async_status(stream); }
 
 int flop_selftest_wait_timeout(int64_t limit_cycles, int* gave_up_dev, void* stream) {
   if (limit_cycles <= 0 || limit_cycles > 2000000000LL || !gave_up_dev) return FLOP_ERR_INVALID_ARG;
@@ -771,6 +923,18 @@ int flop_plan_tile_schedule(const double* cost, int32_t n, int32_t units, int32_
       for (int i = 0; i < n; ++i) unit_of_item[i] = i % units;
     }
   }
+  return FLOP_OK;
+}
+
+int flop_plan_chain_queue(const int32_t* stage, const int64_t* key, int32_t n, int32_t* queue_pos) {
+  if (n < 0 || (n > 0 && (!stage || !key)) || n > tc::kMaxSched) return FLOP_ERR_INVALID_ARG;
+  if (n == 0) return FLOP_OK;
+  static tc::Schedule sched;
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!tc::build_chain_queue(std::vector<int>(stage, stage + n), std::vector<int64_t>(key, key + n), &sched)) return FLOP_ERR_INVALID_ARG;
+  if (queue_pos)
+    for (int i = 0; i < n; ++i) queue_pos[sched.item[i]] = i;
   return FLOP_OK;
 }
 
@@ -1115,8 +1279,15 @@ int flop_gated_lowrank_bwd(const void* dY, int64_t lddy, const void* X, int64_t 
   return FLOP_OK;
 }
 
-int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, void* stream) {
+static int check_sync(const void* sync, size_t sync_bytes) {
+  if (!sync) return FLOP_OK;
+  if ((reinterpret_cast<uintptr_t>(sync) & 15) != 0 || sync_bytes < kSyncBytes) return FLOP_ERR_WORKSPACE;
+  return FLOP_OK;
+}
+
+static int fwd_grouped_impl(const flop_fwd_problem_t* pr, int n, int dt, void* sync, size_t sync_bytes, void* stream) {
   if (n < 0 || (n > 0 && !pr) || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  FLOP_TRY(check_sync(sync, sync_bytes));
   bool grouped = dt == FLOP_BF16;
   for (int i = 0; i < n; ++i) {
     const flop_fwd_problem_t& a = pr[i];
@@ -1157,13 +1328,55 @@ int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, 
     g2.push_back(j2);
   }
   cudaStream_t st = (cudaStream_t)stream;
+  // One launch for both products when the caller brought a sync area: every problem's first product publishes
+  // its 256-row blocks of H', the tiles of the second wait for the block they read.
+  {
+    size_t words = tc::kSyncFixed;
+    std::vector<TcJob> all;
+    std::vector<int> dep_job;
+    for (int i = 0; i < n; ++i) {
+      TcJob j = g1[(size_t)i];
+      j.stage = 0; j.order_class = 0;
+      j.link.sig = (unsigned*)sync + words;
+      words += (size_t)j.pl.tiles_m;
+      all.push_back(j);
+      dep_job.push_back(-1);
+    }
+    for (int i = 0; i < n; ++i) {
+      TcJob j = g2[(size_t)i];
+      const TcJob& src = all[(size_t)i];
+      j.stage = 1; j.order_class = 0;
+      j.link.dep = src.link.sig; j.link.dep_mode = 1;
+      j.link.dep_n_cap = (int)src.N; j.link.dep_bn = src.pl.bn; j.link.dep_dyn_n = src.dyn_n;
+      all.push_back(j);
+      dep_job.push_back(i);
+    }
+    if (chain_ok(all, sync, sync_bytes, words)) return launch_tc_chain(all, dep_job, (unsigned*)sync, (int)words, false, st);
+  }
   FLOP_TRY(launch_tc_group(g1, st));   // H' = (X Q^T) * z for every problem
   FLOP_TRY(launch_tc_group(g2, st));   // Y = H' P^T
   return FLOP_OK;
 }
 
-int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accumulate, int dt, int wgrad_dt, void* stream) {
+int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* pr, int n, int dt, void* stream) {
+  return fwd_grouped_impl(pr, n, dt, nullptr, 0, stream);
+}
+
+int flop_gated_lowrank_fwd_chained(const flop_fwd_problem_t* pr, int n, int dt, void* sync, size_t sync_bytes, void* stream) {
+  if (!sync) return FLOP_ERR_WORKSPACE;
+  return fwd_grouped_impl(pr, n, dt, sync, sync_bytes, stream);
+}
+
+int flop_sync_bytes(size_t* out_bytes) {
+  if (!out_bytes) return FLOP_ERR_INVALID_ARG;
+  *out_bytes = kSyncBytes;
+  return FLOP_OK;
+}
+
+static int bwd_grouped_impl(const flop_bwd_problem_t* pr, int n, int accumulate, int dt, int wgrad_dt, void* sync,
+                            size_t sync_bytes, void* stream) {
   if (n < 0 || (n > 0 && !pr) || !valid_dt(dt) || !valid_dt(wgrad_dt)) return FLOP_ERR_INVALID_ARG;
+  FLOP_TRY(check_sync(sync, sync_bytes));
   if (dt == FLOP_F32 && wgrad_dt != FLOP_F32) return FLOP_ERR_UNSUPPORTED;
   bool grouped = dt == FLOP_BF16;
   for (int i = 0; i < n; ++i) {
@@ -1193,8 +1406,9 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     if (!check_mat(a.dY, a.lddy, a.d_out) || !check_mat(a.X, a.ldx, a.d_in) || !check_mat(a.Q, a.ldq, a.d_in) ||
         !check_mat(a.P, a.ldp, a.r) || !a.z || !check_mat(a.H_save, a.ldh, a.r))
       return FLOP_ERR_INVALID_ARG;
+    if (a.Qz && a.ldqz < a.d_in) return FLOP_ERR_INVALID_ARG;
     if ((a.dX && !bf16_ok(a.dX, a.lddx)) || !bf16_ok(a.dY, a.lddy) || !bf16_ok(a.X, a.ldx) || !bf16_ok(a.Q, a.ldq) ||
-        !bf16_ok(a.P, a.ldp) || !bf16_ok(a.H_save, a.ldh))
+        !bf16_ok(a.P, a.ldp) || !bf16_ok(a.H_save, a.ldh) || (a.Qz && !bf16_ok(a.Qz, a.ldqz)))
       return FLOP_ERR_UNSUPPORTED;
     Arena probe{nullptr, 0, 0};
     FLOP_TRY(check_ws(a.ws, a.ws_bytes, plan_bwd_ws(probe, a.T, a.d_in, a.d_out, a.r, dt, true).bytes));
@@ -1269,11 +1483,12 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
     f.d_out = (int)a.d_out; f.r = (int)a.r; f.dP = direct ? nullptr : a.dP; f.lddp = a.lddp;
     f.slices_q = w.slices_q; f.n_slices_q = w.plan_q.splits; f.slice_elems_q = w.slice_elems_q; f.ld_slice_q = w.ld_slice_q;
     f.d_in = (int)a.d_in; f.dQ = direct ? nullptr : a.dQ; f.lddq = a.lddq; f.z = a.z;
-    f.Q = (const bf16*)a.Q; f.ldq = a.ldq; f.Qz = a.dX ? (bf16*)w.Qz : nullptr; f.ldqz = w.ldqz;
+    // diag(z) Q: the caller's (formed once per step by flop_scale_rows_grouped), else formed here in the workspace
+    f.Q = (const bf16*)a.Q; f.ldq = a.ldq; f.Qz = (a.dX && !a.Qz) ? (bf16*)w.Qz : nullptr; f.ldqz = w.ldqz;
     f.dz_part = w.dz_part; f.n_part = n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.dlog_alpha; f.accumulate = accumulate;
     fin.push_back(f);
     if (a.dX) {
-      TcJob j6{{w.dH, w.lddh, false}, {w.Qz, w.ldqz, true}, a.T, a.d_in, a.r, fixed_plan(a.T, a.d_in, a.r, s6.bn, s6.cta2),
+      TcJob j6{{w.dH, w.lddh, false}, {a.Qz ? a.Qz : w.Qz, a.Qz ? a.ldqz : w.ldqz, true}, a.T, a.d_in, a.r, fixed_plan(a.T, a.d_in, a.r, s6.bn, s6.cta2),
                store_epilogue(a.dX, a.lddx, nullptr)};
       j6.dyn_k = a.r_dev;
       g6.push_back(j6);
@@ -1301,11 +1516,67 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
   // Two balanced launches instead of three uneven ones (gemm_tc2_dual.cuh): the products that need only saved
   // tensors (dH' = dY P and dP = dY^T H') share the first work list, those that need dH' (dQ with the fused
   // <Q, .> row dots, and dX) the second.  diag(z) Q depends on nothing computed here and is formed first; the
-  // ordered second stage of dlog_alpha comes last.  FLOP_STAGE_MERGE=0 keeps the three-launch order.
-  static const char* merge_env = getenv("FLOP_STAGE_MERGE");
-  static const int merge_on = merge_env ? atoi(merge_env) : 1;
+  // ordered second stage of dlog_alpha comes last.
+  const int merge_on = tuning().stage_merge;
   const bool pairs_everywhere = !g3.empty() && g3[0].pl.cta2 && (g4.empty() || g4[0].pl.cta2) && (g5.empty() || g5[0].pl.cta2) &&
                                 (g6.empty() || g6[0].pl.cta2);
+  // With a sync area: the whole backward pass of the call in ONE launch.  dH' tiles publish their row blocks;
+  // dX tiles wait for the block they read and for diag(z) Q, which the launch forms as side work; dQ tiles wait
+  // block by block as their contraction over the tokens advances, and the last tile of every 32-row slab of dQ
+  // adds up the slab's dlog_alpha partials.  No small kernel before or after.
+  if (direct && pairs_everywhere && sync) {
+    size_t words = tc::kSyncFixed;
+    std::vector<TcJob> all;
+    std::vector<int> dep_job;
+    // queue order: dH' tiles (everything else waits for them), the long dP tiles, the long dQ tiles (by then all of
+    // dH' is written), and the short dX tiles last, so that the launch ends on short tiles
+    for (size_t i = 0; i < g3.size(); ++i) {     // one dH' job per problem, in problem order
+      TcJob j = g3[i];
+      j.stage = 0; j.order_class = 0;
+      j.link.sig = (unsigned*)sync + words;
+      words += (size_t)j.pl.tiles_m;
+      all.push_back(j);
+      dep_job.push_back(-1);
+    }
+    for (TcJob j : g4) { j.stage = 0; j.order_class = 1; all.push_back(j); dep_job.push_back(-1); }
+    // g5 / g6 hold one job per problem that asked for dQ or dlog_alpha / for dX, in problem order
+    size_t i6 = 0, i5 = 0;
+    for (int i = 0; i < n; ++i) {
+      const flop_bwd_problem_t& a = pr[i];
+      const TcJob& src = all[(size_t)i];
+      if (a.dQ || a.dlog_alpha) {
+        TcJob j = g5[i5++];
+        j.stage = 1; j.order_class = 0;
+        j.link.dep = src.link.sig; j.link.dep_mode = 2;
+        j.link.dep_n_cap = (int)src.N; j.link.dep_bn = src.pl.bn; j.link.dep_dyn_n = src.dyn_n;
+        if (a.dlog_alpha) {
+          j.link.fin = (unsigned*)sync + words;
+          words += (size_t)j.pl.tiles_m * 8;
+          j.link.dz_dla = a.dz_dla; j.link.dla = a.dlog_alpha; j.link.dla_accumulate = accumulate;
+        }
+        all.push_back(j);
+        dep_job.push_back(i);
+      }
+    }
+    for (int i = 0; i < n; ++i) {
+      const flop_bwd_problem_t& a = pr[i];
+      const TcJob& src = all[(size_t)i];
+      if (a.dX) {
+        TcJob j = g6[i6++];
+        j.stage = 1; j.order_class = 1;
+        j.link.dep = src.link.sig; j.link.dep_mode = 1;
+        j.link.dep_n_cap = (int)src.N; j.link.dep_bn = src.pl.bn; j.link.dep_dyn_n = src.dyn_n;
+        if (!a.Qz) {     // no diag(z) Q from the caller: the launch's helper warps form it in the workspace
+          j.link.side_dep = 1;
+          j.link.sw_q = (const bf16*)a.Q; j.link.sw_ldq = a.ldq; j.link.sw_qz = (bf16*)wss[(size_t)i].Qz; j.link.sw_ldqz = wss[(size_t)i].ldqz;
+          j.link.sw_z = a.z; j.link.sw_rows = (int)a.r; j.link.sw_cols = (int)a.d_in;
+        }
+        all.push_back(j);
+        dep_job.push_back(i);
+      }
+    }
+    if (chain_ok(all, sync, sync_bytes, words)) return launch_tc_chain(all, dep_job, (unsigned*)sync, (int)words, true, st);
+  }
   if (direct && merge_on && pairs_everywhere && g3.size() + g4.size() <= (size_t)tc::kMaxGroup &&
       g5.size() + g6.size() <= (size_t)tc::kMaxGroup) {
     std::vector<BwdFinishArgs> pre = fin, post = fin;
@@ -1328,6 +1599,42 @@ int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accu
   FLOP_TRY(launch_tc_group(g5, st));   // dH'^T X slices + fused <Q, .> row dots
   FLOP_TRY(run_finish(fin));
   FLOP_TRY(launch_tc_group(g6, st));   // dX = dH' (diag(z) Q)
+  return FLOP_OK;
+}
+
+int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* pr, int n, int accumulate, int dt, int wgrad_dt, void* stream) {
+  return bwd_grouped_impl(pr, n, accumulate, dt, wgrad_dt, nullptr, 0, stream);
+}
+
+int flop_gated_lowrank_bwd_chained(const flop_bwd_problem_t* pr, int n, int accumulate, int dt, int wgrad_dt, void* sync,
+                                   size_t sync_bytes, void* stream) {
+  if (!sync) return FLOP_ERR_WORKSPACE;
+  return bwd_grouped_impl(pr, n, accumulate, dt, wgrad_dt, sync, sync_bytes, stream);
+}
+
+int flop_scale_rows_grouped(const flop_scale_rows_t* pr, int n, int dt, void* stream) {
+  if (n < 0 || (n > 0 && !pr) || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  if (dt != FLOP_BF16) return FLOP_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int i0 = 0; i0 < n; i0 += kScaleGroup) {
+    ScaleRowsGroup g;
+    memset(&g, 0, sizeof(g));
+    for (; g.n < kScaleGroup && i0 + g.n < n; ++g.n) {
+      const flop_scale_rows_t& a = pr[i0 + g.n];
+      if (a.r < 0 || a.d_in < 0 || a.r > INT32_MAX || a.d_in > INT32_MAX) return FLOP_ERR_INVALID_ARG;
+      if (a.r > 0 && a.d_in > 0 && (!a.Q || !a.z || !a.Qz || a.ldq < a.d_in || a.ldqz < a.d_in)) return FLOP_ERR_INVALID_ARG;
+      if (a.r > 0 && a.d_in > 0 && (!bf16_ok(a.Q, a.ldq) || !bf16_ok(a.Qz, a.ldqz))) return FLOP_ERR_UNSUPPORTED;
+      ScaleRows& o = g.a[g.n];
+      o.Q = (const bf16*)a.Q; o.ldq = a.ldq; o.z = a.z; o.Qz = (bf16*)a.Qz; o.ldqz = a.ldqz; o.rows = (int)a.r; o.cols = (int)a.d_in;
+      g.unit_begin[g.n + 1] = g.unit_begin[g.n] + (int64_t)o.rows * ((o.cols + 7) >> 3);
+    }
+    const int64_t units = g.unit_begin[g.n];
+    if (units <= 0) continue;
+    const int grid = (int)std::min<int64_t>((units + 4 * 256 - 1) / (4 * 256), (int64_t)num_sms() * 8);
+    launch_k(scale_rows_group_kernel, dim3(grid), dim3(256), (size_t)0, st, g);
+    count_launch();
+    FLOP_CUDA(cudaGetLastError());
+  }
   return FLOP_OK;
 }
 
@@ -1586,9 +1893,8 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
     if (smem > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
     if (dt == FLOP_BF16) {
       if (d_in > 0) launch_k(gather_q_kernel<bf16>, dim3((unsigned)r), dim3(256), (size_t)(0), st, (const bf16*)Q, ldq, idx, k_dev, zsrc, (int)d_in, (bf16*)Qc, ldqc, vq);
-      // rows staged by bulk asynchronous copies when they are 16-byte pieces; FLOP_GATHER_PIPE=0 keeps the plain kernel
-      static const char* pipe_env = getenv("FLOP_GATHER_PIPE");
-      static const int pipe_on = pipe_env ? atoi(pipe_env) : 1;
+      // rows staged by bulk asynchronous copies when they are 16-byte pieces
+      const int pipe_on = tuning().gather_pipe;
       if (d_out > 0 && pipe_on && vp && r % 8 == 0) {
         const size_t row_bytes = (size_t)r * 2, idx_bytes = (row_bytes + 127) & ~(size_t)127;
         int rows_per_stage = (int)std::max<size_t>(1, std::min<size_t>(16, (16 * 1024) / row_bytes));
@@ -1597,11 +1903,9 @@ int flop_compact_ranks(const float* log_alpha_or_z, int mode, flop_hc_params_t h
         while (nbuf > 2 && need(nbuf) > 100 * 1024) --nbuf;   // two blocks per SM where the rows allow it
         if (need(nbuf) <= (size_t)kSmemBudget) {
           const size_t sm = need(nbuf);
-          static size_t configured = 0;
-          if (sm > 48 * 1024 && sm > configured) {
+          static bool configured[kMaxDevices] = {};
+          if (sm > 48 * 1024 && first_use_on_device(configured))
             FLOP_CUDA(cudaFuncSetAttribute(gather_p_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
-            configured = (size_t)kSmemBudget;
-          }
           const int64_t groups = (d_out + rows_per_stage - 1) / rows_per_stage;
           const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(8, (size_t)(224 * 1024) / sm));
           const int grid = (int)std::min<int64_t>(groups, (int64_t)num_sms() * per_sm);

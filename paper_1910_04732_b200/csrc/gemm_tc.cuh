@@ -44,6 +44,22 @@ constexpr uint32_t kTmemCols = 512;
 constexpr long long kWaitCycles = 2000000000LL;   // ~1 s
 constexpr uint32_t kStoreBufBytes = 32 * 128;      // one epilogue warp's staging tile: 32 rows x 64 bf16
 
+// Links between the problems of a chained launch (gemm_tc2_chain.cuh); all-zero for every other launch.
+struct ChainLink {
+  // producing side: every epilogue warp adds 1 to sig[tm] (tm = 256-row block) once its part of the tile is written
+  unsigned* sig;
+  // consuming side: the TMA producer waits until dep[row block] has 16 arrivals per N tile of the producing
+  // problem.  dep_mode 1: the A operand is row block tm of that output; 2: the contraction runs over its rows.
+  const unsigned* dep; int dep_mode;
+  int dep_n_cap, dep_bn; const int* dep_dyn_n;     // N, N tile and device-side N (nullable) of the producing problem
+  int side_dep;                                     // 1: the B operand is the diag(z) Q this launch forms as side work
+  // side work asked for by this problem: sw_qz[k, :] = sw_z[k] * sw_q[k, :]  (sw_rows x sw_cols, bf16)
+  const __nv_bfloat16* sw_q; int64_t sw_ldq; __nv_bfloat16* sw_qz; int64_t sw_ldqz; const float* sw_z; int sw_rows, sw_cols;
+  // second stage of dlog_alpha inside the launch: fin[(tm*2 + cta)*4 + lane quarter] counts the N tiles of a 32-row
+  // slab; the last arrival writes dla[row] (=|+=) dz_dla[row] * sum of the slab's partial row dots
+  unsigned* fin; const float* dz_dla; float* dla; int dla_accumulate;
+};
+
 struct Params {
   int M, N, K;
   int bn;                 // N per tile: 64, 128, 192 or 256
@@ -66,6 +82,7 @@ struct Params {
   // multiple of 64.  An effective size of 0 is treated as 1 (an all-zero block).
   const int* dyn_m; const int* dyn_n; const int* dyn_k;
   int kind;   // 0 or 1: which of the two compile-time configurations of gemm2_dual_kernel serves this problem
+  ChainLink link;
 };
 
 enum { EPI_STORE = 0, EPI_SLICE = 1, EPI_WGRAD = 2 };

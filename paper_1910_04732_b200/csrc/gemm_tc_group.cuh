@@ -20,7 +20,7 @@
 namespace flop {
 namespace tc {
 
-constexpr int kMaxGroup = 16;   // 16 x 576 B of kernel parameters (the limit is 32 KB)
+constexpr int kMaxGroup = 24;   // the four products of six matrices; 24 x 704 B of kernel parameters (the limit is 32 KB)
 
 struct alignas(64) GroupProblem {
   CUtensorMap ta, tb;
@@ -39,6 +39,9 @@ struct GroupParams {
   // dependency wait, [1] = the latest %globaltimer at which a CTA finished (atomic max).  Lets a
   // caller time launches that run inside a replayed CUDA graph, where host events cannot be placed.
   unsigned long long* stamp;
+  // Chained launches only (gemm_tc2_chain.cuh): the zero-initialised sync area, the words in use (the last
+  // unit to finish clears them) and the arrivals that complete the launch's side work (0: none).
+  unsigned* sync; int sync_words; unsigned side_need;
   // Which work items each persistent unit walks (schedule.cuh); n_units == 0: round-robin.
   Schedule sched;
 };

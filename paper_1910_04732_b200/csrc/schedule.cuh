@@ -79,5 +79,31 @@ inline double build_schedule(const std::vector<double>& cost, int units, Schedul
   return makespan;
 }
 
+// Queue of a chained launch (gemm_tc2_chain.cuh): the work list holds the tiles of two stages, a tile of the
+// second stage waits for first-stage tiles, and the persistent units draw tiles from the head of one queue.
+// All first-stage tiles must therefore come before all second-stage tiles (a drawn tile then only waits for
+// tiles that some unit already works on, so no wait can be circular).  Inside a stage the queue follows `key`
+// (ties keep list order): the caller puts first what other tiles wait for, long tiles before short ones, and
+// orders consumers like their producers.  out->item holds the queue (n_units = 1 marks the table as valid).
+// Returns false when the table cannot hold the launch (the kernel then walks the work list in its own order,
+// which the caller keeps stage-ordered).
+inline bool build_chain_queue(const std::vector<int>& stage, const std::vector<int64_t>& key, Schedule* out) {
+  const int n = (int)stage.size();
+  out->n_units = 0;
+  if (n == 0 || n > kMaxSched || (int)key.size() != n) return false;
+  std::vector<int> order((size_t)n);
+  for (int i = 0; i < n; ++i) order[(size_t)i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    const int sa = stage[(size_t)a] != 0, sb = stage[(size_t)b] != 0;
+    if (sa != sb) return sa < sb;
+    return key[(size_t)a] < key[(size_t)b];
+  });
+  for (int i = 0; i < n; ++i) out->item[i] = (uint16_t)order[(size_t)i];
+  out->begin[0] = 0;
+  for (int u = 1; u <= kMaxUnits; ++u) out->begin[u] = (uint16_t)n;
+  out->n_units = 1;
+  return true;
+}
+
 }  // namespace tc
 }  // namespace flop

@@ -6,7 +6,7 @@ import torch
 
 from oracle import flop_oracle as O
 from paper_1910_04732_b200 import inputs as I
-from tests._util import HC, empty_dev, host, rel_fro, to_dev
+from tests._util import HC, assert_close, empty_dev, host, rel_fro, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -48,9 +48,7 @@ def _check_against_oracle(e, tag):
     for name, got, want in (("H", e["H" + tag], Hp), ("Y", e["Y" + tag], Y), ("dX", e["dX" + tag], G["dX"]),
                             ("dP", e["dP" + tag], G["dP"]), ("dQ", e["dQ" + tag], G["dQ"]),
                             ("dla", e["dla" + tag], G["dlog_alpha"])):
-        g = host(got)
-        assert np.all(np.isfinite(g)), name
-        assert rel_fro(g, want) < 2e-2, (e["m"], name, rel_fro(g, want))
+        assert_close(got, want, "bf16", f"{e['m'].name}.{name}")
 
 
 @pytest.mark.parametrize("wgrad", [torch.bfloat16, torch.float32])
@@ -97,16 +95,17 @@ def test_more_problems_than_one_launch_holds_and_optional_outputs(b):
     for i, e in enumerate(es):
         p = e["prob"]
         G = O.gated_lowrank_bwd(p["dY"], p["X"], p["Q"], p["P"], e["z_np"], e["dzd_np"])
+        # accumulating outputs hold bf16(0.25 + g): they are compared as stored, against 0.25 + the oracle's g
         if i % 3 != 0:
-            assert rel_fro(host(e["dXg"]), G["dX"]) < 2e-2
+            assert_close(e["dXg"], G["dX"], "bf16", "dX")
         else:
             assert torch.isnan(e["dXg"]).all()                      # untouched
         if i % 4 != 1:
-            assert rel_fro(host(e["dPg"]) - 0.25, G["dP"]) < 3e-2
+            assert_close(e["dPg"], G["dP"] + 0.25, "bf16", "dP")
         else:
             assert torch.all(e["dPg"] == 0.25)
-        assert rel_fro(host(e["dQg"]) - 0.25, G["dQ"]) < 3e-2
-        assert rel_fro(host(e["dlag"]) - 0.25, G["dlog_alpha"]) < 2e-2
+        assert_close(e["dQg"], G["dQ"] + 0.25, "bf16", "dQ")
+        assert_close(e["dlag"], G["dlog_alpha"] + 0.25, "bf16", "dla")
 
 
 def test_grouped_falls_back_per_problem_for_fp32_and_empty_problems(b):
@@ -165,13 +164,13 @@ def test_two_launch_backward_with_optional_outputs(b):
         if i in (1, 5):
             assert torch.isnan(e["dXg"]).all()
         else:
-            assert rel_fro(host(e["dXg"]), G["dX"]) < 2e-2
+            assert_close(e["dXg"], G["dX"], "bf16", "dX")
         if i in (2, 5):
             assert torch.isnan(e["dPg"]).all()
         else:
-            assert rel_fro(host(e["dPg"]), G["dP"]) < 2e-2
-        assert rel_fro(host(e["dQg"]), G["dQ"]) < 2e-2
+            assert_close(e["dPg"], G["dP"], "bf16", "dP")
+        assert_close(e["dQg"], G["dQ"], "bf16", "dQ")
         if i == 3:
             assert torch.isnan(e["dlag"]).all()
         else:
-            assert rel_fro(host(e["dlag"]), G["dlog_alpha"]) < 2e-2
+            assert_close(e["dlag"], G["dlog_alpha"], "bf16", "dla")

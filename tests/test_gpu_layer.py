@@ -10,7 +10,7 @@ import torch
 
 from oracle import flop_oracle as O
 from paper_1910_04732_b200 import inputs as I
-from tests._util import HC, empty_dev, host, rel_fro, to_dev
+from tests._util import HC, assert_close, empty_dev, host, rel_fro, to_dev
 
 pytestmark = pytest.mark.gpu
 TOL = {"f32": 1e-5, "bf16": 2e-2}
@@ -59,11 +59,9 @@ def run_layer(b, prob, dtype, seed=0, offset=0, wgrad_dtype=None, accumulate=Fal
         for k in ("dP", "dQ", "dlog_alpha"):
             ref[k] = ref[k] + 0.5
     if check:
-        tol = TOL[dtype]
+        # global relative Frobenius error (1e-5 / 2e-2) plus per-block and per-element bounds
         for k in ("Hp", "Y", "dX", "dP", "dQ", "dlog_alpha"):
-            assert np.all(np.isfinite(gpu[k])), k
-            err = rel_fro(gpu[k], ref[k])
-            assert err < tol, f"{k}: rel. Frobenius error {err:.3e} >= {tol}"
+            assert_close(gpu[k], ref[k], dtype, k)
     return gpu, ref
 
 
