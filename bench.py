@@ -170,13 +170,19 @@ class Job:
                 chunk = self.mats[i:i + group]
                 fwd = b.problem_array([b.fwd_problem(e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]], e["Y"], e["H"])
                                        for e in chunk])
-                bwd = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]],
-                                                     self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
-                                                     self.dlog_alpha[e["lo"]:e["hi"]], e["ws"], Qz=e["Qz"]) for e in chunk])
-                bwd_plain = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]],
-                                                           self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
-                                                           self.dlog_alpha[e["lo"]:e["hi"]], e["ws"]) for e in chunk])
-                self.groups.append((fwd, bwd, bwd_plain))
+                mk = lambda e, **kw: b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]],
+                                                   self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
+                                                   self.dlog_alpha[e["lo"]:e["hi"]], e["ws"], **kw)
+                # default: diag(z) Q comes from the one launch after sampling, the second stage of dlog_alpha is left
+                # to the one launch at the end of the step; "plain": every backward call does both itself
+                bwd = b.problem_array([mk(e, Qz=e["Qz"], defer_dlog_alpha=True) for e in chunk])
+                bwd_chain = b.problem_array([mk(e, Qz=e["Qz"]) for e in chunk])
+                bwd_plain = b.problem_array([mk(e) for e in chunk])
+                self.groups.append((fwd, bwd, bwd_chain, bwd_plain))
+            self.bwd_all = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], self.z[e["lo"]:e["hi"]],
+                                                          self.dz_dla[e["lo"]:e["hi"]], e["H"], e["dX"], e["dP"], e["dQ"],
+                                                          self.dlog_alpha[e["lo"]:e["hi"]], e["ws"], Qz=e["Qz"],
+                                                          defer_dlog_alpha=True) for e in self.mats])
         # data parallelism: one gradient bucket per grouped call (a layer), reduced while later layers compute
         n_per = group if group > 0 else len(self.mats)
         sizes_w = [e["dP"].shape[0] * r8(e["m"].r) + e["m"].r * r8(e["m"].d_in) for e in self.mats]
@@ -190,6 +196,7 @@ class Job:
         self.world = 1
         # chained calls: one launch for the two forward products, one for the whole backward pass of a layer
         self.chain = False
+        self.plain = False
         self.sync = b.alloc_sync(device)
 
     def enable_active_ranks(self):
@@ -250,7 +257,9 @@ class Job:
         self.b.gate_sample_devoff(self.log_alpha, HC, 0, 0, self.offset_dev, self.z, self.mask, self.dz_dla)
         self.offset_dev.add_(1 << 24)
 
-    def finish(self):
+    def finish(self, deferred=False):
+        if deferred:
+            self.b.dlog_alpha_finish_grouped(self.bwd_all)            # second stage of dlog_alpha, all matrices, one launch
         self.b.expected_l0_lagrangian(self.log_alpha, self.seg_off, self.seg_size, HC, self.target, self.lam,
                                       self.out4, None, self.dlog_alpha, self.ws_l0)
         if self.world > 1:
@@ -268,15 +277,15 @@ class Job:
             if self.world > 1 and self.reducer is None:
                 from paper_1910_04732_b200 import dp
                 self.reducer = dp.BucketedReducer(self.wgrad, self.bucket_bounds)
-            if self.chain:
+            if not self.plain:
                 self.b.scale_rows_grouped(self.scale)                 # diag(z) Q of every matrix: one launch per step
-            for i, (fwd, bwd, bwd_plain) in enumerate(self.groups):
+            for i, (fwd, bwd, bwd_chain, bwd_plain) in enumerate(self.groups):
                 if self.chain:
                     self.b.gated_lowrank_fwd_chained(fwd, self.sync)
-                    self.b.gated_lowrank_bwd_chained(bwd, self.sync)
+                    self.b.gated_lowrank_bwd_chained(bwd_chain, self.sync)
                 else:
                     self.b.gated_lowrank_fwd_grouped(fwd)
-                    self.b.gated_lowrank_bwd_grouped(bwd_plain)
+                    self.b.gated_lowrank_bwd_grouped(bwd_plain if self.plain else bwd)
                 if self.reducer is not None:
                     self.reducer.launch(i)                            # this layer's dP, dQ are final
         elif self.n_streams == 1:
@@ -294,7 +303,7 @@ class Job:
             for k, s in enumerate(self.streams):
                 self.ev_done[k].record(s)
                 main.wait_event(self.ev_done[k])
-        self.finish()
+        self.finish(deferred=self.group > 0 and not self.chain and not self.plain)
 
 
 def capture_step(job: Job, fn=None, stamps=None):
@@ -456,6 +465,8 @@ def main():
     ap.add_argument("--chain", action="store_true", help="chained calls (one launch for the forward products, one for the backward pass of a layer, "
                     "ordered on the device) instead of the grouped calls (a launch per GEMM stage); measured slower on B200, see profiles/")
     ap.add_argument("--no-chain", action="store_true", help="(default) grouped calls")
+    ap.add_argument("--plain", action="store_true", help="every backward call forms diag(z) Q and finishes dlog_alpha itself "
+                    "(two more small launches per layer) instead of one launch per step for each")
     ap.add_argument("--group", type=int, default=-1, help="matrices per grouped call (0: one call per matrix; default: one layer)")
     ap.add_argument("--streams", type=int, default=1, help="streams over which independent matrices are issued")
     args = ap.parse_args()
@@ -486,6 +497,7 @@ def main():
     job = Job(w, torch.device("cuda", local), seed=1234 + rank, n_streams=args.streams, group=group)
     job.world = world
     job.chain = bool(args.chain) and not args.no_chain
+    job.plain = bool(args.plain)
     for _ in range(args.warmup):
         job.step()
     torch.cuda.synchronize()

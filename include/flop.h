@@ -215,6 +215,7 @@ typedef struct {
   void* ws; size_t ws_bytes;
   const int32_t* r_dev; /* nullable */
   const void* Qz; int64_t ldqz; /* nullable: diag(z) Q formed beforehand by flop_scale_rows_grouped (same z, same Q) */
+  int32_t defer_dlog_alpha;     /* != 0: leave the partial row dots of dlog_alpha in ws; flop_dlog_alpha_finish_grouped adds them up */
 } flop_bwd_problem_t;
 
 /* diag(z) Q for n matrices in one launch: Qz[k, :] = z[k] * Q[k, :] (r x d_in, bf16, rounded once).  The
@@ -226,6 +227,15 @@ typedef struct {
   const void* Q; int64_t ldq; const float* z; void* Qz; int64_t ldqz; int64_t r, d_in;
 } flop_scale_rows_t;
 int flop_scale_rows_grouped(const flop_scale_rows_t* problems, int n, int dt, void* stream);
+
+/* Second stage of dlog_alpha for n problems in one launch (Section 3: alpha receives gradients with theta).  The
+ * grouped / chained backward calls fuse dz_k = <Q[k,:], (dH'^T X)[k,:]> into the dQ product as partial row dots;
+ * adding the partials and multiplying by dz_dla is a small second stage.  A problem with defer_dlog_alpha != 0
+ * leaves its partials in its workspace instead; this call then writes dlog_alpha (=|+= with accumulate) for every
+ * problem given, in fixed summation order.  Pass the same problem structs (ws, sizes, dz_dla, dlog_alpha) as to the
+ * backward calls, any number of them together (e.g. all matrices of a model once per step); a workspace must not be
+ * reused by another backward call in between.  bf16 only.  HOST array. */
+int flop_dlog_alpha_finish_grouped(const flop_bwd_problem_t* problems, int n, int accumulate, int dt, void* stream);
 
 int flop_gated_lowrank_fwd_grouped(const flop_fwd_problem_t* problems, int n, int dt, void* stream);
 int flop_gated_lowrank_bwd_grouped(const flop_bwd_problem_t* problems, int n, int accumulate, int dt,

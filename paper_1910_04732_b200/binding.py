@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD, OP_EMBEDDING_BWD = range(6)
 
 EXPORTS = ("flop_status_string", "flop_last_async_status", "flop_device_status", "flop_sync_bytes",
-           "flop_gated_lowrank_fwd_chained", "flop_gated_lowrank_bwd_chained", "flop_selftest_wait_timeout", "flop_launch_count", "flop_plan_tile_schedule", "flop_plan_chain_queue", "flop_scale_rows_grouped", "flop_gemm_timing_begin",
+           "flop_gated_lowrank_fwd_chained", "flop_gated_lowrank_bwd_chained", "flop_selftest_wait_timeout", "flop_launch_count", "flop_plan_tile_schedule", "flop_plan_chain_queue", "flop_scale_rows_grouped", "flop_dlog_alpha_finish_grouped", "flop_gemm_timing_begin",
            "flop_gemm_timing_end", "flop_gemm_stamps_begin", "flop_gemm_stamps_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
@@ -51,7 +51,7 @@ class BwdProblem(ctypes.Structure):
                 ("dQ", ctypes.c_void_p), ("lddq", ctypes.c_int64), ("dlog_alpha", ctypes.c_void_p),
                 ("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
                 ("ws", ctypes.c_void_p), ("ws_bytes", ctypes.c_size_t), ("r_dev", ctypes.c_void_p),
-                ("Qz", ctypes.c_void_p), ("ldqz", ctypes.c_int64)]
+                ("Qz", ctypes.c_void_p), ("ldqz", ctypes.c_int64), ("defer_dlog_alpha", ctypes.c_int32)]
 
 
 class ScaleRows(ctypes.Structure):
@@ -110,6 +110,7 @@ def load_library() -> ctypes.CDLL:
     lib.flop_plan_chain_queue.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32,
                                           ctypes.POINTER(ctypes.c_int32)]
     lib.flop_scale_rows_grouped.argtypes = [ctypes.POINTER(ScaleRows), ci, ci, vp]
+    lib.flop_dlog_alpha_finish_grouped.argtypes = [ctypes.POINTER(BwdProblem), ci, ci, ci, vp]
     lib.flop_selftest_wait_timeout.argtypes = [i64, vp, vp]
     lib.flop_gemm_timing_begin.argtypes = []
     lib.flop_gemm_timing_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
@@ -317,13 +318,20 @@ def fwd_problem(X, Q, P, z, Y, H_save, r_dev=None) -> FwdProblem:
                       T, d_in, d_out, r, _p(r_dev))
 
 
-def bwd_problem(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws, r_dev=None, Qz=None) -> BwdProblem:
+def bwd_problem(dY, X, Q, P, z, dz_dla, H_save, dX, dP, dQ, dlog_alpha, ws, r_dev=None, Qz=None,
+                defer_dlog_alpha: bool = False) -> BwdProblem:
     T, d_in = X.shape
     d_out, r = P.shape
     ld = lambda t: _ld(t) if t is not None else 0
     return BwdProblem(_p(dY), _ld(dY), _p(X), _ld(X), _p(Q), _ld(Q), _p(P), _ld(P), _p(z), _p(dz_dla), _p(H_save),
                       _ld(H_save), _p(dX), ld(dX), _p(dP), ld(dP), _p(dQ), ld(dQ), _p(dlog_alpha), T, d_in, d_out, r,
-                      _p(ws), ws.numel() if ws is not None else 0, _p(r_dev), _p(Qz), ld(Qz))
+                      _p(ws), ws.numel() if ws is not None else 0, _p(r_dev), _p(Qz), ld(Qz), int(defer_dlog_alpha))
+
+
+def dlog_alpha_finish_grouped(problems, accumulate: bool = False, dt: int = BF16) -> None:
+    arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
+    _check(load_library().flop_dlog_alpha_finish_grouped(arr, len(arr), int(accumulate), dt, _stream()),
+           "flop_dlog_alpha_finish_grouped")
 
 
 def scale_rows_problem(Q, z, Qz) -> ScaleRows:

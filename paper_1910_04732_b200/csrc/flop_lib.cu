@@ -69,9 +69,10 @@ inline bool debug_on() {
 //   FLOP_NO_SMALL_T=1, FLOP_NO_SKINNY=1   few-token forward kernels off
 //   FLOP_STAGE_MERGE=0     backward in three launches per stage instead of two shared ones
 //   FLOP_GATHER_PIPE=0     plain P gather kernel                     FLOP_NO_CHAIN=1   chained calls run unchained
+//   FLOP_CHAIN_STAGES=2    chained calls put dependent products in ONE launch (default 1: a launch per stage)
 struct Tuning {
   int no_pdl = 0, tc_bn = 0, tc_stages = 0, tc_cta2 = 0, no_tma_store = 0, no_sched = 0, group_bn = 0, group_cta2 = 0,
-      wgrad_bn = 0, wgrad_cta2 = 0, no_small_t = 0, no_skinny = 0, stage_merge = 1, gather_pipe = 1, no_chain = 0;
+      wgrad_bn = 0, wgrad_cta2 = 0, no_small_t = 0, no_skinny = 0, stage_merge = 1, gather_pipe = 1, no_chain = 0, chain_stages = 1;
 };
 inline const Tuning& tuning() {
   static const Tuning t = [] {
@@ -83,6 +84,7 @@ inline const Tuning& tuning() {
     v.group_bn = get("FLOP_TC_GROUP_BN", 0); v.group_cta2 = get("FLOP_TC_GROUP_CTA2", 0); v.wgrad_bn = get("FLOP_TC_WGRAD_BN", 0);
     v.wgrad_cta2 = get("FLOP_TC_WGRAD_CTA2", 0); v.no_small_t = get("FLOP_NO_SMALL_T", 0); v.no_skinny = get("FLOP_NO_SKINNY", 0);
     v.stage_merge = get("FLOP_STAGE_MERGE", 1); v.gather_pipe = get("FLOP_GATHER_PIPE", 1); v.no_chain = get("FLOP_NO_CHAIN", 0);
+    v.chain_stages = get("FLOP_CHAIN_STAGES", 1);
 #endif
     return v;
   }();
@@ -312,7 +314,7 @@ struct TcEpilogue {
   int kind;   // tc::EPI_STORE or tc::EPI_SLICE
   bf16* out; int64_t ldo; const float* col_scale;
   float* slices; int64_t slice_elems, ld_slice;
-  const bf16* qdot; int64_t ldq; float* dz_part; int64_t dz_stride;
+  const bf16* qdot; int64_t ldq; float* dz_part; int64_t dz_stride; int* dz_meta;
   void* wg_out; int wg_f32; const float* row_scale; int accumulate;   // tc::EPI_WGRAD (ldo is shared with out)
 };
 
@@ -414,7 +416,7 @@ int add_problem(tc::GroupParams& gp, const TcJob& j, std::vector<double>& item_c
   p.splits = j.pl.splits; p.kb_per_split = j.pl.kb_per_split; p.num_kb = j.pl.num_kb;
   p.out = j.ep.out; p.ldo = j.ep.ldo; p.col_scale = j.ep.col_scale;
   p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
-  p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride;
+  p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride; p.dz_meta = j.ep.dz_meta;
   p.wg_out = j.ep.wg_out; p.wg_f32 = j.ep.wg_f32; p.row_scale = j.ep.row_scale; p.accumulate = j.ep.accumulate;
   p.dyn_m = j.dyn_m; p.dyn_n = j.dyn_n; p.dyn_k = j.dyn_k;
   p.link = j.link;
@@ -778,6 +780,7 @@ struct BwdWs {
   float* slices_p; float* slices_q;   // fp32 split-K slices of dY^T H' and dH'^T X
   int64_t ld_slice_p, ld_slice_q, slice_elems_p, slice_elems_q;
   float* dz_part; int n_part;
+  int* dz_meta;                  // device word: partial vectors the last backward call left in dz_part
   TcPlan plan_p, plan_q;
   size_t bytes;
 };
@@ -805,6 +808,7 @@ BwdWs plan_bwd_ws(Arena& ar, int64_t T, int64_t d_in, int64_t d_out, int64_t r, 
   // room for the partials of any tile shape: the direct-epilogue path may use another N tile than plan_q
   const int64_t part_cap = std::max<int64_t>(w.n_part, 2 * ((d_in + 63) / 64));
   w.dz_part = (float*)ar.take((size_t)part_cap * std::max<int64_t>(r, 1) * 4);
+  w.dz_meta = (int*)ar.take(256);
   w.bytes = ar.used;
   return w;
 }
@@ -1351,7 +1355,13 @@ static int fwd_grouped_impl(const flop_fwd_problem_t* pr, int n, int dt, void* s
       all.push_back(j);
       dep_job.push_back(i);
     }
-    if (chain_ok(all, sync, sync_bytes, words)) return launch_tc_chain(all, dep_job, (unsigned*)sync, (int)words, false, st);
+    if (chain_ok(all, sync, sync_bytes, words)) {
+      if (tuning().chain_stages >= 2) return launch_tc_chain(all, dep_job, (unsigned*)sync, (int)words, false, st);
+      // a launch per product, each drawing its tiles from a queue (nothing waits inside a launch)
+      const std::vector<int> none((size_t)n, -1);
+      FLOP_TRY(launch_tc_chain(g1, none, (unsigned*)sync, tc::kSyncFixed, false, st));
+      return launch_tc_chain(g2, none, (unsigned*)sync, tc::kSyncFixed, false, st);
+    }
   }
   FLOP_TRY(launch_tc_group(g1, st));   // H' = (X Q^T) * z for every problem
   FLOP_TRY(launch_tc_group(g2, st));   // Y = H' P^T
@@ -1387,7 +1397,7 @@ static int bwd_grouped_impl(const flop_bwd_problem_t* pr, int n, int accumulate,
   if (!grouped) {
     for (int i = 0; i < n; ++i) {
       const flop_bwd_problem_t& a = pr[i];
-      if (a.r_dev) return FLOP_ERR_UNSUPPORTED;
+      if (a.r_dev || a.defer_dlog_alpha) return FLOP_ERR_UNSUPPORTED;
       FLOP_TRY(flop_gated_lowrank_bwd(a.dY, a.lddy, a.X, a.ldx, a.Q, a.ldq, a.P, a.ldp, a.z, a.dz_dla, a.H_save, a.ldh, a.dX,
                                       a.lddx, a.dP, a.lddp, a.dQ, a.lddq, a.dlog_alpha, accumulate, a.T, a.d_in, a.d_out, a.r, dt,
                                       wgrad_dt, a.ws, a.ws_bytes, stream));
@@ -1473,7 +1483,7 @@ static int bwd_grouped_impl(const flop_bwd_problem_t* pr, int n, int accumulate,
       } else {
         e.kind = tc::EPI_SLICE; e.slices = w.slices_q; e.slice_elems = w.slice_elems_q; e.ld_slice = w.ld_slice_q;
       }
-      if (a.dlog_alpha) { e.qdot = (const bf16*)a.Q; e.ldq = a.ldq; e.dz_part = w.dz_part; e.dz_stride = a.r; }
+      if (a.dlog_alpha) { e.qdot = (const bf16*)a.Q; e.ldq = a.ldq; e.dz_part = w.dz_part; e.dz_stride = a.r; e.dz_meta = a.defer_dlog_alpha ? w.dz_meta : nullptr; }
       TcJob j5{{w.dH, w.lddh, true}, {a.X, a.ldx, true}, a.r, a.d_in, a.T, pl, e};
       j5.dyn_m = a.r_dev;
       g5.push_back(j5);
@@ -1485,7 +1495,7 @@ static int bwd_grouped_impl(const flop_bwd_problem_t* pr, int n, int accumulate,
     f.d_in = (int)a.d_in; f.dQ = direct ? nullptr : a.dQ; f.lddq = a.lddq; f.z = a.z;
     // diag(z) Q: the caller's (formed once per step by flop_scale_rows_grouped), else formed here in the workspace
     f.Q = (const bf16*)a.Q; f.ldq = a.ldq; f.Qz = (a.dX && !a.Qz) ? (bf16*)w.Qz : nullptr; f.ldqz = w.ldqz;
-    f.dz_part = w.dz_part; f.n_part = n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.dlog_alpha; f.accumulate = accumulate;
+    f.dz_part = w.dz_part; f.n_part = n_part; f.dz_dla = a.dz_dla; f.dlog_alpha = a.defer_dlog_alpha ? nullptr : a.dlog_alpha; f.accumulate = accumulate;
     fin.push_back(f);
     if (a.dX) {
       TcJob j6{{w.dH, w.lddh, false}, {a.Qz ? a.Qz : w.Qz, a.Qz ? a.ldqz : w.ldqz, true}, a.T, a.d_in, a.r, fixed_plan(a.T, a.d_in, a.r, s6.bn, s6.cta2),
@@ -1549,7 +1559,7 @@ static int bwd_grouped_impl(const flop_bwd_problem_t* pr, int n, int accumulate,
         j.stage = 1; j.order_class = 0;
         j.link.dep = src.link.sig; j.link.dep_mode = 2;
         j.link.dep_n_cap = (int)src.N; j.link.dep_bn = src.pl.bn; j.link.dep_dyn_n = src.dyn_n;
-        if (a.dlog_alpha) {
+        if (a.dlog_alpha && !a.defer_dlog_alpha) {
           j.link.fin = (unsigned*)sync + words;
           words += (size_t)j.pl.tiles_m * 8;
           j.link.dz_dla = a.dz_dla; j.link.dla = a.dlog_alpha; j.link.dla_accumulate = accumulate;
@@ -1575,7 +1585,29 @@ static int bwd_grouped_impl(const flop_bwd_problem_t* pr, int n, int accumulate,
         dep_job.push_back(i);
       }
     }
-    if (chain_ok(all, sync, sync_bytes, words)) return launch_tc_chain(all, dep_job, (unsigned*)sync, (int)words, true, st);
+    if (chain_ok(all, sync, sync_bytes, words)) {
+      if (tuning().chain_stages >= 2) return launch_tc_chain(all, dep_job, (unsigned*)sync, (int)words, true, st);
+      // Two launches (dH' with dP, then dQ with dX), each drawing its tiles from a queue; nothing waits inside a
+      // launch.  The second still finishes dlog_alpha by itself; diag(z) Q comes from the caller, else from the
+      // small kernel before the first launch.
+      std::vector<TcJob> one, two;
+      for (TcJob j : all) {
+        const bool second = j.stage != 0;
+        j.stage = 0; j.order_class = 0;      // no waits inside a launch: long tiles first
+        j.link.sig = nullptr; j.link.dep = nullptr; j.link.dep_mode = 0; j.link.side_dep = 0; j.link.sw_qz = nullptr;
+        (second ? two : one).push_back(j);
+      }
+      bool need_pre = false;
+      std::vector<BwdFinishArgs> pre = fin;
+      for (size_t i = 0; i < pre.size(); ++i) {
+        pre[i].dlog_alpha = nullptr;
+        if (pre[i].Qz) need_pre = true;
+      }
+      if (need_pre) FLOP_TRY(run_finish(pre));
+      FLOP_TRY(launch_tc_chain(one, std::vector<int>(one.size(), -1), (unsigned*)sync, tc::kSyncFixed, true, st));
+      if (!two.empty()) FLOP_TRY(launch_tc_chain(two, std::vector<int>(two.size(), -1), (unsigned*)sync, (int)words, true, st));
+      return FLOP_OK;
+    }
   }
   if (direct && merge_on && pairs_everywhere && g3.size() + g4.size() <= (size_t)tc::kMaxGroup &&
       g5.size() + g6.size() <= (size_t)tc::kMaxGroup) {
@@ -1610,6 +1642,36 @@ int flop_gated_lowrank_bwd_chained(const flop_bwd_problem_t* pr, int n, int accu
                                    size_t sync_bytes, void* stream) {
   if (!sync) return FLOP_ERR_WORKSPACE;
   return bwd_grouped_impl(pr, n, accumulate, dt, wgrad_dt, sync, sync_bytes, stream);
+}
+
+int flop_dlog_alpha_finish_grouped(const flop_bwd_problem_t* pr, int n, int accumulate, int dt, void* stream) {
+  if (n < 0 || (n > 0 && !pr) || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  if (dt != FLOP_BF16) return FLOP_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int i0 = 0; i0 < n; i0 += kDlaGroup) {
+    DlaFinishGroup g;
+    memset(&g, 0, sizeof(g));
+    int max_r = 0;
+    for (; g.n < kDlaGroup && i0 + g.n < n; ++g.n) {
+      const flop_bwd_problem_t& a = pr[i0 + g.n];
+      if (a.T < 0 || a.d_in < 0 || a.d_out < 0 || a.r < 0 || a.r > INT32_MAX) return FLOP_ERR_INVALID_ARG;
+      DlaFinish& o = g.a[g.n];
+      if (!a.dlog_alpha || a.T == 0 || a.r == 0 || a.d_in == 0 || a.d_out == 0) { o.r = 0; continue; }
+      if (!a.dz_dla) return FLOP_ERR_INVALID_ARG;
+      Arena probe{nullptr, 0, 0};
+      FLOP_TRY(check_ws(a.ws, a.ws_bytes, plan_bwd_ws(probe, a.T, a.d_in, a.d_out, a.r, dt, true).bytes));
+      Arena ar{(unsigned char*)a.ws, a.ws_bytes, 0};
+      const BwdWs w = plan_bwd_ws(ar, a.T, a.d_in, a.d_out, a.r, dt, true);
+      o.dz_part = w.dz_part; o.n_part = w.dz_meta; o.cap = (int)std::max<int64_t>(w.n_part, 2 * ((a.d_in + 63) / 64));
+      o.dz_dla = a.dz_dla; o.dla = a.dlog_alpha; o.r = (int)a.r;
+      max_r = std::max(max_r, o.r);
+    }
+    if (max_r == 0) continue;
+    launch_k(dalpha_group_kernel, dim3((unsigned)((max_r + 255) / 256), (unsigned)g.n), dim3(256), (size_t)0, st, g, accumulate);
+    count_launch();
+    FLOP_CUDA(cudaGetLastError());
+  }
+  return FLOP_OK;
 }
 
 int flop_scale_rows_grouped(const flop_scale_rows_t* pr, int n, int dt, void* stream) {

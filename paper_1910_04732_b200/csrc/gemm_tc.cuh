@@ -72,6 +72,7 @@ struct Params {
   float* slices; int64_t slice_elems; int64_t ld_slice;
   const __nv_bfloat16* qdot; int64_t ldq;      // nullable: dz_part[(split*tiles_n+tn)*dz_stride + m] = sum_n acc*qdot[m,n]
   float* dz_part; int64_t dz_stride;
+  int* dz_meta;                                // nullable: receives the number of partial vectors, 2 * tiles_n * splits
   // EPI_WGRAD (splits == 1): wg_out[m*ldo + n] (=|+=) row_scale[m] * acc, bf16 or fp32; same fused row dot
   void* wg_out; int wg_f32; const float* row_scale; int accumulate;
   int tma_store;   // 1: bf16 output tiles leave through shared memory and a TMA store (tensor map given)
@@ -510,8 +511,10 @@ __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap*
       else mbar_arrive(release_bar);
     }
   }
-  if (EPI != EPI_STORE && p.qdot && row_ok)
+  if (EPI != EPI_STORE && p.qdot && row_ok) {
     p.dz_part[(int64_t)((split * p.tiles_n + tn) * 2 + h) * p.dz_stride + row] = dot;
+    if (p.dz_meta && row == 0 && tn == 0 && split == 0 && h == 0) *p.dz_meta = 2 * p.tiles_n * p.splits;
+  }
 }
 
 }  // namespace tc

@@ -284,39 +284,43 @@ __device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr) {
 }
 
 // Leader's TMA thread: draws the next entry and hands it to the pair.  Returns the work-list index, -1 when the
-// queue is exhausted, -2 when a wait gave up.  `ticket` carries the ticket drawn ahead for the next call (the
-// atomic's latency then overlaps the loads of the current tile).
-// Scopes: operations at cluster scope cost the issuing thread the better part of a microsecond each, so the
-// leader's own readers (the MMA thread above all) are served with CTA-scope operations on the leader's copy of
-// the ring, and only the peer's copy is written and signalled at cluster scope.  The wait for a free slot needs
-// no acquire: the readers publish nothing with their arrivals.
+// queue is exhausted, -2 when a wait gave up.  The first two entries of a pair are fixed (queue positions pair and
+// npairs + pair); from the third on the position is 2 * npairs + ticket, with `ticket` drawn one call ahead, so
+// that the atomic's latency overlaps the loads of a tile.
+// Cost: release / acquire operations at cluster scope cost the issuing thread the better part of a microsecond
+// each (measured), per tile and per reader.  So the leader's own readers (the MMA thread above all) are served
+// with CTA-scope operations on the leader's copy of the ring, and the peer's copy is written with ONE
+// asynchronous remote store that also completes the peer's barrier (st.async ... complete_tx): the leader never
+// waits for the peer.  The peer's TMA thread arms its barriers (arrive.expect_tx, 4 bytes) one use ahead.  The
+// wait for a free slot needs no acquire: the readers publish nothing with their arrivals.
 __device__ __forceinline__ int queue_draw(const GroupParams& gp, const QueueRing& q, int& cursor, int pair, int npairs, unsigned& ticket,
                                           volatile int* abort_flag) {
   const int s = cursor & (kQueueSlots - 1);
   const uint32_t use = (uint32_t)(cursor / kQueueSlots) & 1u;
   if (!mbar_wait(q.empty(s), use ^ 1u, abort_flag)) return -2;     // the readers of the slot's previous entry are done
-  const int pos = cursor == 0 ? pair : npairs + (int)ticket;
+  const int pos = cursor == 0 ? pair : cursor == 1 ? npairs + pair : 2 * npairs + (int)ticket;
   const int idx = pos < gp.total_work ? work_at(gp, pos) : -1;
   asm volatile("st.shared.u32 [%0], %1;" ::"r"(q.slot(s)), "r"((uint32_t)idx) : "memory");
   mbar_arrive(q.full(s));                                          // release at CTA scope: the leader's readers
-  st_shared_cluster_u32(map_to_cta(q.slot(s), 1), (uint32_t)idx);
-  mbar_arrive_cluster(map_to_cta(q.full(s), 1));                   // release at cluster scope: the peer's readers
-  if (idx >= 0) ticket = atomicAdd(gp.sync + kSyncWork, 1u);
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];"
+               ::"r"(map_to_cta(q.slot(s), 1)), "r"((uint32_t)idx), "r"(map_to_cta(q.full(s), 1)) : "memory");
+  if (idx >= 0 && cursor >= 1) ticket = atomicAdd(gp.sync + kSyncWork, 1u);   // for the draw after the next
   ++cursor;
   return idx;
 }
-// Every other role (one thread per reader): the next entry of the pair's sequence.
-__device__ __forceinline__ int queue_next(const QueueRing& q, int& cursor, uint32_t rank, volatile int* abort_flag) {
+// Every other role (one thread per reader): the next entry of the pair's sequence.  `rearm`: the peer's TMA
+// thread arms the slot's barrier for its next use before it hands the slot back.
+__device__ __forceinline__ int queue_next(const QueueRing& q, int& cursor, uint32_t rank, bool rearm, volatile int* abort_flag) {
   const int s = cursor & (kQueueSlots - 1);
   const uint32_t use = (uint32_t)(cursor / kQueueSlots) & 1u;
-  if (rank == 0) {
-    if (!mbar_wait(q.full(s), use, abort_flag)) return -2;
-  } else {
-    if (!mbar_wait_cluster(q.full(s), use, abort_flag)) return -2;
-  }
+  if (!mbar_wait(q.full(s), use, abort_flag)) return -2;
   const int idx = (int)ld_shared_u32(q.slot(s));
-  if (rank == 0) mbar_arrive(q.empty(s));
-  else asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(map_to_cta(q.empty(s), 0)) : "memory");
+  if (rank == 0) {
+    mbar_arrive(q.empty(s));
+  } else {
+    if (rearm) mbar_expect_tx(q.full(s), 4u);
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(map_to_cta(q.empty(s), 0)) : "memory");
+  }
   ++cursor;
   return idx;
 }
@@ -375,7 +379,9 @@ gemm2_chain_kernel(const __grid_constant__ GroupParams gp) {
       unsigned ticket = 0;
       // The leader keeps the ring one entry ahead of its own loads: the entry of the next tile is published before
       // the loads of the current one, so that no reader (the peer's TMA thread least of all) learns of a tile late.
-      int w = rank == 0 ? queue_draw(gp, queue, cursor, pair, npairs, ticket, abort_flag) : queue_next(queue, cursor, rank, abort_flag);
+      if (rank != 0)
+        for (int s = 0; s < kQueueSlots; ++s) mbar_expect_tx(queue.full(s), 4u);     // first use of every slot
+      int w = rank == 0 ? queue_draw(gp, queue, cursor, pair, npairs, ticket, abort_flag) : queue_next(queue, cursor, rank, true, abort_flag);
       while (ok && w >= 0) {
         int w_next = -1;
         if (rank == 0) w_next = queue_draw(gp, queue, cursor, pair, npairs, ticket, abort_flag);
@@ -384,7 +390,7 @@ gemm2_chain_kernel(const __grid_constant__ GroupParams gp) {
           if (gp.prob[it.g].p.kind == 0) ok = chain_produce_item<A0, B0>(gp, it, rank, smem_base, sbytes, bars, stage, phase, abort_flag, cs);
           else                           ok = chain_produce_item<A1, B1>(gp, it, rank, smem_base, sbytes, bars, stage, phase, abort_flag, cs);
         }
-        if (rank != 0 && ok) w_next = queue_next(queue, cursor, rank, abort_flag);
+        if (rank != 0 && ok) w_next = queue_next(queue, cursor, rank, true, abort_flag);
         w = w_next;
       }
       if (w == -2) ok = false;
@@ -405,7 +411,7 @@ gemm2_chain_kernel(const __grid_constant__ GroupParams gp) {
       bool ok = true;
       int cursor = 0;
       while (ok) {
-        const int w = queue_next(queue, cursor, 0u, abort_flag);
+        const int w = queue_next(queue, cursor, 0u, false, abort_flag);
         if (w < 0) break;
         const GroupItem it = decode_group(gp, w, BM2);
         if (!it.active) continue;
@@ -426,7 +432,7 @@ gemm2_chain_kernel(const __grid_constant__ GroupParams gp) {
     int cursor = 0;
     while (ok) {
       int w = 0;
-      if (lane == 0) w = queue_next(queue, cursor, rank, abort_flag);    // one lane reads the ring: the warp cannot disagree
+      if (lane == 0) w = queue_next(queue, cursor, rank, false, abort_flag);    // one lane reads the ring: the warp cannot disagree
       w = __shfl_sync(0xffffffffu, w, 0);
       if (w < 0) break;
       const GroupItem it = decode_group(gp, w, BM2);

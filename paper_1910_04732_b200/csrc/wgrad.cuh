@@ -238,6 +238,27 @@ bwd_finish_group_kernel(const __grid_constant__ BwdFinishGroup g) {
   }
 }
 
+// The second stage of dlog_alpha for many matrices in one launch: a training step may leave the partial row dots
+// of every backward call in that call's workspace and add them up once, at the end of the step.  The number of
+// partial vectors is read from the word the backward GEMM left next to them.  Partials are added in index order.
+constexpr int kDlaGroup = 96;
+struct DlaFinish { const float* dz_part; const int* n_part; int cap; const float* dz_dla; float* dla; int r; };
+struct DlaFinishGroup { DlaFinish a[kDlaGroup]; int n; };
+
+__global__ void __launch_bounds__(256)
+dalpha_group_kernel(const __grid_constant__ DlaFinishGroup g, int accumulate) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const DlaFinish& a = g.a[blockIdx.y];
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= a.r) return;
+  const int n_part = min(max(*a.n_part, 0), a.cap);
+  float s = 0.f;
+  for (int p = 0; p < n_part; ++p) s += a.dz_part[(int64_t)p * a.r + k];
+  const float v = s * a.dz_dla[k];
+  a.dla[k] = accumulate ? a.dla[k] + v : v;
+}
+
 // diag(z) Q of many matrices in one launch (it depends only on the gate sample and the weights, so a training
 // step forms it once, right after sampling, for every matrix of the model).  16-byte units, four per thread in
 // flight; rows are 16-byte aligned.

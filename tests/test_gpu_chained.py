@@ -89,9 +89,9 @@ def test_chained_layer_is_one_launch_each_way_and_matches_grouped_and_oracle(b, 
     for rep in range(2):            # the second call finds the area as the first left it
         n0 = b.launch_count()
         b.gated_lowrank_fwd_chained(_fwd(b, es, "c"), sync)
-        assert b.launch_count() - n0 == 1
+        assert b.launch_count() - n0 == 2                  # one launch per product, no small kernels
         b.gated_lowrank_bwd_chained(_bwd(b, es, "c"), sync, wgrad_dt=wd)
-        assert b.launch_count() - n0 == 2
+        assert b.launch_count() - n0 == 5                  # diag(z) Q, then {dH', dP} and {dQ, dX}; dlog_alpha inside
         assert b.device_status() == b.OK
         assert int(sync.view(torch.int32).abs().sum().item()) == 0       # left zero-filled
         if rep == 0:
@@ -125,7 +125,7 @@ def test_chained_optional_outputs_and_accumulate(b):
     b.gated_lowrank_fwd_chained(_fwd(b, es, "c"), sync)
     n0 = b.launch_count()
     b.gated_lowrank_bwd_chained(_bwd(b, es, "c", skip), sync, accumulate=True)
-    assert b.launch_count() - n0 == 1
+    assert b.launch_count() - n0 == 3
     assert b.device_status() == b.OK
     assert int(sync.view(torch.int32).abs().sum().item()) == 0
     for i, e in enumerate(es):
@@ -153,7 +153,7 @@ def test_chained_full_size_layer_as_the_benchmark_issues_it(b, name):
     n0 = b.launch_count()
     b.gated_lowrank_fwd_chained(_fwd(b, es, "c"), sync)
     b.gated_lowrank_bwd_chained(_bwd(b, es, "c", qz=True), sync)
-    assert b.launch_count() - n0 == 2
+    assert b.launch_count() - n0 == 4
     assert b.device_status() == b.OK
     assert int(sync.view(torch.int32).abs().sum().item()) == 0
     for e in es:
@@ -173,7 +173,7 @@ def test_chained_sru_layer_with_more_tiles_than_the_schedule_table(b):
         n0 = b.launch_count()
         b.gated_lowrank_fwd_chained(_fwd(b, es, "c"), sync)
         b.gated_lowrank_bwd_chained(_bwd(b, es, "c"), sync)
-        assert b.launch_count() - n0 == 2
+        assert b.launch_count() - n0 == 5
         assert b.device_status() == b.OK
         assert int(sync.view(torch.int32).abs().sum().item()) == 0
         for e in es:
