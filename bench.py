@@ -50,6 +50,31 @@ def measured_peaks():
         return dict(FALLBACK_PEAKS), "fallback"
 
 
+def roofline_traffic(workload: str, group: int):
+    """DRAM bytes per GEMM launch from the ncu capture summarised in profiles/gemm_traffic.txt, valid only while the
+    GEMM kernel sources are the ones the capture was taken with (the file records their hash)."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "gemm_traffic.txt")
+    try:
+        fields = {}
+        for ln in open(path):
+            if "=" in ln and not ln.startswith("#"):
+                k, v = ln.strip().split("=", 1)
+                fields[k.strip()] = v.strip()
+        h = hashlib.sha1()
+        d = os.path.join(ROOT, "paper_1910_04732_b200", "csrc")
+        for f in sorted(os.listdir(d)):
+            if f.startswith("gemm_tc") or f == "schedule.cuh":
+                h.update(open(os.path.join(d, f), "rb").read())
+        if fields.get("workload") != workload or int(fields.get("matrices_per_call", -1)) != group:
+            return None, "no capture for this workload"
+        if fields.get("kernel_sources_sha1") != h.hexdigest():
+            return None, "the GEMM kernels have changed since the capture in profiles/gemm_traffic.txt"
+        return float(fields["dram_bytes_per_launch"]), fields.get("note", "")
+    except Exception:
+        return None, "profiles/gemm_traffic.txt not found"
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
@@ -115,7 +140,9 @@ class Job:
         self.w, self.b, self.torch = w, b, torch
         bf = torch.bfloat16
         g = torch.Generator(device=device)
-        g.manual_seed(seed)
+        g.manual_seed(seed)                 # activations: every rank its own batch
+        gw = torch.Generator(device=device)
+        gw.manual_seed(1234)                # weights: one model on every rank (their gradients are summed)
         mats = w.all_matrices()
         self.n_gates = w.n_gates()
         # gate state, concatenated over all matrices
@@ -139,11 +166,11 @@ class Job:
         n_w = sum(m.d_out * r8(m.r) + m.r * r8(m.d_in) for _, _, m in mats)
         self.wgrad = torch.zeros(n_w, dtype=bf, device=device)
         self.mats, pos, ws_bytes = [], 0, 0
-        randn = lambda rows, cols, scale=1.0: (torch.randn(rows, r8(cols), generator=g, device=device) * scale).to(bf)[:, :cols]
+        randn = lambda rows, cols, scale=1.0, gen=g: (torch.randn(rows, r8(cols), generator=gen, device=device) * scale).to(bf)[:, :cols]
         for (l, i, m), lo in zip(mats, offs):
             e = dict(m=m, lo=lo, hi=lo + m.r)
             e["X"], e["dY"] = randn(w.T, m.d_in), randn(w.T, m.d_out)
-            e["Q"], e["P"] = randn(m.r, m.d_in, m.d_in ** -0.5), randn(m.d_out, m.r, m.r ** -0.5)
+            e["Q"], e["P"] = randn(m.r, m.d_in, m.d_in ** -0.5, gw), randn(m.d_out, m.r, m.r ** -0.5, gw)
             e["H"], e["Y"], e["dX"] = (b.padded(w.T, c, bf, device) for c in (m.r, m.d_out, m.d_in))
             e["dP"] = self.wgrad[pos:pos + m.d_out * r8(m.r)].view(m.d_out, r8(m.r))[:, :m.r]; pos += m.d_out * r8(m.r)
             e["dQ"] = self.wgrad[pos:pos + m.r * r8(m.d_in)].view(m.r, r8(m.d_in))[:, :m.d_in]; pos += m.r * r8(m.d_in)
@@ -184,11 +211,9 @@ class Job:
                                                           self.dlog_alpha[e["lo"]:e["hi"]], e["ws"], Qz=e["Qz"],
                                                           defer_dlog_alpha=True) for e in self.mats])
         # data parallelism: one gradient bucket per grouped call (a layer), reduced while later layers compute
-        n_per = group if group > 0 else len(self.mats)
-        sizes_w = [e["dP"].shape[0] * r8(e["m"].r) + e["m"].r * r8(e["m"].d_in) for e in self.mats]
-        self.bucket_bounds = [0]
-        for i in range(0, len(sizes_w), n_per):
-            self.bucket_bounds.append(self.bucket_bounds[-1] + sum(sizes_w[i:i + n_per]))
+        from paper_1910_04732_b200 import dp
+        self.bucket_bounds = dp.bucket_bounds(dp.weight_gradient_sizes([e["m"] for e in self.mats]),
+                                              group if group > 0 else len(self.mats))
         self.reducer = None
         self.ws_l0 = b.alloc_workspace(b.workspace_bytes(b.OP_L0, self.n_gates, 0, 0, len(sizes), b.F32), device)
         self.offset_dev = torch.zeros(1, dtype=torch.int64, device=device)
@@ -354,30 +379,53 @@ def time_steps(job: Job, steps: int, world: int, use_graph: bool = False):
 
 
 def time_e2e(job: Job, steps: int, world: int):
-    """The same step fed from pinned host memory: every X and dY crosses PCIe inside the timed
-    region (copy stream, overlapped with compute), dlog_alpha and the Lagrangian scalars come back."""
+    """The same step through the same grouped calls, fed from and drained to pinned host memory inside the timed
+    region: every X and dY crosses PCIe on a copy stream, layer by layer ahead of the compute; Y and dX of every
+    matrix, the flat weight-gradient buffer, dlog_alpha and the Lagrangian scalars come back on a second copy
+    stream as soon as the layer that produced them is done."""
     import torch
+    assert job.group > 0
+    pin = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory()
     host_in = [(e["X"].cpu().pin_memory(), e["dY"].cpu().pin_memory()) for e in job.mats]
-    host_dla = torch.empty(job.n_gates, dtype=torch.float32).pin_memory()
-    host_out4 = torch.empty(4, dtype=torch.float32).pin_memory()
-    copy_stream = torch.cuda.Stream()
+    host_out = [(pin(e["Y"]), pin(e["dX"])) for e in job.mats]
+    host_wgrad, host_dla, host_out4 = pin(job.wgrad), pin(job.dlog_alpha), pin(job.out4)
+    h2d, d2h = torch.cuda.Stream(), torch.cuda.Stream()
     main = torch.cuda.current_stream()
-    events = [torch.cuda.Event() for _ in job.mats]
+    n_groups = len(job.groups)
+    per = job.group
+    ev_in = [torch.cuda.Event() for _ in range(n_groups)]
+    ev_done = [torch.cuda.Event() for _ in range(n_groups)]
+    ev_end = torch.cuda.Event()
 
     def one_step():
-        copy_stream.wait_stream(main)          # the previous step has consumed the device buffers
-        with torch.cuda.stream(copy_stream):
-            for (hx, hdy), e, ev in zip(host_in, job.mats, events):
-                e["X"].copy_(hx, non_blocking=True)
-                e["dY"].copy_(hdy, non_blocking=True)
-                ev.record(copy_stream)
+        h2d.wait_stream(main)                  # the previous step has consumed the device input buffers
+        d2h.wait_stream(main)
+        with torch.cuda.stream(h2d):
+            for gi in range(n_groups):
+                for k in range(gi * per, min((gi + 1) * per, len(job.mats))):
+                    job.mats[k]["X"].copy_(host_in[k][0], non_blocking=True)
+                    job.mats[k]["dY"].copy_(host_in[k][1], non_blocking=True)
+                ev_in[gi].record(h2d)
         job.sample_gates()
-        for e, ev in zip(job.mats, events):
-            main.wait_event(ev)
-            job.run_matrix(e)
-        job.finish()
-        host_dla.copy_(job.dlog_alpha, non_blocking=True)
-        host_out4.copy_(job.out4, non_blocking=True)
+        job.b.scale_rows_grouped(job.scale)
+        for gi, (fwd, bwd, bwd_chain, bwd_plain) in enumerate(job.groups):
+            main.wait_event(ev_in[gi])
+            job.b.gated_lowrank_fwd_grouped(fwd)
+            job.b.gated_lowrank_bwd_grouped(bwd)
+            ev_done[gi].record(main)
+            with torch.cuda.stream(d2h):
+                d2h.wait_event(ev_done[gi])
+                for k in range(gi * per, min((gi + 1) * per, len(job.mats))):
+                    host_out[k][0].copy_(job.mats[k]["Y"], non_blocking=True)
+                    host_out[k][1].copy_(job.mats[k]["dX"], non_blocking=True)
+        job.finish(deferred=True)
+        ev_end.record(main)
+        with torch.cuda.stream(d2h):
+            d2h.wait_event(ev_end)
+            host_wgrad.copy_(job.wgrad, non_blocking=True)
+            host_dla.copy_(job.dlog_alpha, non_blocking=True)
+            host_out4.copy_(job.out4, non_blocking=True)
+        main.wait_stream(d2h)                  # the step ends when its results are on the host
 
     one_step()
     if world > 1:
@@ -396,10 +444,13 @@ def time_e2e(job: Job, steps: int, world: int):
         t = torch.tensor([ms], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
-    h2d = sum(hx.numel() * 2 + hdy.numel() * 2 for hx, hdy in host_in)
-    d2h = host_dla.numel() * 4 + 16
+    nbytes = lambda t: t.numel() * t.element_size()
+    h2d_bytes = sum(nbytes(hx) + nbytes(hdy) for hx, hdy in host_in)
+    d2h_bytes = sum(nbytes(y) + nbytes(dx) for y, dx in host_out) + nbytes(host_wgrad) + nbytes(host_dla) + nbytes(host_out4)
     assert np.isfinite(host_out4.numpy()).all()
-    return ms, h2d, d2h
+    assert torch.isfinite(host_out[-1][0].float()).all() and torch.isfinite(host_wgrad.float()).all()
+    returned = "Y and dX of every matrix, all weight gradients (dP, dQ), dlog_alpha, the four Lagrangian scalars"
+    return ms, h2d_bytes, d2h_bytes, returned
 
 
 # ----------------------------------------------------------------------------- oracle arm
@@ -429,6 +480,8 @@ def oracle_sample(w: I.Workload):
 
 
 def run_reference(args, w: I.Workload):
+    """The oracle as it stands, on the host cores.  One timed step = the bounded sample (layer 0 at the full token
+    count); the throughput of a full step is extrapolated from it (every layer has the same shapes) and labelled so."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -437,11 +490,14 @@ def run_reference(args, w: I.Workload):
         dt, sample, threads = oracle_sample(w)
         if i >= args.warmup:
             times.append(dt)
-    step_s = float(np.mean(times)) * w.layers
+    sample_s = float(np.mean(times))
+    step_s = sample_s * w.layers
     value = w.T / step_s
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sample_s * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "extrapolated_from": f"a timed step is layer 0 of {w.layers} (all layers have the same shapes); value = T / (ms_per_step x {w.layers})",
+            "ms_per_full_step_extrapolated": step_s * 1e3,
             "tflops": w.flops_per_step() / step_s / 1e12,
             "config": {"workload": w.name, "T": w.T, "layers": w.layers,
                        "matrices": [[m.name, m.d_in, m.d_out, m.r] for m in w.matrices]},
@@ -517,18 +573,31 @@ def main():
             job.graph.replay()
     torch.cuda.synchronize()
     ms = time_steps(job, args.steps, world, use_graph)
-    # the GEMM launches of the last replayed step, timed on the device (%globaltimer stamps written by the kernels)
+    # Roofline of the dominant kernels (the tensor-core GEMM launches).  Inside the replayed graph every launch
+    # stamps %globaltimer when its first CTA passes the dependency wait and when its last CTA ends; a second pass
+    # replays the same graph, reads the stamps after EVERY replay and brackets each replay with events, so that
+    # the kernel time and the step time it is compared with come from the same replays.
     graph_gemm = None
     if use_graph:
         n_st, fl_st = job.stamped
-        st = stamps[: 2 * n_st].view(n_st, 2).cpu().numpy()
-        dur_ns = float((st[:, 1] - st[:, 0]).clip(min=0).sum())
-        if n_st > 0 and dur_ns > 0:
-            graph_gemm = {"launches": n_st, "kernel_ms_per_step": dur_ns / 1e6, "tflops": fl_st / dur_ns / 1e3}
-            if os.environ.get("FLOP_BENCH_DUMP_STAMPS"):
+        k_rep = max(3, min(args.steps, 50))
+        kern_ms, step_ms_rep = [], []
+        for _ in range(k_rep):
+            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            r0.record(); job.graph.replay(); r1.record()
+            torch.cuda.synchronize()
+            st = stamps[: 2 * n_st].view(n_st, 2).cpu().numpy()
+            kern_ms.append(float((st[:, 1] - st[:, 0]).clip(min=0).sum()) / 1e6)
+            step_ms_rep.append(r0.elapsed_time(r1))
+            if os.environ.get("FLOP_BENCH_DUMP_STAMPS") and len(kern_ms) == k_rep:
                 rel = (st - st[0, 0]) / 1e3
                 print("stamps_us " + " ".join(f"[{a:.1f},{b:.1f}]" for a, b in rel[:16]), file=sys.stderr)
-    # second pass of the same steps with CUDA events around every tensor-core GEMM launch
+        if n_st > 0 and min(kern_ms) > 0:
+            km, sm = float(np.mean(kern_ms)), float(np.mean(step_ms_rep))
+            graph_gemm = {"launches": n_st, "replays": k_rep, "kernel_ms_per_step": km, "step_ms_same_replays": sm,
+                          "tflops": fl_st / (km * 1e-3) / 1e12, "flops_per_step": fl_st}
+            assert km <= sm * 1.005, f"stamped kernel time {km:.3f} ms exceeds the step it was taken in ({sm:.3f} ms)"
+    # the same launches issued eagerly with CUDA events recorded around every GEMM launch (no dependent-launch overlap)
     b.gemm_timing_begin()
     ms_timed_pass = time_steps(job, args.steps, world)
     gemm_ms, gemm_flops, gemm_launches = b.gemm_timing_end()
@@ -565,11 +634,12 @@ def main():
         assert b.device_status() == b.OK
 
     e2e = None
-    if not args.no_e2e:
-        e2e_ms, h2d, d2h = time_e2e(job, max(3, min(args.steps, 20)), world)
+    if not args.no_e2e and group > 0:
         e2e_steps = max(3, min(args.steps, 20))
+        e2e_ms, h2d, d2h, returned = time_e2e(job, e2e_steps, world)
         e2e = {"value": w.T * world / (e2e_ms / e2e_steps / 1e3), "unit": "tokens/s", "ms_per_step": e2e_ms / e2e_steps,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "returned": returned,
+               "path": "the grouped calls of the headline step (eager issue: copies and compute overlap layer by layer)"}
 
     if rank != 0:
         if world > 1:
@@ -581,31 +651,49 @@ def main():
     step_ms = ms / args.steps
     tokens_s = w.T * world / (step_ms / 1e3)
     tflops = w.flops_per_step() * world / (step_ms / 1e3) / 1e12
-    gemm_tflops = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
-    # dram__bytes_read.sum + dram__bytes_write.sum of the GEMM launches of one bert layer, from the ncu capture
-    # summarised under profiles/ (grouped calls of six matrices): mean per launch
-    traffic = 118.6e6 if (w.name == "bert" and group == 6) else None
+    event_tflops = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
+    # Which measured peak bounds this run: the burst figure (a kernel timed alone, clocks near the maximum) while the
+    # timed region is short or the sampled clock is above the clock the sustained figure was taken at; the sustained
+    # figure (a seconds-long loop under the power cap) otherwise.
+    timed_s = ms / 1e3
+    clk_sustained = None
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            clk_sustained = float(json.load(f)["clocks_under_load"]["sm_mhz_median"])
+    except Exception:
+        pass
+    sm_mhz = clocks.get("sm_mhz") if clocks else None
+    use_burst = timed_s < 1.0 or (clk_sustained is not None and sm_mhz is not None and sm_mhz > clk_sustained * 1.05)
+    peak = peaks["bf16_tflops"] if use_burst else peaks["bf16_tflops_sustained"]
+    achieved = graph_gemm["tflops"] if graph_gemm is not None else event_tflops
+    fracs = lambda tf: {"nominal_2250": tf / NOMINAL_BF16_TFLOPS, "measured_burst": tf / peaks["bf16_tflops"],
+                        "measured_sustained": tf / peaks["bf16_tflops_sustained"]}
+    traffic, traffic_note = roofline_traffic(w.name, group)
     line = {
         "metric": METRIC, "value": tokens_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "tflops": tflops, "pct_of_bf16_peak_nominal": 100.0 * tflops / world / NOMINAL_BF16_TFLOPS,
-        "pct_of_bf16_peak_measured_sustained": 100.0 * tflops / world / peaks["bf16_tflops_sustained"],
+        "tflops": tflops, "step_frac_of_bf16_peak": fracs(tflops / world),
         "config": {"workload": w.name, "T": w.T, "layers": w.layers,
                    "matrices": [[m.name, m.d_in, m.d_out, m.r] for m in w.matrices],
-                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}", "streams": args.streams, "matrices_per_grouped_call": group, "cuda_graph": bool(use_graph),
+                   "gates": job.n_gates, "weight_grad_dtype": "bf16", "parallelism": f"dp{world}", "streams": args.streams,
+                   "matrices_per_grouped_call": group, "cuda_graph": bool(use_graph),
+                   "calls": "chained" if job.chain else ("grouped, self-contained backward" if job.plain else "grouped; diag(z)Q and dlog_alpha second stage once per step"),
                    "l2": f"inputs larger than L2: {job.input_bytes() / 1e6:.0f} MB of X and dY per step, each matrix its own buffers"},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "tensor", "achieved": gemm_tflops, "peak": peaks["bf16_tflops_sustained"],
-                     "unit": "TFLOP/s", "frac": gemm_tflops / peaks["bf16_tflops_sustained"], "traffic": traffic,
-                     "traffic_note": "DRAM read+write bytes per GEMM launch, mean of the four launches of one layer (ncu capture in profiles/)" if traffic else None,
-                     "peak_kind": f"{peak_kind} (sustained; burst {peaks['bf16_tflops']})",
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_kind": f"{peak_kind} {'burst' if use_burst else 'sustained'} cuBLAS bf16 (timed region {timed_s:.2f} s, median SM clock {sm_mhz} MHz; "
+                                  f"burst {peaks['bf16_tflops']}, sustained {peaks['bf16_tflops_sustained']} at {clk_sustained} MHz)",
+                     "frac_of": fracs(achieved),
+                     "how": "sum of 2MNK of the GEMM launches / their device-stamped time inside the replayed graph, mean over the replays of a stamped pass"
+                            if graph_gemm is not None else "sum of 2MNK of the GEMM launches / their CUDA-event time, eager issue",
+                     "traffic": traffic, "traffic_note": traffic_note,
                      "kernel": "tc::gemm2_group_kernel (forward) / tc::gemm2_dual_kernel (backward): every GEMM launch of the step",
                      "launches_per_step": gemm_launches // args.steps,
-                     "kernel_ms_per_step": gemm_ms / args.steps, "step_ms_in_timed_pass": ms_timed_pass / args.steps,
-                     "frac_of_nominal": gemm_tflops / NOMINAL_BF16_TFLOPS,
-                     # the same launches inside the replayed graph, timed by device-side stamps (no event gaps, PDL overlap kept)
-                     "in_graph": None if graph_gemm is None else dict(graph_gemm, frac=graph_gemm["tflops"] / peaks["bf16_tflops_sustained"])},
+                     "in_graph": graph_gemm,
+                     # the same launches bracketed by CUDA events in an eagerly issued pass (events break the dependent-launch overlap)
+                     "event_timed": {"tflops": event_tflops, "kernel_ms_per_step": gemm_ms / args.steps,
+                                     "step_ms_same_pass": ms_timed_pass / args.steps, "frac_of": fracs(event_tflops)}},
         "clocks": clocks,
     }
     if e2e is not None:

@@ -41,7 +41,7 @@ extern "C" {
 
 typedef enum {
   FLOP_OK = 0,
-  FLOP_ERR_INVALID_ARG = 1, /* null pointer, negative size, ld too small, bad enum          */
+  FLOP_ERR_INVALID_ARG = 1, /* null pointer, negative size, ld too small, bad enum; a bad device-side table */
   FLOP_ERR_UNSUPPORTED = 2, /* alignment / leading-dimension / size limit of the kernels   */
   FLOP_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than flop_workspace_bytes */
   FLOP_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed                           */
@@ -68,8 +68,9 @@ typedef enum {
 
 const char* flop_status_string(int status);
 
-/* Synchronises `stream`, returns the device status word (FLOP_OK, or FLOP_ERR_TIMEOUT when a bounded
- * device-side wait of an earlier call gave up) and clears it.  flop_device_status is the same call
+/* Synchronises `stream`, returns the device status word (FLOP_OK; FLOP_ERR_TIMEOUT when a bounded
+ * device-side wait of an earlier call gave up; FLOP_ERR_INVALID_ARG when a kernel found a device-side
+ * table it cannot use, see flop_expected_l0_lagrangian) and clears it.  flop_device_status is the same call
  * under its older name. */
 int flop_last_async_status(void* stream);
 int flop_device_status(void* stream);
@@ -309,9 +310,13 @@ int flop_active_ranks_scatter(const flop_active_scatter_t* problems, int n, int 
  *     s = sum_j pi_j size_j / sum_j size_j,   g = lambda1 (s - t) + lambda2 (s - t)^2
  * out4 = {s, g, dg/dlambda1, dg/dlambda2}; seg_expected[n_seg] (nullable) =
  * sum of pi_j per segment; dlog_alpha[n] (nullable) += dg/dlog_alpha.
- * n is the total number of gates (= seg_off[n_seg]).  target[1] and
- * lambda[2] are DEVICE pointers so that an optimiser can update them on the
- * device.  n_seg <= 4096. */
+ * n is the total number of gates.  seg_off[n_seg + 1] (DEVICE) must partition
+ * [0, n): seg_off[0] = 0, ascending, seg_off[n_seg] = n.  The table is in device
+ * memory, so it is checked on the device: a table that breaks this rule makes the
+ * call write NaN to out4, leave everything else untouched and record
+ * FLOP_ERR_INVALID_ARG in the status word flop_last_async_status() returns.
+ * target[1] and lambda[2] are DEVICE pointers so that an optimiser can update
+ * them on the device.  n_seg <= 4096. */
 int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t* seg_off,
                                 const float* seg_size, int32_t n_seg, flop_hc_params_t hc,
                                 const float* target, const float* lambda, float* out4,
@@ -354,7 +359,9 @@ int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const
  *             repeat across tokens: clear dE before the first call of a step; the order of the adds
  *             is not fixed, so dE is reproducible only to fp32 rounding),
  *             dlog_alpha = dz_dla * sum_t E[ids[t], :] dH'[t, :]  (fixed summation order).
- *   Any of dE, dO, dlog_alpha may be NULL.  Workspace: flop_workspace_bytes(FLOP_OP_EMBEDDING_BWD, T,
+ *   Any of dE, dO, dlog_alpha may be NULL.  dO is written in place with 16-byte stores: its pointer must be
+ *   16-byte aligned and lddo a multiple of 8 (bf16) or 4 (fp32) elements, else FLOP_ERR_UNSUPPORTED (checked
+ *   before anything is launched).  Workspace: flop_workspace_bytes(FLOP_OP_EMBEDDING_BWD, T,
  *   0, 0, d_i, dt).  The tied softmax side of the same cluster, logits = ((h O^T) * z) E^T, is
  *   flop_gated_lowrank_fwd/bwd with Q = O^T and P = E. */
 int flop_gated_embedding_fwd(const int32_t* ids, int64_t T, const void* E, int64_t lde, int64_t n_rows,

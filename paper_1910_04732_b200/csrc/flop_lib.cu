@@ -1781,13 +1781,13 @@ int flop_expected_l0_lagrangian(const float* log_alpha, int64_t n, const int64_t
   const int64_t chunks = (n + kL0Chunk - 1) / kL0Chunk + n_seg;
   if (chunks > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
   if (chunks > 0 && n_seg > 0) {
-    launch_k(l0_chunk_kernel<false>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
+    launch_k(l0_chunk_kernel<false>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr, n, (int)chunks);
     count_launch();
   }
-  launch_k(l0_finalize_kernel, dim3(1), dim3(kL0Threads), (size_t)(0), st, seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
+  launch_k(l0_finalize_kernel, dim3(1), dim3(kL0Threads), (size_t)(0), st, seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected, n, (int)chunks);
   count_launch();
   if (dlog_alpha && chunks > 0 && n_seg > 0) {
-    launch_k(l0_chunk_kernel<true>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
+    launch_k(l0_chunk_kernel<true>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha, n, (int)chunks);
     count_launch();
   }
   FLOP_CUDA(cudaGetLastError());
@@ -1816,13 +1816,14 @@ int flop_expected_l0_lagrangian_noalloc(const float* log_alpha, int64_t n, const
   // Nothing in the scratch has to start at zero: every chunk sum that the finalisation reads and
   // the gradient coefficient are rewritten by this call before they are read.
   if (chunks > 0 && n_seg > 0) {
-    launch_k(l0_chunk_kernel<false>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr);
+    launch_k(l0_chunk_kernel<false>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, nullptr, n, (int)chunks);
     count_launch();
   }
-  launch_k(l0_finalize_kernel, dim3(1), dim3(kL0Threads), (size_t)(0), st, seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected);
+  // the grid, and so the chunk sums this call may use, is sized from the host's n and n_seg; it never exceeds the built-in array
+  launch_k(l0_finalize_kernel, dim3(1), dim3(kL0Threads), (size_t)(0), st, seg_off, seg_size, n_seg, target, lambda, sc, out4, seg_expected, n, (int)chunks);
   count_launch();
   if (dlog_alpha && chunks > 0 && n_seg > 0) {
-    launch_k(l0_chunk_kernel<true>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha);
+    launch_k(l0_chunk_kernel<true>, dim3((unsigned)chunks), dim3(kL0Threads), (size_t)(0), st, log_alpha, seg_off, seg_size, n_seg, thr, sc, dlog_alpha, n, (int)chunks);
     count_launch();
   }
   FLOP_CUDA(cudaGetLastError());
@@ -1892,6 +1893,7 @@ int flop_gated_embedding_bwd(const void* dY, int64_t lddy, const int32_t* ids, i
   if (!bf16_ok(dY, lddy) || !bf16_ok(E, lde) || !bf16_ok(O, ldo) || !bf16_ok(H_save, ldh)) return FLOP_ERR_UNSUPPORTED;
   if (T > INT32_MAX || n_rows > INT32_MAX || d_i > INT32_MAX) return FLOP_ERR_UNSUPPORTED;
   if ((size_t)kEmbWarps * d_i * 4 > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
+  if (dO && !wgrad_direct_ok(dO, lddo, wgrad_dt)) return FLOP_ERR_UNSUPPORTED;   // dO is written in place with 16-byte stores
   FLOP_TRY(check_ws(ws, ws_bytes, embedding_ws_bytes(T, d_i)));
   Arena ar{(unsigned char*)ws, ws_bytes, 0};
   const int64_t lddh = round_up(d_i, 8);
@@ -1903,12 +1905,8 @@ int flop_gated_embedding_bwd(const void* dY, int64_t lddy, const int32_t* ids, i
                      store_epilogue(dH, lddh, nullptr), st));
   if (dO) {
     // dO[d_i, d] = H'^T dY: contraction over tokens, written in place when the output allows 16-byte vectors
-    if (wgrad_direct_ok(dO, lddo, wgrad_dt)) {
-      TcPlan pl = plan_tc(d_i, d, T, false, true);
-      FLOP_TRY(launch_tc({H_save, ldh, true}, {dY, lddy, true}, d_i, d, T, pl, wgrad_epilogue(dO, lddo, wgrad_dt, nullptr, accumulate), st));
-    } else {
-      return FLOP_ERR_UNSUPPORTED;
-    }
+    TcPlan pl = plan_tc(d_i, d, T, false, true);
+    FLOP_TRY(launch_tc({H_save, ldh, true}, {dY, lddy, true}, d_i, d, T, pl, wgrad_epilogue(dO, lddo, wgrad_dt, nullptr, accumulate), st));
   }
   if (dE || dlog_alpha) {
     const size_t smem = (size_t)kEmbWarps * d_i * 4;

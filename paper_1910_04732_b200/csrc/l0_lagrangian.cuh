@@ -1,13 +1,17 @@
 // Expected L0 size and augmented-Lagrangian penalty (Eq. 3 and Section 4.3).
 //
 // Three launches, no atomics, fixed summation order (bit-reproducible):
-//   1. l0_partial_kernel : every block owns one chunk of kChunk gates of ONE
+//   1. l0_chunk_kernel<false>: every block owns one chunk of kL0Chunk gates of ONE
 //      segment and writes sum(pi_j) of the chunk (fp64) to scratch.
-//   2. l0_finalize_kernel: one block adds the chunk sums per segment in chunk
+//   2. l0_finalize_kernel    : one block adds the chunk sums per segment in chunk
 //      order, forms s, g, dg/dlambda and the gradient coefficient.
-//   3. l0_grad_kernel    : dlog_alpha_j += coef * size_seg * pi_j (1 - pi_j).
+//   3. l0_chunk_kernel<true> : dlog_alpha_j += coef * size_seg * pi_j (1 - pi_j).
 // Blocks find their (segment, chunk) from the segment table alone: chunk
 // counts per segment are prefix-summed in shared memory by every block.
+// The segment table lives in device memory, so the host cannot check it: the kernels
+// do.  A table that needs more chunk sums than the scratch holds (`capacity`), or
+// that points outside [0, n), touches nothing; the finalisation then reports
+// FLOP_ERR_INVALID_ARG in the device status word and writes NaN to out4.
 #pragma once
 #include "common.cuh"
 
@@ -70,7 +74,7 @@ template <bool kGrad>
 __global__ void __launch_bounds__(kL0Threads)
 l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__ seg_off,
                 const float* __restrict__ seg_size, int n_seg, float thr, L0Scratch* __restrict__ sc,
-                float* __restrict__ dlog_alpha) {
+                float* __restrict__ dlog_alpha, int64_t n, int capacity) {
   pdl_wait();
   pdl_launch_dependents();
   __shared__ int first_chunk[kL0MaxSeg + 1];
@@ -78,12 +82,14 @@ l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__
   __shared__ double red[32];
   l0_chunk_table(seg_off, n_seg, first_chunk, scan_scratch);
   const int b = blockIdx.x;
+  if (first_chunk[n_seg] > capacity) return;   // the table asks for more chunk sums than the scratch holds
   if (b >= first_chunk[n_seg]) {            // surplus block of the upper-bound grid
     return;
   }
   const int seg = l0_find_segment(first_chunk, n_seg, b);
   const int64_t lo = seg_off[seg] + (int64_t)(b - first_chunk[seg]) * kL0Chunk;
   const int64_t hi = min(seg_off[seg + 1], lo + (int64_t)kL0Chunk);
+  if (lo < 0 || hi > n) return;             // a segment outside the gate vector: nothing is read or written
   // vector v of thread t covers gates lo + (v*256 + t)*4 .. +3: consecutive threads, consecutive 16 bytes
   constexpr int kVec = kL0PerThread / 4;
   const bool al_a = (reinterpret_cast<uintptr_t>(log_alpha + lo) & 15) == 0;
@@ -143,13 +149,28 @@ l0_chunk_kernel(const float* __restrict__ log_alpha, const int64_t* __restrict__
 __global__ void __launch_bounds__(kL0Threads)
 l0_finalize_kernel(const int64_t* __restrict__ seg_off, const float* __restrict__ seg_size, int n_seg,
                    const float* __restrict__ target, const float* __restrict__ lambda, L0Scratch* __restrict__ sc,
-                   float* __restrict__ out4, float* __restrict__ seg_expected) {
+                   float* __restrict__ out4, float* __restrict__ seg_expected, int64_t n, int capacity) {
   pdl_wait();
   pdl_launch_dependents();
   __shared__ int first_chunk[kL0MaxSeg + 1];
   __shared__ int scan_scratch[33];
   __shared__ double red_w[32], red_s[32];
+  __shared__ int bad;
+  if (threadIdx.x == 0) bad = 0;
   l0_chunk_table(seg_off, n_seg, first_chunk, scan_scratch);
+  // the segments must partition [0, n): ascending offsets from 0 to n (the chunk sums of anything else were not written)
+  for (int s = threadIdx.x; s < n_seg; s += blockDim.x)
+    if (seg_off[s] < 0 || seg_off[s + 1] < seg_off[s] || seg_off[s + 1] > n) bad = 1;
+  __syncthreads();
+  if (first_chunk[n_seg] > capacity || bad || (n_seg > 0 && (seg_off[0] != 0 || seg_off[n_seg] != n))) {
+    if (threadIdx.x == 0) {
+      atomicExch(&g_device_status, (int)FLOP_ERR_INVALID_ARG);
+      const float nan = __int_as_float(0x7fc00000);
+      out4[0] = nan; out4[1] = nan; out4[2] = nan; out4[3] = nan;
+      sc->coef = 0.0;
+    }
+    return;
+  }
   // One warp per segment (segments w, w + nwarp, ...): lanes stride over the segment's chunk sums,
   // a butterfly adds them, and every warp keeps running totals over its own segments.  The
   // assignment is fixed, so the result is bit-reproducible.

@@ -35,6 +35,23 @@ def allreduce_gradients(flat_buffers: Iterable[torch.Tensor], group=None) -> Non
         dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
 
 
+def weight_gradient_sizes(matrices) -> list:
+    """Elements each matrix takes in the flat weight-gradient buffer: dP [d_out, r] then dQ [r, d_in], both with
+    the leading dimension padded to 8 elements (16-byte rows of bf16).  `matrices` yields objects with d_in, d_out, r."""
+    r8 = lambda v: (v + 7) // 8 * 8
+    return [m.d_out * r8(m.r) + m.r * r8(m.d_in) for m in matrices]
+
+
+def bucket_bounds(sizes, per_bucket: int) -> list:
+    """Bounds of the gradient buckets in the flat buffer: one bucket per `per_bucket` consecutive matrices (the
+    matrices of one grouped call, i.e. of one layer)."""
+    per_bucket = max(1, int(per_bucket))
+    bounds = [0]
+    for i in range(0, len(sizes), per_bucket):
+        bounds.append(bounds[-1] + sum(sizes[i:i + per_bucket]))
+    return bounds
+
+
 class BucketedReducer:
     """Sums one flat gradient buffer over all ranks bucket by bucket, each bucket as soon as it is final.
 
