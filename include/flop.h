@@ -407,6 +407,17 @@ int flop_compact_fwd(const void* X, int64_t ldx, const void* Qc, int64_t ldqc, c
                      int64_t ldpc, void* Y, int64_t ldy, int64_t T, int64_t d_in, int64_t d_out,
                      int64_t k, int dt, void* ws, size_t ws_bytes, void* stream);
 
+/* On-chip forward chain (Section 4.1: y = P G Q x as two products): Y = ((X Q^T) * z) P^T in ONE launch; the
+ * rank-r intermediate is accumulated in tensor memory, gated, rounded to bf16 and handed to the second product
+ * through shared memory, so it never reaches global memory (nothing is saved for a backward pass: this is an
+ * inference call).  z is f32[r] or NULL (compact factors from flop_compact_ranks carry the gate in Qc already:
+ * pass Qc, Pc, k as Q, P, r).  bf16 only, r <= 512 (FLOP_ERR_UNSUPPORTED beyond; use flop_compact_fwd /
+ * flop_gated_lowrank_fwd, which choose between this kernel and two launches by shape).  Needs no workspace.
+ * Results equal the two-launch path's up to fp32 summation order. */
+int flop_chain_fwd(const void* X, int64_t ldx, const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                   const float* z, void* Y, int64_t ldy, int64_t T, int64_t d_in, int64_t d_out, int64_t r,
+                   int dt, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

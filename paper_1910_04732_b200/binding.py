@@ -28,7 +28,7 @@ EXPORTS = ("flop_status_string", "flop_last_async_status", "flop_device_status",
            "flop_expected_l0_lagrangian",
            "flop_expected_l0_lagrangian_noalloc", "flop_agp_gates", "flop_gated_embedding_fwd",
            "flop_gated_embedding_bwd",
-           "flop_compact_ranks", "flop_compact_fwd")
+           "flop_compact_ranks", "flop_compact_fwd", "flop_chain_fwd")
 
 
 class HcParams(ctypes.Structure):
@@ -126,6 +126,7 @@ def load_library() -> ctypes.CDLL:
     lib.flop_gated_lowrank_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, vp, vp, i64,
                                            vp, i64, vp, i64, vp, i64, vp, ci,
                                            i64, i64, i64, i64, ci, ci, vp, sz, vp]
+    lib.flop_chain_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, i64, i64, i64, i64, i64, ci, vp]
     lib.flop_gated_lowrank_fwd_grouped.argtypes = [ctypes.POINTER(FwdProblem), ci, ci, vp]
     lib.flop_gated_lowrank_bwd_grouped.argtypes = [ctypes.POINTER(BwdProblem), ci, ci, ci, ci, vp]
     lib.flop_active_ranks_gather.argtypes = [ctypes.POINTER(ActiveGather), ci, ci, vp]
@@ -383,6 +384,14 @@ def gated_lowrank_bwd_grouped(problems, accumulate: bool = False, dt: int = BF16
     arr = problems if isinstance(problems, ctypes.Array) else problem_array(problems)
     _check(load_library().flop_gated_lowrank_bwd_grouped(arr, len(arr), int(accumulate), dt, wgrad_dt, _stream()),
            "flop_gated_lowrank_bwd_grouped")
+
+
+def chain_fwd(X, Q, P, z, Y, dt: int = BF16) -> None:
+    """flop_chain_fwd: Y = ((X Q^T) * z) P^T in one launch (z may be None)."""
+    T, d_in = X.shape
+    d_out, r = P.shape
+    _check(load_library().flop_chain_fwd(_ptr(X), _ld(X), _ptr(Q), _ld(Q), _ptr(P), _ld(P), _ptr(z), _ptr(Y), _ld(Y),
+                                         T, d_in, d_out, r, dt, _stream()), "flop_chain_fwd")
 
 
 def sync_bytes() -> int:

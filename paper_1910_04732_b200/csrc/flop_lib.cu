@@ -25,6 +25,7 @@
 #include "gemm_tc2_group.cuh"
 #include "gemm_tc2_dual.cuh"
 #include "gemm_tc2_chain.cuh"
+#include "gemm_tc_chainfwd.cuh"
 #include "l0_lagrangian.cuh"
 #include "wgrad.cuh"
 #include "active_ranks.cuh"
@@ -673,6 +674,42 @@ bool wgrad_direct_ok(const void* out, int64_t ldo, int wgrad_dt) {
   return aligned16(out) && (ldo % (wgrad_dt == FLOP_F32 ? 4 : 8)) == 0;
 }
 
+// On-chip forward chain (gemm_tc_chainfwd.cuh): Y = ((X Q^T) * z) P^T in one launch, H' kept in shared memory.
+// FLOP_ERR_UNSUPPORTED when the rank does not fit (k > 512) -- the caller then runs the two products as two launches.
+int launch_chain_fwd(const void* X, int64_t ldx, const void* Q, int64_t ldq, const void* P, int64_t ldp, const float* z, void* Y,
+                     int64_t ldy, int64_t T, int64_t d_in, int64_t d_out, int64_t k, cudaStream_t st) {
+  if (k < 1 || k > tc::kChainMaxK || T < 1 || d_in < 1 || d_out < 1 || T > INT32_MAX || d_in > INT32_MAX || d_out > INT32_MAX)
+    return FLOP_ERR_UNSUPPORTED;
+  const int64_t row_blocks = (T + tc::BM - 1) / tc::BM;
+  if (row_blocks > 65535) return FLOP_ERR_UNSUPPORTED;
+  static bool configured[kMaxDevices] = {};
+  if (first_use_on_device(configured))
+    FLOP_CUDA(cudaFuncSetAttribute(tc::chain_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kChainSmemBytes));
+  tc::ChainFwdParams cp;
+  memset(&cp, 0, sizeof(cp));
+  FLOP_TRY(make_tmap(&cp.tx, X, T, d_in, ldx, tc::BK, tc::BM));
+  FLOP_TRY(make_tmap(&cp.tq, Q, k, d_in, ldq, tc::BK, 64));
+  FLOP_TRY(make_tmap(&cp.tp, P, d_out, k, ldp, tc::BK, tc::kChainBN));
+  FLOP_TRY(make_tmap(&cp.ty, Y, T, d_out, ldy, 64, 32));
+  cp.z = z;
+  cp.T = (int)T; cp.d_in = (int)d_in; cp.d_out = (int)d_out; cp.k = (int)k; cp.k_pad = (int)round_up(k, 64);
+  cp.tiles_n = (int)((d_out + tc::kChainBN - 1) / tc::kChainBN);
+  // Every CTA of a row block recomputes H, so a row block is cut into as few slices as fill the machine.
+  const int slices = (int)std::min<int64_t>(cp.tiles_n, std::max<int64_t>(1, num_sms() / row_blocks));
+  cp.tiles_per_cta = (cp.tiles_n + slices - 1) / slices;
+  tc::Params& y = cp.y;
+  y.M = (int)T; y.N = (int)d_out; y.K = (int)k; y.bn = tc::kChainBN; y.tiles_n = cp.tiles_n; y.tiles_m = (int)row_blocks;
+  y.splits = 1; y.out = (bf16*)Y; y.ldo = ldy; y.tma_store = 1;
+  const dim3 grid((unsigned)((cp.tiles_n + cp.tiles_per_cta - 1) / cp.tiles_per_cta), (unsigned)row_blocks);
+  {
+    GemmTimer timer(st, 2.0 * (double)T * (double)k * ((double)d_in + (double)d_out));
+    launch_k(tc::chain_fwd_kernel, grid, dim3(tc::kThreads), (size_t)tc::kChainSmemBytes, st, cp);
+  }
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
 // Few-token forward product C = (A B^T) * col_scale on the CUDA cores (see gemm_small_t.cuh).
 // Returns FLOP_ERR_UNSUPPORTED when the shape does not fit (the caller then uses the tensor-core path).
 template <int TT>
@@ -1128,6 +1165,19 @@ int flop_gated_lowrank_fwd(const void* X, int64_t ldx, const void* Q, int64_t ld
       return FLOP_ERR_UNSUPPORTED;
   }
   return fwd_impl(X, ldx, Q, ldq, P, ldp, z, Y, ldy, H, ldh, T, d_in, d_out, r, dt, (cudaStream_t)stream);
+}
+
+int flop_chain_fwd(const void* X, int64_t ldx, const void* Q, int64_t ldq, const void* P, int64_t ldp, const float* z, void* Y,
+                   int64_t ldy, int64_t T, int64_t d_in, int64_t d_out, int64_t r, int dt, void* stream) {
+  if (T < 0 || d_in < 0 || d_out < 0 || r < 0 || !valid_dt(dt)) return FLOP_ERR_INVALID_ARG;
+  if (dt != FLOP_BF16) return FLOP_ERR_UNSUPPORTED;
+  if (T == 0 || d_out == 0) return FLOP_OK;
+  if (!check_mat(Y, ldy, d_out)) return FLOP_ERR_INVALID_ARG;
+  if (!bf16_ok(Y, ldy)) return FLOP_ERR_UNSUPPORTED;
+  if (r == 0 || d_in == 0) return zero_2d<bf16>(Y, ldy, T, d_out, (cudaStream_t)stream);
+  if (!check_mat(X, ldx, d_in) || !check_mat(Q, ldq, d_in) || !check_mat(P, ldp, r)) return FLOP_ERR_INVALID_ARG;
+  if (!bf16_ok(X, ldx) || !bf16_ok(Q, ldq) || !bf16_ok(P, ldp)) return FLOP_ERR_UNSUPPORTED;
+  return launch_chain_fwd(X, ldx, Q, ldq, P, ldp, z, Y, ldy, T, d_in, d_out, r, (cudaStream_t)stream);
 }
 
 int flop_compact_fwd(const void* X, int64_t ldx, const void* Qc, int64_t ldqc, const void* Pc, int64_t ldpc, void* Y,

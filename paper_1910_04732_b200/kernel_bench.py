@@ -129,16 +129,18 @@ def main():
     t_c = timed(lambda: b.compact_ranks(la, 0, HC, idx, kd, zd, P, Q, Pc, Qc))
     k = int(kd.item())
     print(f"\npruned inference, d_in={mtx.d_in} d_out={mtx.d_out} r={mtx.r}: k = {k} survive; compaction (select + gather) {t_c * 1e6:.1f} us")
-    print(f"{'T':>6s} {'compact fwd us':>15s} {'gated fwd us':>13s} {'speed-up':>9s} {'compact GFLOP/s':>16s} {'weight GB/s':>12s}")
-    for T in (1, 4, 8, 16, 64, 256, 4096):
-        Xt = X[:T]
+    print(f"{'T':>6s} {'compact fwd us':>15s} {'on-chip chain us':>17s} {'gated fwd us':>13s} {'speed-up':>9s} {'compact GFLOP/s':>16s} {'weight GB/s':>12s}")
+    for T in (1, 4, 8, 16, 17, 64, 256, 1024, 4096, 16384):
+        Xt = X[:T] if T <= X.shape[0] else torch.cat([X] * (T // X.shape[0]))
         Y, H = b.padded(T, mtx.d_out, bf), b.padded(T, mtx.r, bf)
         wsc = b.alloc_workspace(b.workspace_bytes(b.OP_COMPACT_FWD, T, mtx.d_in, mtx.d_out, k, b.BF16))
         tc_ = timed(lambda: b.compact_fwd(Xt, Qc[:k], Pc[:, :k], Y, k, wsc), iters=50, graph=True)
+        # the same product through the on-chip chain (one launch, H' in shared memory), whatever compact_fwd chose
+        tch = timed(lambda: b.chain_fwd(Xt, Qc[:k], Pc[:, :k], None, Y), iters=50, graph=True) if k <= 512 else float("nan")
         tg_ = timed(lambda: b.gated_lowrank_fwd(Xt, Q, P, zd, Y, H, None), iters=50, graph=True)
         flops = 2.0 * T * k * (mtx.d_in + mtx.d_out)
         wbytes = 2.0 * k * (mtx.d_in + mtx.d_out)
-        print(f"{T:6d} {tc_ * 1e6:15.1f} {tg_ * 1e6:13.1f} {tg_ / tc_:9.2f} {flops / tc_ / 1e9:16.0f} {wbytes / tc_ / 1e9:12.0f}")
+        print(f"{T:6d} {tc_ * 1e6:15.1f} {tch * 1e6:17.1f} {tg_ * 1e6:13.1f} {tg_ / tc_:9.2f} {flops / tc_ / 1e9:16.0f} {wbytes / tc_ / 1e9:12.0f}")
     # ---- training on the active rank components: one BERT-shaped layer (six matrices, T = 4096)
     for wl in ("bert", "sru"):
         active_table(I.WORKLOADS[wl], g)
