@@ -132,7 +132,7 @@ int flop_workspace_bytes(int op, int64_t T, int64_t d_in, int64_t d_out, int64_t
  * optional col_scale[n]; (MN,MN) writes fp32 split-K slices
  * slices[s][m*ldN + n] with ldN = N rounded up to 4 and slice stride M*ldN, which
  * the caller adds up (the buffer must hold 32 slices unless splits is given).
- * bn (64, 128, 192, 256), cta2 (0: one CTA per 128-row tile; 1: a CTA pair per
+ * bn (64, 128, 192, 256; 208 for a CTA pair with K-major B), cta2 (0: one CTA per 128-row tile; 1: a CTA pair per
  * 256-row tile) and splits fix the tile shape; bn = 0, cta2 = -1, splits = 0 leave
  * each choice to the library.  *n_slices_out (HOST, nullable) receives the number
  * of slices written (1 for a bf16 store). */

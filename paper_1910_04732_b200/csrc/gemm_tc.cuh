@@ -62,7 +62,7 @@ struct ChainLink {
 
 struct Params {
   int M, N, K;
-  int bn;                 // N per tile: 64, 128, 192 or 256
+  int bn;                 // N per tile: 64, 128, 192, 208 (CTA pairs, K-major B) or 256
   int stages;
   int tiles_m, tiles_n, splits, kb_per_split, num_kb;
   // EPI_STORE: out[m*ldo + n] = acc * col_scale[n]  (bf16)
@@ -203,6 +203,8 @@ __device__ __forceinline__ uint32_t instr_desc(bool a_mn, bool b_mn, int n) {
 }
 
 __host__ __device__ inline uint32_t stage_bytes(int bn) { return kATileBytes + (uint32_t)bn * BK * 2; }
+// tensor-memory columns between the two accumulator buffers (a multiple of 64; 2 x 256 is all there is)
+__host__ __device__ inline uint32_t acc_stride(int bn_max) { return (uint32_t)((bn_max + 63) & ~63); }
 // shared memory after the stage ring: the epilogue warps' staging tiles, then the barriers
 constexpr uint32_t kStoreBufTotal = kEpiWarps * kStoreBufBytes;
 
@@ -245,10 +247,11 @@ __global__ void wait_selftest_kernel(long long limit_cycles, int* gave_up) {
 }
 
 // One 32-column chunk of one accumulator row (held by this thread) through the epilogue.
+// n_end: first column that is not this tile's (the tile's end or the matrix's, whichever comes first).
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32], int row, bool row_ok, int n0, int split,
-                                               float& dot) {
-    const bool full_chunk = n0 + 32 <= p.N;
+                                               float& dot, int n_end) {
+    const bool full_chunk = n0 + 32 <= n_end;
     if (EPI == EPI_STORE) {
       if (row_ok) {
         __nv_bfloat16* o = p.out + (int64_t)row * p.ldo + n0;
@@ -265,12 +268,29 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
           for (int i = 0; i < 4; ++i)
             *reinterpret_cast<uint4*>(o + 8 * i) = make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
         } else {
+          // ragged chunk: whole 8-column pieces as 16-byte stores (the tail of a 208-column tile is two of them),
+          // the rest element by element
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            if (n0 + i < p.N) {
-              float a = __uint_as_float(v[i]);
-              if (p.col_scale) a *= __ldg(p.col_scale + n0 + i);
-              o[i] = __float2bfloat16_rn(a);
+          for (int i = 0; i < 4; ++i) {
+            if (n0 + 8 * i + 8 <= n_end) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float a = __uint_as_float(v[8 * i + 2 * e]), b = __uint_as_float(v[8 * i + 2 * e + 1]);
+                if (p.col_scale) { a *= __ldg(p.col_scale + n0 + 8 * i + 2 * e); b *= __ldg(p.col_scale + n0 + 8 * i + 2 * e + 1); }
+                __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                pk[e] = *reinterpret_cast<uint32_t*>(&h);
+              }
+              *reinterpret_cast<uint4*>(o + 8 * i) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                if (n0 + 8 * i + e < n_end) {
+                  float a = __uint_as_float(v[8 * i + e]);
+                  if (p.col_scale) a *= __ldg(p.col_scale + n0 + 8 * i + e);
+                  o[8 * i + e] = __float2bfloat16_rn(a);
+                }
+              }
             }
           }
         }
@@ -285,7 +305,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i)
-            if (n0 + i < p.N) o[i] = __uint_as_float(v[i]);
+            if (n0 + i < n_end) o[i] = __uint_as_float(v[i]);
         }
         if (p.qdot) {
           const __nv_bfloat16* qr = p.qdot + (int64_t)row * p.ldq + n0;
@@ -304,7 +324,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+              if (n0 + i < n_end) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
           }
         }
       }
@@ -329,7 +349,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+              if (n0 + i < n_end) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
           }
         }
         const float rs = p.row_scale ? __ldg(p.row_scale + row) : 1.f;
@@ -349,7 +369,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (n0 + i < p.N) o[i] = (p.accumulate ? o[i] : 0.f) + __uint_as_float(v[i]) * rs;
+              if (n0 + i < n_end) o[i] = (p.accumulate ? o[i] : 0.f) + __uint_as_float(v[i]) * rs;
           }
         } else {
           __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.wg_out) + (int64_t)row * p.ldo + n0;
@@ -379,7 +399,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (n0 + i < p.N)
+              if (n0 + i < n_end)
                 o[i] = __float2bfloat16_rn((p.accumulate ? __bfloat162float(o[i]) : 0.f) + __uint_as_float(v[i]) * rs);
           }
         }
@@ -389,9 +409,9 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, uint32_t (&v)[32
 
 // The row dot product <Q[row, n0..n0+31], acc> of the fused dz reduction, for the TMA-store path
 // (the other paths compute it inside epilogue_chunk).
-__device__ __forceinline__ void qdot_chunk(const Params& p, const uint32_t (&v)[32], int row, int n0, float& dot) {
+__device__ __forceinline__ void qdot_chunk(const Params& p, const uint32_t (&v)[32], int row, int n0, float& dot, int n_end) {
   const __nv_bfloat16* qr = p.qdot + (int64_t)row * p.ldq + n0;
-  if (n0 + 32 <= p.N) {
+  if (n0 + 32 <= n_end) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 raw = __ldg(reinterpret_cast<const uint4*>(qr + 8 * i));
@@ -406,7 +426,7 @@ __device__ __forceinline__ void qdot_chunk(const Params& p, const uint32_t (&v)[
   } else {
 #pragma unroll
     for (int i = 0; i < 32; ++i)
-      if (n0 + i < p.N) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
+      if (n0 + i < n_end) dot = fmaf(__uint_as_float(v[i]), __bfloat162float(qr[i]), dot);
   }
 }
 
@@ -467,6 +487,10 @@ __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap*
   const uint32_t t_row = t_acc + ((uint32_t)(q * 32) << 16);
   const int nchunks = (min(p.bn, n_limit - n_base) + 31) >> 5;   // 32-column chunks that hold columns of D
   const int ngroups = (nchunks + 1) >> 1;                    // 64-column groups
+  // An N tile that is not a multiple of 64 columns wide (208) ends inside its last group: the staged 64-column
+  // store would run into the next tile, so that group is written by per-thread stores masked at the tile's end
+  // (at the matrix's edge the tensor map clips, as for every tile).
+  const int tile_end = min(n_base + p.bn, p.N);
   float dot = 0.f;
   bool released = false;
   for (int g = h; g < ngroups; g += 2) {
@@ -486,10 +510,10 @@ __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap*
       released = true;
     }
     const int n0 = n_base + c0 * 32;
-    if (p.tma_store) {
+    if (p.tma_store && !(n0 + 64 > tile_end && tile_end < p.N)) {
       if (EPI != EPI_STORE && p.qdot && row_ok) {
-        qdot_chunk(p, v0, row, n0, dot);
-        if (two) qdot_chunk(p, v1, row, n0 + 32, dot);
+        qdot_chunk(p, v0, row, n0, dot, tile_end);
+        if (two) qdot_chunk(p, v1, row, n0 + 32, dot, tile_end);
       }
       if (lane == 0) tma_store_wait_read();   // the previous block has left the staging tile
       __syncwarp();
@@ -499,8 +523,8 @@ __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap*
       __syncwarp();
       if (lane == 0 && row0 + q * 32 < p.M) tma_store_2d(tmap_out, n0, row0 + q * 32, store_buf);   // never start a store outside the tensor
     } else {
-      epilogue_chunk<EPI>(p, v0, row, row_ok, n0, split, dot);
-      if (two) epilogue_chunk<EPI>(p, v1, row, row_ok, n0 + 32, split, dot);
+      epilogue_chunk<EPI>(p, v0, row, row_ok, n0, split, dot, tile_end);
+      if (two) epilogue_chunk<EPI>(p, v1, row, row_ok, n0 + 32, split, dot, tile_end);
     }
   }
   if (!released) {   // this warp had no group in the tile

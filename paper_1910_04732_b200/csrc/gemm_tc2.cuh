@@ -99,7 +99,8 @@ __device__ __forceinline__ uint32_t instr_desc2(bool a_mn, bool b_mn, int n) {
 }
 
 // bytes one CTA of the pair loads per stage: its 128 rows of A and half of the B tile
-__host__ __device__ inline uint32_t stage_bytes2(int bn) { return kATileBytes + (uint32_t)(bn / 2) * BK * 2; }
+// (rounded up to 1 KB: every stage must start on a swizzle-atom boundary, and half of a 208-column tile is 13 KB)
+__host__ __device__ inline uint32_t stage_bytes2(int bn) { return kATileBytes + (((uint32_t)(bn / 2) * BK * 2 + 1023u) & ~1023u); }
 
 }  // namespace tc
 }  // namespace flop

@@ -442,7 +442,7 @@ gemm2_chain_kernel(const __grid_constant__ GroupParams gp) {
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      const uint32_t sbuf = store_base + (uint32_t)(warp - 2) * kStoreBufBytes, t_acc = tmem_base + (uint32_t)(acc * gp.bn_max);
+      const uint32_t sbuf = store_base + (uint32_t)(warp - 2) * kStoreBufBytes, t_acc = tmem_base + (uint32_t)acc * acc_stride(gp.bn_max);
       const int row0 = it.tm * BM2 + (int)rank * BM;
       const uint32_t rel = map_to_cta(bars.tempty(acc), 0);
       if (p.kind == 0) {

@@ -68,7 +68,7 @@ __device__ __forceinline__ bool pair_mma_item(const GroupParams& gp, const Group
   const uint32_t idesc = instr_desc2(A_MN, B_MN, gp.prob[it.g].p.bn);
   if (!mbar_wait2(bars.tempty(acc), acc_phase ^ 1u, abort_flag)) return false;
   tcgen05_fence_after();
-  const uint32_t d_tmem = tmem_base + (uint32_t)(acc * gp.bn_max);
+  const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_stride(gp.bn_max);
   for (int kb = it.kb0; kb < it.kb1; ++kb) {
     if (!mbar_wait2(bars.full(stage), phase, abort_flag)) return false;
     tcgen05_fence_after();
@@ -176,7 +176,7 @@ gemm2_dual_kernel(const __grid_constant__ GroupParams gp) {
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      const uint32_t sbuf = store_base + (uint32_t)(warp - 2) * kStoreBufBytes, t_acc = tmem_base + (uint32_t)(acc * gp.bn_max);
+      const uint32_t sbuf = store_base + (uint32_t)(warp - 2) * kStoreBufBytes, t_acc = tmem_base + (uint32_t)acc * acc_stride(gp.bn_max);
       const int row0 = it.tm * BM2 + (int)rank * BM;
       const uint32_t rel = map_to_cta(bars.tempty(acc), 0);
       if (p.kind == 0) run_epilogue<E0, true>(p, &gp.prob[it.g].tout, sbuf, t_acc, row0, it.tn * p.bn, it.n_limit, it.split, it.tn, warp, lane, rel);

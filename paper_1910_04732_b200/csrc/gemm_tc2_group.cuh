@@ -112,7 +112,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
         const uint32_t idesc = instr_desc2(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait2(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * gp.bn_max);
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_stride(gp.bn_max);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait2(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tcgen05_fence_after();
@@ -144,7 +144,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      run_epilogue<EPI, true>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.n_limit, it.split, it.tn,
+      run_epilogue<EPI, true>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)acc * acc_stride(gp.bn_max), it.tm * BM2 + (int)rank * BM, it.tn * p.bn, it.n_limit, it.split, it.tn,
                               warp, lane, map_to_cta(tempty_bar(acc), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }

@@ -183,7 +183,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
         const uint32_t idesc = instr_desc(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tcgen05_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * gp.bn_max);
+        const uint32_t d_tmem = tmem_base + (uint32_t)acc * acc_stride(gp.bn_max);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tcgen05_fence_after();
@@ -215,7 +215,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      run_epilogue<EPI, false>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)(acc * gp.bn_max), it.tm * BM, it.tn * p.bn, it.n_limit, it.split, it.tn, warp, lane,
+      run_epilogue<EPI, false>(p, &gp.prob[it.g].tout, store_base + (uint32_t)(warp - 2) * kStoreBufBytes, tmem_base + (uint32_t)acc * acc_stride(gp.bn_max), it.tm * BM, it.tn * p.bn, it.n_limit, it.split, it.tn, warp, lane,
                                tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }

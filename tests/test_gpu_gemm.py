@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from paper_1910_04732_b200 import inputs as I
-from tests._util import empty_dev, host, rel_fro, to_dev
+from tests._util import assert_close, empty_dev, host, rel_fro, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -27,7 +27,7 @@ def _operands(M, N, K, seed):
 
 SHAPES = [(128, 64, 64), (256, 256, 128), (300, 200, 136), (1000, 410, 410), (520, 72, 900), (77, 768, 520),
           (2048, 768, 768)]
-TILES = [(0, -1), (64, 0), (128, 0), (192, 0), (256, 0), (64, 1), (128, 1), (192, 1), (256, 1)]
+TILES = [(0, -1), (64, 0), (128, 0), (192, 0), (256, 0), (64, 1), (128, 1), (192, 1), (208, 1), (256, 1)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -38,9 +38,12 @@ def test_k_major_operands(b, M, N, K, bn, cta2):
     scale = np.linspace(0.0, 2.0, N).astype(np.float32)
     b.tc_gemm(to_dev(A, "bf16"), False, to_dev(B, "bf16"), False, M, N, K, D=D, bn=bn, cta2=cta2)
     assert rel_fro(host(D), want) < 4e-3            # one bf16 rounding of the output
+    assert_close(D, want, "bf16", "D")              # and no element or block off (tile seams, ragged tails)
+    D.fill_(float("nan"))
     b.tc_gemm(to_dev(A, "bf16"), False, to_dev(B, "bf16"), False, M, N, K, D=D,
               col_scale=torch.from_numpy(scale).cuda(), bn=bn, cta2=cta2)
     assert rel_fro(host(D), want * scale[None, :]) < 4e-3
+    assert_close(D, want * scale[None, :], "bf16", "D scaled")
     assert np.all(host(D)[:, 0] == 0)               # a closed gate zeroes its column exactly
     assert b.device_status() == b.OK
 
