@@ -71,9 +71,10 @@ inline bool debug_on() {
 //   FLOP_STAGE_MERGE=0     backward in three launches per stage instead of two shared ones
 //   FLOP_GATHER_PIPE=0     plain P gather kernel                     FLOP_NO_CHAIN=1   chained calls run unchained
 //   FLOP_CHAIN_STAGES=2    chained calls put dependent products in ONE launch (default 1: a launch per stage)
+//   FLOP_SCHED_EPI=c       per-tile fixed cost (SM cycles) in the tile schedule's cost model instead of 400 + 4 bn
 struct Tuning {
   int no_pdl = 0, tc_bn = 0, tc_stages = 0, tc_cta2 = 0, no_tma_store = 0, no_sched = 0, group_bn = 0, group_cta2 = 0,
-      wgrad_bn = 0, wgrad_cta2 = 0, no_small_t = 0, no_skinny = 0, stage_merge = 1, gather_pipe = 1, no_chain = 0, chain_stages = 1;
+      wgrad_bn = 0, wgrad_cta2 = 0, no_small_t = 0, no_skinny = 0, stage_merge = 1, gather_pipe = 1, no_chain = 0, chain_stages = 1, sched_epi = 0;
 };
 inline const Tuning& tuning() {
   static const Tuning t = [] {
@@ -85,7 +86,7 @@ inline const Tuning& tuning() {
     v.group_bn = get("FLOP_TC_GROUP_BN", 0); v.group_cta2 = get("FLOP_TC_GROUP_CTA2", 0); v.wgrad_bn = get("FLOP_TC_WGRAD_BN", 0);
     v.wgrad_cta2 = get("FLOP_TC_WGRAD_CTA2", 0); v.no_small_t = get("FLOP_NO_SMALL_T", 0); v.no_skinny = get("FLOP_NO_SKINNY", 0);
     v.stage_merge = get("FLOP_STAGE_MERGE", 1); v.gather_pipe = get("FLOP_GATHER_PIPE", 1); v.no_chain = get("FLOP_NO_CHAIN", 0);
-    v.chain_stages = get("FLOP_CHAIN_STAGES", 1);
+    v.chain_stages = get("FLOP_CHAIN_STAGES", 1); v.sched_epi = get("FLOP_SCHED_EPI", 0);
 #endif
     return v;
   }();
@@ -433,7 +434,7 @@ int add_problem(tc::GroupParams& gp, const TcJob& j, std::vector<double>& item_c
   pr.work_begin = gp.total_work;
   gp.total_work += p.tiles_m * p.tiles_n * p.splits;
   const double bytes = j.pl.cta2 ? (double)tc::stage_bytes2(p.bn) : (double)tc::stage_bytes(p.bn);
-  const double per_kb = std::max(2.0 * p.bn, bytes / 50.0), epi = 400.0 + 4.0 * p.bn;
+  const double per_kb = std::max(2.0 * p.bn, bytes / 50.0), epi = tuning().sched_epi > 0 ? (double)tuning().sched_epi : 400.0 + 4.0 * p.bn;
   if (item_cost.size() <= (size_t)tc::kMaxSched)
     for (int sp = 0; sp < p.splits; ++sp) {
       const int kbs = std::min(p.kb_per_split, p.num_kb - sp * p.kb_per_split);
@@ -1737,6 +1738,7 @@ int flop_scale_rows_grouped(const flop_scale_rows_t* pr, int n, int dt, void* st
   for (int i0 = 0; i0 < n; i0 += kScaleGroup) {
     ScaleRowsGroup g;
     memset(&g, 0, sizeof(g));
+    int64_t max_units = 0;
     for (; g.n < kScaleGroup && i0 + g.n < n; ++g.n) {
       const flop_scale_rows_t& a = pr[i0 + g.n];
       if (a.r < 0 || a.d_in < 0 || a.r > INT32_MAX || a.d_in > INT32_MAX) return FLOP_ERR_INVALID_ARG;
@@ -1744,12 +1746,11 @@ int flop_scale_rows_grouped(const flop_scale_rows_t* pr, int n, int dt, void* st
       if (a.r > 0 && a.d_in > 0 && (!bf16_ok(a.Q, a.ldq) || !bf16_ok(a.Qz, a.ldqz))) return FLOP_ERR_UNSUPPORTED;
       ScaleRows& o = g.a[g.n];
       o.Q = (const bf16*)a.Q; o.ldq = a.ldq; o.z = a.z; o.Qz = (bf16*)a.Qz; o.ldqz = a.ldqz; o.rows = (int)a.r; o.cols = (int)a.d_in;
-      g.unit_begin[g.n + 1] = g.unit_begin[g.n] + (int64_t)o.rows * ((o.cols + 7) >> 3);
+      if (o.cols > 0) max_units = std::max<int64_t>(max_units, o.rows);
     }
-    const int64_t units = g.unit_begin[g.n];
-    if (units <= 0) continue;
-    const int grid = (int)std::min<int64_t>((units + 4 * 256 - 1) / (4 * 256), (int64_t)num_sms() * 8);
-    launch_k(scale_rows_group_kernel, dim3(grid), dim3(256), (size_t)0, st, g);
+    if (max_units <= 0) continue;
+    const int gx = (int)std::min<int64_t>((max_units + kScaleRows - 1) / kScaleRows, 1024);
+    launch_k(scale_rows_group_kernel, dim3((unsigned)gx, (unsigned)g.n), dim3(256), (size_t)0, st, g);
     count_launch();
     FLOP_CUDA(cudaGetLastError());
   }

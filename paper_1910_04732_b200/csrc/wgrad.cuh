@@ -260,61 +260,55 @@ dalpha_group_kernel(const __grid_constant__ DlaFinishGroup g, int accumulate) {
 }
 
 // diag(z) Q of many matrices in one launch (it depends only on the gate sample and the weights, so a training
-// step forms it once, right after sampling, for every matrix of the model).  16-byte units, four per thread in
-// flight; rows are 16-byte aligned.
+// step forms it once, right after sampling, for every matrix of the model).  16-byte units; rows are 16-byte aligned.
 constexpr int kScaleGroup = 96;
 struct ScaleRows { const __nv_bfloat16* Q; int64_t ldq; const float* z; __nv_bfloat16* Qz; int64_t ldqz; int rows, cols; };
 struct ScaleRowsGroup {
   ScaleRows a[kScaleGroup];
-  int64_t unit_begin[kScaleGroup + 1];
   int n;
 };
 
+// blockIdx.y = matrix.  A block takes kScaleRows rows at a time, four per warp; a warp reads 512 consecutive bytes
+// of each of its rows per pass and keeps the loads of its four rows (two passes) in flight before it stores.
+constexpr int kScaleRows = 32;
 __global__ void __launch_bounds__(256)
 scale_rows_group_kernel(const __grid_constant__ ScaleRowsGroup g) {
   pdl_wait();
   pdl_launch_dependents();
-  const int64_t total = g.unit_begin[g.n];
-  const int64_t step = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t u0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u0 < total; u0 += 4 * step) {
-    uint4 raw[4];
+  const ScaleRows& a = g.a[blockIdx.y];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int r0 = blockIdx.x * kScaleRows; r0 < a.rows; r0 += gridDim.x * kScaleRows) {
     float gate[4];
-    __nv_bfloat16* dst[4];
-    bool full[4];
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int64_t u = u0 + b * step;
-      dst[b] = nullptr; full[b] = false; gate[b] = 0.f; raw[b] = make_uint4(0u, 0u, 0u, 0u);
-      if (u >= total) continue;
-      int lo = 0, hi = g.n - 1;            // the matrix that owns unit u
-      while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (u >= g.unit_begin[mid]) lo = mid; else hi = mid - 1;
-      }
-      const ScaleRows& a = g.a[lo];
-      const int c8 = (a.cols + 7) >> 3;
-      const int64_t v = u - g.unit_begin[lo];
-      const int row = (int)(v / c8), c0 = (int)(v - (int64_t)row * c8) * 8;
-      const __nv_bfloat16* q = a.Q + (int64_t)row * a.ldq + c0;
-      dst[b] = a.Qz + (int64_t)row * a.ldqz + c0;
-      gate[b] = __ldg(a.z + row);
-      if (c0 + 8 <= a.cols) {
-        full[b] = true;
-        raw[b] = __ldg(reinterpret_cast<const uint4*>(q));
-      } else {
-        for (int k = 0; k < a.cols - c0; ++k) dst[b][k] = __float2bfloat16_rn(__bfloat162float(q[k]) * gate[b]);
-      }
+    for (int i = 0; i < 4; ++i) {
+      const int row = r0 + warp + 8 * i;
+      gate[i] = row < a.rows ? __ldg(a.z + row) : 0.f;
     }
+    for (int c0 = lane * 8; c0 < a.cols; c0 += 512) {
+      uint4 raw[8];
+      bool full[8];
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      if (!full[b]) continue;
-      __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw[b]);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 x = __bfloat1622float2(h[e]);
-        h[e] = __floats2bfloat162_rn(x.x * gate[b], x.y * gate[b]);
+      for (int j = 0; j < 8; ++j) {
+        const int row = r0 + warp + 8 * (j & 3), c = c0 + 256 * (j >> 2);
+        full[j] = row < a.rows && c + 8 <= a.cols;
+        if (full[j]) raw[j] = __ldcs(reinterpret_cast<const uint4*>(a.Q + (int64_t)row * a.ldq + c));
       }
-      *reinterpret_cast<uint4*>(dst[b]) = raw[b];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int row = r0 + warp + 8 * (j & 3), c = c0 + 256 * (j >> 2);
+        if (full[j]) {
+          __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&raw[j]);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 x = __bfloat1622float2(h[e]);
+            h[e] = __floats2bfloat162_rn(x.x * gate[j & 3], x.y * gate[j & 3]);
+          }
+          *reinterpret_cast<uint4*>(a.Qz + (int64_t)row * a.ldqz + c) = raw[j];
+        } else if (row < a.rows && c < a.cols) {            // ragged last piece of a row
+          for (int k = 0; k < a.cols - c; ++k)
+            a.Qz[(int64_t)row * a.ldqz + c + k] = __float2bfloat16_rn(__bfloat162float(a.Q[(int64_t)row * a.ldq + c + k]) * gate[j & 3]);
+        }
+      }
     }
   }
 }

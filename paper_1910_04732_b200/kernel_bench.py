@@ -104,10 +104,23 @@ def main():
                  2 * d_out * r + 2 * k * d_out + 4 * k * d_in + 4 * r, t_all - t_sel))
     del P, Q, Pc, Qc
 
-    print(f"HBM peak used: {peak:.0f} GB/s (measured copy)\n")
-    print(f"{'kernel(s)':44s} {'size':58s} {'MB':>9s} {'us':>9s} {'GB/s':>8s} {'of peak':>8s}")
+    # ---- diag(z) Q of every matrix of a model in one launch: 2 B read + 2 B written per element
+    wl = I.WORKLOADS["bert"]
+    reps = 1 if args.small else 4          # four models' worth of matrices: 255 MB read, 255 MB written (beyond L2)
+    qs = []
+    for _ in range(reps):
+        for _, _, mm in wl.all_matrices():
+            q = torch.randn(mm.r, mm.d_in, generator=g, device="cuda").bfloat16()
+            qs.append((q, torch.rand(mm.r, generator=g, device="cuda"), torch.empty_like(q)))
+    arr = b.problem_array([b.scale_rows_problem(q, zz, o) for q, zz, o in qs])
+    t = timed(lambda: b.scale_rows_grouped(arr))
+    rows.append(("scale_rows_group_kernel", f"{len(qs)} bert-shaped factors Q (r x d_in)", sum(4 * q.numel() for q, _, _ in qs), t))
+    del qs
+
+    print(f"HBM peak used: {peak:.0f} GB/s (measured copy); 'of 8 TB/s' = against the nominal figure\n")
+    print(f"{'kernel(s)':44s} {'size':58s} {'MB':>9s} {'us':>9s} {'GB/s':>8s} {'of peak':>8s} {'of 8 TB/s':>10s}")
     for name, what, nbytes, t in rows:
-        print(f"{name:44s} {what:58s} {nbytes / 1e6:9.1f} {t * 1e6:9.1f} {nbytes / t / 1e9:8.0f} {nbytes / t / 1e9 / peak:8.2f}")
+        print(f"{name:44s} {what:58s} {nbytes / 1e6:9.1f} {t * 1e6:9.1f} {nbytes / t / 1e9:8.0f} {nbytes / t / 1e9 / peak:8.2f} {nbytes / t / 1e9 / 8000.0:10.2f}")
 
     if args.only_membound:
         return
@@ -141,11 +154,58 @@ def main():
         flops = 2.0 * T * k * (mtx.d_in + mtx.d_out)
         wbytes = 2.0 * k * (mtx.d_in + mtx.d_out)
         print(f"{T:6d} {tc_ * 1e6:15.1f} {tch * 1e6:17.1f} {tg_ * 1e6:13.1f} {tg_ / tc_:9.2f} {flops / tc_ / 1e9:16.0f} {wbytes / tc_ / 1e9:12.0f}")
+    library_table(g)
     # ---- training on the active rank components: one BERT-shaped layer (six matrices, T = 4096)
     for wl in ("bert", "sru"):
         active_table(I.WORKLOADS[wl], g)
     embedding_table(g)
     assert b.device_status() == b.OK
+
+
+def library_table(g):
+    """Context for the roofline denominators: the six products of every matrix of one layer issued one by one through
+    the vendor library (torch.matmul on the same bf16 tensors, outputs preallocated, replayed from a CUDA graph; no
+    gate, no dlog_alpha), beside this library's grouped forward + backward of the same layer.  The measured bf16 peak
+    is the library's rate on an 8192^3 product; this is its rate on the products this path is made of."""
+    bf = torch.bfloat16
+    print("\none layer, forward + backward: this library's grouped calls against the six products per matrix through torch.matmul")
+    print(f"{'workload':>9s} {'grouped us':>11s} {'TFLOP/s':>8s} {'torch.matmul us':>16s} {'TFLOP/s':>8s}")
+    for name in ("bert", "txl", "sru"):
+        w = I.WORKLOADS[name]
+        T = w.T
+        es = []
+        for m in w.matrices:
+            r8 = lambda v: (v + 7) // 8 * 8
+            rnd = lambda a, c: torch.randn(a, r8(c), generator=g, device="cuda").to(bf)[:, :c]
+            e = dict(m=m, X=rnd(T, m.d_in), dY=rnd(T, m.d_out), Q=rnd(m.r, m.d_in), P=rnd(m.d_out, m.r),
+                     z=torch.rand(m.r, device="cuda"), dzd=torch.rand(m.r, device="cuda"))
+            e["Y"], e["H"], e["dX"] = (b.padded(T, c, bf) for c in (m.d_out, m.r, m.d_in))
+            e["dH"], e["dP"], e["dQ"] = b.padded(T, m.r, bf), b.padded(m.d_out, m.r, bf), b.padded(m.r, m.d_in, bf)
+            e["dla"] = torch.zeros(m.r, device="cuda")
+            e["ws"] = b.alloc_workspace(b.workspace_bytes(b.OP_BWD, T, m.d_in, m.d_out, m.r, b.BF16))
+            es.append(e)
+        fwd = b.problem_array([b.fwd_problem(e["X"], e["Q"], e["P"], e["z"], e["Y"], e["H"]) for e in es])
+        bwd = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Q"], e["P"], e["z"], e["dzd"], e["H"], e["dX"], e["dP"], e["dQ"],
+                                             e["dla"], e["ws"]) for e in es])
+
+        def ours():
+            b.gated_lowrank_fwd_grouped(fwd)
+            b.gated_lowrank_bwd_grouped(bwd)
+
+        def library():
+            for e in es:
+                torch.matmul(e["X"], e["Q"].t(), out=e["H"])
+                torch.matmul(e["H"], e["P"].t(), out=e["Y"])
+                torch.matmul(e["dY"], e["P"], out=e["dH"])
+                torch.matmul(e["dY"].t(), e["H"], out=e["dP"])
+                torch.matmul(e["dH"].t(), e["X"], out=e["dQ"])
+                torch.matmul(e["dH"], e["Q"], out=e["dX"])
+        t_o = timed(ours, iters=20, graph=True)
+        t_l = timed(library, iters=20, graph=True)
+        flops = sum(6.0 * T * m.r * (m.d_in + m.d_out) for m in w.matrices)
+        print(f"{name:>9s} {t_o * 1e6:11.1f} {flops / t_o / 1e12:8.0f} {t_l * 1e6:16.1f} {flops / t_l / 1e12:8.0f}")
+        del es
+        torch.cuda.empty_cache()
 
 
 def embedding_table(g):
