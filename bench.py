@@ -63,9 +63,8 @@ def roofline_traffic(workload: str, group: int):
                 fields[k.strip()] = v.strip()
         h = hashlib.sha1()
         d = os.path.join(ROOT, "paper_1910_04732_b200", "csrc")
-        for f in sorted(os.listdir(d)):
-            if f.startswith("gemm_tc") or f == "schedule.cuh":
-                h.update(open(os.path.join(d, f), "rb").read())
+        for f in ("gemm_tc.cuh", "gemm_tc2.cuh", "gemm_tc_group.cuh", "gemm_tc2_group.cuh", "gemm_tc2_dual.cuh", "schedule.cuh"):
+            h.update(open(os.path.join(d, f), "rb").read())
         if fields.get("workload") != workload or int(fields.get("matrices_per_call", -1)) != group:
             return None, "no capture for this workload"
         if fields.get("kernel_sources_sha1") != h.hexdigest():

@@ -53,14 +53,16 @@ compact_select_kernel(const float* __restrict__ in, int mode, double thr, int r,
           if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
         }
         __syncthreads();
-        if (tid == 0) {
-          int acc = 0, b = 255;
-          for (; b > 0; --b) {
-            if (acc + hist[b] >= need) break;
-            acc += hist[b];
+        {
+          // the bin that holds the need-th largest key: a block scan over the bins from the top (thread t holds bin
+          // 255 - t), instead of one thread walking 256 counters
+          const int h = tid < 256 ? hist[255 - tid] : 0;
+          int tot = 0;
+          const int above = block_exclusive_scan(h, scan_scratch, &tot);
+          if (tid < 256 && above < need && need <= above + h) {
+            s_prefix = prefix | ((uint32_t)(255 - tid) << shift);
+            s_need = need - above;
           }
-          s_prefix = prefix | ((uint32_t)b << shift);
-          s_need = need - acc;
         }
         __syncthreads();
         prefix = s_prefix;
