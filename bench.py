@@ -2,16 +2,21 @@
 """Benchmark of the FLOP gated low-rank hot path on B200.
 
 One step = one pass of the whole hot path over one batch of synthetic input:
-sample every gate of every layer (one launch), then for every factorized matrix
-of every layer the gated forward (2 GEMMs) and backward (4 GEMMs + the fused
-dlog_alpha reduction; grouped per layer into two forward and two backward launches), then the expected-L0 / Lagrangian term over all gates.
+sample every gate of every layer (one launch), form diag(z)Q of every matrix
+(one launch), then for every factorized matrix of every layer the gated forward
+(2 GEMMs) and backward (4 GEMMs + the fused dlog_alpha row dots; grouped per
+layer into two forward and two backward launches), the second stage of
+dlog_alpha for every matrix (one launch), then the expected-L0 / Lagrangian term
+over all gates.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload bert|sru|txl] [--impl ours|reference]
 
 Prints ONE JSON line.  `value` is tokens/s with inputs resident in HBM; `e2e`
-is the same step fed from pinned host memory (H2D of every X and dY inside the
-timed region, D2H of dlog_alpha and the Lagrangian scalars); `roofline` times
-the tensor-core GEMM launches with CUDA events; `cpu_baseline` is the fp64
+is the same step through the same calls with every X and dY copied from pinned
+host memory and Y, dX, all weight gradients, dlog_alpha and the Lagrangian
+scalars copied back inside the timed region; `roofline` times the tensor-core
+GEMM launches with device-side stamps inside the replayed CUDA graph (and, for
+comparison, with CUDA events in an eager pass); `cpu_baseline` is the fp64
 oracle timed on the host cores on a bounded sample.  `--impl reference` times
 the oracle alone.  Under torchrun every rank processes its own token batch
 with the same gate sample and the weight gradients are all-reduced (NCCL).
@@ -330,7 +335,7 @@ class Job:
         self.finish(deferred=self.group > 0 and not self.chain and not self.plain)
 
 
-def capture_step(job: Job, fn=None, stamps=None):
+def capture_step(job: Job, fn=None, stamps=None, acc=None):
     """One whole step captured in a CUDA graph (the library's launches, programmatic dependent
     launch edges included); replays cost one host call instead of ~25."""
     import torch
@@ -345,6 +350,8 @@ def capture_step(job: Job, fn=None, stamps=None):
             job.b.gemm_stamps_begin(stamps)
         with torch.cuda.graph(g, stream=side):
             fn()
+            if stamps is not None and acc is not None:      # adds this replay's GEMM kernel time up on the device
+                job.b.gemm_stamps_accumulate(stamps, acc)
         if stamps is not None:
             job.stamped = job.b.gemm_stamps_end()
     torch.cuda.current_stream().wait_stream(side)
@@ -518,7 +525,7 @@ def main():
     ap.add_argument("--no-active", action="store_true", help="skip the extra active-rank-training measurement")
     ap.add_argument("--no-graph", action="store_true", help="issue every step from the host instead of replaying a CUDA graph")
     ap.add_argument("--chain", action="store_true", help="chained calls (one launch for the forward products, one for the backward pass of a layer, "
-                    "ordered on the device) instead of the grouped calls (a launch per GEMM stage); measured slower on B200, see profiles/")
+                    "ordered on the device) instead of the grouped calls (a launch per GEMM stage); measured slower on B200")
     ap.add_argument("--no-chain", action="store_true", help="(default) grouped calls")
     ap.add_argument("--plain", action="store_true", help="every backward call forms diag(z) Q and finishes dlog_alpha itself "
                     "(two more small launches per layer) instead of one launch per step for each")
@@ -566,36 +573,33 @@ def main():
     launches = b.launch_count() - n0            # kernels of this library per step (the same inside a graph replay)
     use_graph = not args.no_graph and world == 1   # NCCL all-reduces stay outside graphs here
     stamps = torch.zeros(2 * 4096, dtype=torch.int64, device="cuda") if use_graph else None
+    acc = torch.zeros(2, dtype=torch.int64, device="cuda") if use_graph else None
     if use_graph:
-        capture_step(job, stamps=stamps)
+        capture_step(job, stamps=stamps, acc=acc)
+        launches += 1                              # the stamp-adding kernel at the end of the captured step
         for _ in range(3):
             job.graph.replay()
+        torch.cuda.synchronize()
+        acc.zero_()
     torch.cuda.synchronize()
     ms = time_steps(job, args.steps, world, use_graph)
     # Roofline of the dominant kernels (the tensor-core GEMM launches).  Inside the replayed graph every launch
-    # stamps %globaltimer when its first CTA passes the dependency wait and when its last CTA ends; a second pass
-    # replays the same graph, reads the stamps after EVERY replay and brackets each replay with events, so that
-    # the kernel time and the step time it is compared with come from the same replays.
+    # stamps %globaltimer when its first CTA passes the dependency wait and when its last CTA ends, and a one-block
+    # kernel at the end of the captured step adds (end - start) of all of them to a device counter: the kernel time
+    # comes from the very replays whose step time is the headline, with no host work in between.
     graph_gemm = None
     if use_graph:
         n_st, fl_st = job.stamped
-        k_rep = max(3, min(args.steps, 50))
-        kern_ms, step_ms_rep = [], []
-        for _ in range(k_rep):
-            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            r0.record(); job.graph.replay(); r1.record()
-            torch.cuda.synchronize()
+        tot_ns, n_rep = (int(v) for v in acc.cpu().tolist())
+        if os.environ.get("FLOP_BENCH_DUMP_STAMPS"):
             st = stamps[: 2 * n_st].view(n_st, 2).cpu().numpy()
-            kern_ms.append(float((st[:, 1] - st[:, 0]).clip(min=0).sum()) / 1e6)
-            step_ms_rep.append(r0.elapsed_time(r1))
-            if os.environ.get("FLOP_BENCH_DUMP_STAMPS") and len(kern_ms) == k_rep:
-                rel = (st - st[0, 0]) / 1e3
-                print("stamps_us " + " ".join(f"[{a:.1f},{b:.1f}]" for a, b in rel[:16]), file=sys.stderr)
-        if n_st > 0 and min(kern_ms) > 0:
-            km, sm = float(np.mean(kern_ms)), float(np.mean(step_ms_rep))
-            graph_gemm = {"launches": n_st, "replays": k_rep, "kernel_ms_per_step": km, "step_ms_same_replays": sm,
+            rel = (st - st[0, 0]) / 1e3
+            print("stamps_us " + " ".join(f"[{a:.1f},{b:.1f}]" for a, b in rel[:16]), file=sys.stderr)
+        if n_st > 0 and n_rep == args.steps and tot_ns > 0:
+            km = tot_ns / 1e6 / n_rep
+            graph_gemm = {"launches": n_st, "replays": n_rep, "kernel_ms_per_step": km, "step_ms_same_replays": ms / args.steps,
                           "tflops": fl_st / (km * 1e-3) / 1e12, "flops_per_step": fl_st}
-            assert km <= sm * 1.005, f"stamped kernel time {km:.3f} ms exceeds the step it was taken in ({sm:.3f} ms)"
+            assert km <= ms / args.steps * 1.005, f"stamped kernel time {km:.3f} ms exceeds the step it was taken in"
     # the same launches issued eagerly with CUDA events recorded around every GEMM launch (no dependent-launch overlap)
     b.gemm_timing_begin()
     ms_timed_pass = time_steps(job, args.steps, world)

@@ -118,6 +118,12 @@ int flop_gemm_timing_end(double* total_ms, double* total_flops, int64_t* launche
  * Single-threaded use only, like the event timing above. */
 int flop_gemm_stamps_begin(unsigned long long* stamps_dev, int capacity);
 int flop_gemm_stamps_end(int* launches, double* total_flops);
+/* One small kernel on `stream`: acc_dev[0] += the sum of (end - start) over the `capacity` stamp pairs of stamps_dev
+ * that have been written (unwritten pairs are zero), acc_dev[1] += 1 (DEVICE u64[2], zeroed by the caller).  Issued
+ * at the end of a step that is captured in a CUDA graph, it adds up the GEMM kernel time of every replay on the
+ * device, in the very replays that are being timed. */
+int flop_gemm_stamps_accumulate(const unsigned long long* stamps_dev, int capacity, unsigned long long* acc_dev,
+                                void* stream);
 
 /* Bytes of scratch the given call needs (HOST out pointer).  For FLOP_OP_L0
  * pass the total number of gates as T and the number of segments as r. */

@@ -22,7 +22,7 @@ OP_FWD, OP_BWD, OP_L0, OP_COMPACT, OP_COMPACT_FWD, OP_EMBEDDING_BWD = range(6)
 
 EXPORTS = ("flop_status_string", "flop_last_async_status", "flop_device_status", "flop_sync_bytes",
            "flop_gated_lowrank_fwd_chained", "flop_gated_lowrank_bwd_chained", "flop_selftest_wait_timeout", "flop_launch_count", "flop_plan_tile_schedule", "flop_plan_chain_queue", "flop_scale_rows_grouped", "flop_dlog_alpha_finish_grouped", "flop_gemm_timing_begin",
-           "flop_gemm_timing_end", "flop_gemm_stamps_begin", "flop_gemm_stamps_end", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
+           "flop_gemm_timing_end", "flop_gemm_stamps_begin", "flop_gemm_stamps_end", "flop_gemm_stamps_accumulate", "flop_workspace_bytes", "flop_tc_gemm", "flop_gate_sample", "flop_gate_sample_devoff",
            "flop_gated_lowrank_fwd", "flop_gated_lowrank_bwd", "flop_gated_lowrank_fwd_grouped",
            "flop_gated_lowrank_bwd_grouped", "flop_active_ranks_gather", "flop_active_ranks_scatter",
            "flop_expected_l0_lagrangian",
@@ -119,6 +119,7 @@ def load_library() -> ctypes.CDLL:
                                  ctypes.POINTER(ctypes.c_int), vp]
     lib.flop_gemm_stamps_begin.argtypes = [vp, ci]
     lib.flop_gemm_stamps_end.argtypes = [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double)]
+    lib.flop_gemm_stamps_accumulate.argtypes = [vp, ci, vp, vp]
     lib.flop_gate_sample.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp]
     lib.flop_gate_sample_devoff.argtypes = [vp, i64, HcParams, ctypes.c_uint64, ctypes.c_uint64, vp, vp, vp, vp, vp]
     lib.flop_gated_lowrank_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, vp, i64, vp, i64,
@@ -247,6 +248,13 @@ def gemm_stamps_end():
     n, fl = ctypes.c_int(0), ctypes.c_double(0)
     _check(load_library().flop_gemm_stamps_end(ctypes.byref(n), ctypes.byref(fl)), "flop_gemm_stamps_end")
     return int(n.value), fl.value
+
+
+def gemm_stamps_accumulate(stamps: torch.Tensor, acc: torch.Tensor) -> None:
+    """acc (zeroed int64[2] device tensor): [0] += stamped GEMM kernel time (ns) of the step just issued, [1] += 1."""
+    assert stamps.element_size() == 8 and acc.element_size() == 8 and acc.numel() >= 2
+    _check(load_library().flop_gemm_stamps_accumulate(_ptr(stamps), stamps.numel() // 2, _ptr(acc), _stream()),
+           "flop_gemm_stamps_accumulate")
 
 
 def device_status() -> int:

@@ -991,6 +991,36 @@ int flop_gemm_stamps_begin(unsigned long long* stamps_dev, int capacity) {
   return FLOP_OK;
 }
 
+// acc[0] += sum over the stamp pairs of (end - start) where both were written; acc[1] += 1.
+__global__ void __launch_bounds__(256)
+stamps_accumulate_kernel(const unsigned long long* __restrict__ stamps, int capacity, unsigned long long* __restrict__ acc) {
+  pdl_wait();
+  pdl_launch_dependents();
+  __shared__ unsigned long long part[8];
+  unsigned long long s = 0;
+  for (int i = threadIdx.x; i < capacity; i += blockDim.x) {
+    const unsigned long long a = stamps[2 * i], e = stamps[2 * i + 1];
+    if (a != 0 && e > a) s += e - a;
+  }
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long t = 0;
+    for (int w = 0; w < 8; ++w) t += part[w];
+    acc[0] += t;
+    acc[1] += 1;
+  }
+}
+
+int flop_gemm_stamps_accumulate(const unsigned long long* stamps_dev, int capacity, unsigned long long* acc_dev, void* stream) {
+  if (!stamps_dev || capacity <= 0 || !acc_dev) return FLOP_ERR_INVALID_ARG;
+  launch_k(stamps_accumulate_kernel, dim3(1), dim3(256), (size_t)0, (cudaStream_t)stream, stamps_dev, capacity, acc_dev);
+  count_launch();
+  FLOP_CUDA(cudaGetLastError());
+  return FLOP_OK;
+}
+
 int flop_gemm_stamps_end(int* launches, double* total_flops) {
   if (launches) *launches = g_stamps.used;
   if (total_flops) *total_flops = g_stamps.flops;

@@ -20,7 +20,7 @@ def b():
     return binding
 
 
-def _run(b, w: I.Workload, seed, alpha_shift=0.0, wdt=torch.bfloat16, accumulate=False):
+def _run(b, w: I.Workload, seed, alpha_shift=0.0, wdt=torch.bfloat16, accumulate=False, chained=False):
     bf = torch.bfloat16
     es, gat, fwd, bwd, sca = [], [], [], [], []
     for i, m in enumerate(w.matrices):
@@ -55,8 +55,14 @@ def _run(b, w: I.Workload, seed, alpha_shift=0.0, wdt=torch.bfloat16, accumulate
         es.append(e)
     wd = b.BF16 if wdt == torch.bfloat16 else b.F32
     b.active_ranks_gather(gat)
-    b.gated_lowrank_fwd_grouped(fwd)
-    b.gated_lowrank_bwd_grouped(bwd, wgrad_dt=wd)
+    if chained:
+        sync = b.alloc_sync()
+        b.gated_lowrank_fwd_chained(fwd, sync)
+        b.gated_lowrank_bwd_chained(bwd, sync, wgrad_dt=wd)
+        assert int(sync.view(torch.int32).abs().sum().item()) == 0
+    else:
+        b.gated_lowrank_fwd_grouped(fwd)
+        b.gated_lowrank_bwd_grouped(bwd, wgrad_dt=wd)
     b.active_ranks_scatter(sca, accumulate=accumulate, wgrad_dt=wd)
     assert b.device_status() == b.OK
     for e in es:
@@ -106,3 +112,10 @@ def test_active_ranks_fp32_weight_gradients_and_accumulate(b):
     w = I.Workload("a", "bf16", 500, 1, (I.Matrix("x", 264, 520, 200), I.Matrix("y", 384, 64, 192)), ("bimodal", 3.0, 0.5), 0.5)
     _run(b, w, 2, wdt=torch.float32)
     _run(b, w, 2, accumulate=True)
+
+
+def test_active_ranks_through_the_chained_calls(b):
+    """The device-side rank with the queue-drawn launches (dlog_alpha finished inside the second backward launch)."""
+    w = I.WORKLOADS["bert"]
+    es = _run(b, I.Workload("a", "bf16", 1024, 1, w.matrices, w.alpha, w.target), 4, chained=True)
+    assert all(0 < int(e["k"].item()) < e["m"].r for e in es)
