@@ -229,8 +229,9 @@ class Job:
         self.sync = b.alloc_sync(device)
 
     def enable_active_ranks(self):
-        """Buffers and argument arrays for training on the active components only (z_k > 0): per layer one
-        gather, the grouped forward and backward with the rank read on the device, one scatter."""
+        """Buffers and argument arrays for training on the active components only (z_k > 0): per step one
+        select + gather (which also writes diag(z_c) Q_c), one dlog_alpha_c finish and one scatter over all matrices; per layer the
+        grouped forward and backward with the rank read on the device."""
         torch, b = self.torch, self.b
         bf = torch.bfloat16
         dev = self.log_alpha.device
@@ -245,28 +246,35 @@ class Job:
             e["zc"], e["dzc"], e["dlac"] = (torch.zeros(m.r, device=dev) for _ in range(3))
             e["Pc"], e["Qc"] = b.padded(m.d_out, m.r, bf, dev), b.padded(m.r, m.d_in, bf, dev)
             e["dPc"], e["dQc"] = b.padded(m.d_out, m.r, bf, dev), b.padded(m.r, m.d_in, bf, dev)
+            e["Qzc"] = b.padded(m.r, m.d_in, bf, dev)
         g = self.group if self.group > 0 else len(self.w.matrices)
-        for i in range(0, len(self.mats), g):
-            ch = self.mats[i:i + g]
-            z = lambda e: self.z[e["lo"]:e["hi"]]
-            gat = b.problem_array([b.active_gather_problem(z(e), self.dz_dla[e["lo"]:e["hi"]], e["P"], e["Q"], e["idx"], e["pos"],
-                                                           e["k"], e["zc"], e["dzc"], e["Pc"], e["Qc"]) for e in ch])
+        z = lambda e: self.z[e["lo"]:e["hi"]]
+        ms = self.mats
+        # once per step for the whole model: select + gather (with diag(z_c) Q_c), the dlog_alpha_c finish, the scatter
+        self.active_gather = b.problem_array([b.active_gather_problem(z(e), self.dz_dla[e["lo"]:e["hi"]], e["P"], e["Q"], e["idx"], e["pos"],
+                                                                      e["k"], e["zc"], e["dzc"], e["Pc"], e["Qc"], Qz_c=e["Qzc"]) for e in ms])
+        self.active_scatter = b.problem_array([b.active_scatter_problem(e["idx"], e["pos"], e["k"], e["m"].d_in, e["m"].d_out, e["m"].r,
+                                                                        e["dPc"], e["dQc"], e["dlac"], e["dP"], e["dQ"],
+                                                                        self.dlog_alpha[e["lo"]:e["hi"]]) for e in ms])
+        bwd_all = []
+        for i in range(0, len(ms), g):
+            ch = ms[i:i + g]
             fwd = b.problem_array([b.fwd_problem(e["X"], e["Qc"], e["Pc"], e["zc"], e["Y"], e["H"], r_dev=e["k"]) for e in ch])
-            bwd = b.problem_array([b.bwd_problem(e["dY"], e["X"], e["Qc"], e["Pc"], e["zc"], e["dzc"], e["H"], e["dX"], e["dPc"],
-                                                 e["dQc"], e["dlac"], e["ws"], r_dev=e["k"]) for e in ch])
-            sca = b.problem_array([b.active_scatter_problem(e["idx"], e["pos"], e["k"], e["m"].d_in, e["m"].d_out, e["m"].r,
-                                                            e["dPc"], e["dQc"], e["dlac"], e["dP"], e["dQ"],
-                                                            self.dlog_alpha[e["lo"]:e["hi"]]) for e in ch])
-            self.active_groups.append((gat, fwd, bwd, sca))
+            bl = [b.bwd_problem(e["dY"], e["X"], e["Qc"], e["Pc"], e["zc"], e["dzc"], e["H"], e["dX"], e["dPc"], e["dQc"], e["dlac"],
+                                e["ws"], r_dev=e["k"], Qz=e["Qzc"], defer_dlog_alpha=True) for e in ch]
+            bwd_all += bl
+            self.active_groups.append((fwd, b.problem_array(bl)))
+        self.active_finish = b.problem_array(bwd_all)
 
     def step_active(self):
         b = self.b
         self.sample_gates()
-        for gat, fwd, bwd, sca in self.active_groups:
-            b.active_ranks_gather(gat)
+        b.active_ranks_gather(self.active_gather)
+        for fwd, bwd in self.active_groups:
             b.gated_lowrank_fwd_grouped(fwd)
             b.gated_lowrank_bwd_grouped(bwd)
-            b.active_ranks_scatter(sca)
+        b.dlog_alpha_finish_grouped(self.active_finish)
+        b.active_ranks_scatter(self.active_scatter)
         self.finish()
 
     def input_bytes(self) -> int:
@@ -633,7 +641,7 @@ def main():
         frac = float(job.mask.float().mean().item())
         active = {"ms_per_step": act_ms, "value": w.T / (act_ms / 1e3), "unit": "tokens/s",
                   "active_fraction_last_step": frac,
-                  "note": "gather z>0 components, grouped fwd/bwd with device-side rank, scatter; same outputs as the dense step"}
+                  "note": "select + gather of the z>0 components (writing diag(z_c)Q_c too), dlog_alpha_c finish and scatter once per step for all matrices; grouped fwd/bwd per layer with device-side rank; same outputs as the dense step"}
         assert b.device_status() == b.OK
 
     e2e = None

@@ -279,8 +279,10 @@ int flop_gated_lowrank_bwd_chained(const flop_bwd_problem_t* problems, int n, in
  * inverse (-1 for closed gates), *k_dev = their number, z_c = z[idx],
  * dz_dla_c = dz_dla[idx] (both zero beyond k), Q_c[c,:] = Q[idx[c],:] (NOT scaled by
  * the gate), P_c[:,c] = P[:,idx[c]]; rows of Q_c / columns of P_c from k up to the
- * next multiple of 64 are zero.  All compact buffers have the capacity of the full
- * rank r.  bf16 only.
+ * next multiple of 64 are zero.  Qz_c (nullable, leading dimension ldqzc) receives
+ * diag(z_c) Q_c in the same launch, rounded to bf16 as flop_scale_rows_grouped rounds
+ * it: the buffer a backward problem takes as Qz.  All compact buffers have the
+ * capacity of the full rank r.  bf16 only.
  *
  * The grouped forward/backward calls then take the compact buffers in place of
  * P, Q, z, dz_dla, H_save, dP, dQ, dlog_alpha, with r = the capacity and
@@ -296,6 +298,7 @@ typedef struct {
   int64_t d_in, d_out, r;
   int32_t* idx; int32_t* pos; int32_t* k_dev; float* z_c; float* dz_dla_c;
   void* P_c; int64_t ldpc; void* Q_c; int64_t ldqc;
+  void* Qz_c; int64_t ldqzc;
 } flop_active_gather_t;
 
 typedef struct {

@@ -65,7 +65,8 @@ class ActiveGather(ctypes.Structure):
                 ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64),
                 ("idx", ctypes.c_void_p), ("pos", ctypes.c_void_p), ("k_dev", ctypes.c_void_p),
                 ("z_c", ctypes.c_void_p), ("dz_dla_c", ctypes.c_void_p),
-                ("P_c", ctypes.c_void_p), ("ldpc", ctypes.c_int64), ("Q_c", ctypes.c_void_p), ("ldqc", ctypes.c_int64)]
+                ("P_c", ctypes.c_void_p), ("ldpc", ctypes.c_int64), ("Q_c", ctypes.c_void_p), ("ldqc", ctypes.c_int64),
+                ("Qz_c", ctypes.c_void_p), ("ldqzc", ctypes.c_int64)]
 
 
 class ActiveScatter(ctypes.Structure):
@@ -354,11 +355,12 @@ def scale_rows_grouped(problems, dt: int = BF16) -> None:
     _check(load_library().flop_scale_rows_grouped(arr, len(arr), dt, _stream()), "flop_scale_rows_grouped")
 
 
-def active_gather_problem(z, dz_dla, P, Q, idx, pos, k_dev, z_c, dz_dla_c, P_c, Q_c) -> ActiveGather:
+def active_gather_problem(z, dz_dla, P, Q, idx, pos, k_dev, z_c, dz_dla_c, P_c, Q_c, Qz_c=None) -> ActiveGather:
     d_out, r = P.shape
     d_in = Q.shape[1]
     return ActiveGather(_p(z), _p(dz_dla), _p(P), _ld(P), _p(Q), _ld(Q), d_in, d_out, r, _p(idx), _p(pos), _p(k_dev),
-                        _p(z_c), _p(dz_dla_c), _p(P_c), _ld(P_c), _p(Q_c), _ld(Q_c))
+                        _p(z_c), _p(dz_dla_c), _p(P_c), _ld(P_c), _p(Q_c), _ld(Q_c), _p(Qz_c),
+                        _ld(Qz_c) if Qz_c is not None else 0)
 
 
 def active_scatter_problem(idx, pos, k_dev, d_in, d_out, r, dP_c, dQ_c, dla_c, dP, dQ, dla) -> ActiveScatter:

@@ -10,7 +10,8 @@
 //   active_gather_kernel   Q_c[c,:] = Q[idx[c],:] (UNscaled: the gate stays in the GEMM epilogue and
 //                          the fused <Q, .> reduction needs the raw rows), P_c[:,c] = P[:,idx[c]];
 //                          rows / columns from k up to the next multiple of 64 are zero-filled,
-//                          because the GEMMs' K loops and N extents run to that boundary
+//                          because the GEMMs' K loops and N extents run to that boundary; optionally
+//                          also Qz_c = diag(z_c) Q_c, the backward pass's B operand for dX
 //   active_scatter_kernel  dP[:,idx] = dP_c, dQ[idx,:] = dQ_c, dlog_alpha[idx] = dlog_alpha_c and
 //                          exact zeros everywhere else (or += when accumulating)
 #pragma once
@@ -18,7 +19,7 @@
 
 namespace flop {
 
-constexpr int kActiveGroup = 8;
+constexpr int kActiveGroup = 96;   // matrices per launch: a whole model's worth in one group (argument block ~13 KB)
 
 struct ActiveGather {
   const float* z; const float* dz_dla;                 // [r], dz_dla nullable
@@ -27,6 +28,7 @@ struct ActiveGather {
   int32_t* idx; int32_t* pos; int32_t* k_dev;          // [r], [r], [1]
   float* z_c; float* dz_dla_c;                         // [r], dz_dla_c nullable
   __nv_bfloat16* P_c; int64_t ldpc; __nv_bfloat16* Q_c; int64_t ldqc;
+  __nv_bfloat16* Qz_c; int64_t ldqzc;                  // nullable: diag(z_c) Q_c
 };
 struct ActiveGatherGroup { ActiveGather a[kActiveGroup]; int n; };
 
@@ -79,14 +81,37 @@ active_gather_kernel(const __grid_constant__ ActiveGatherGroup g, int smem_row_e
     const int c = t;
     if (c >= kp) return;
     __nv_bfloat16* o = a.Q_c + (int64_t)c * a.ldqc;
+    __nv_bfloat16* oz = a.Qz_c ? a.Qz_c + (int64_t)c * a.ldqzc : nullptr;
     if (c < k) {
-      const __nv_bfloat16* q = a.Q + (int64_t)a.idx[c] * a.ldq;
+      const int src = a.idx[c];
+      const __nv_bfloat16* q = a.Q + (int64_t)src * a.ldq;
+      const float zc = a.z[src];
       for (int j = lane * 8; j < a.d_in; j += 32 * 8) {     // rows are 16-byte aligned (ld % 8 == 0)
-        if (j + 8 <= a.d_in) *reinterpret_cast<uint4*>(o + j) = *reinterpret_cast<const uint4*>(q + j);
-        else for (int e = j; e < a.d_in; ++e) o[e] = q[e];
+        if (j + 8 <= a.d_in) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(q + j);
+          *reinterpret_cast<uint4*>(o + j) = raw;
+          if (oz) {
+            uint4 sc = raw;
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&sc);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 x = __bfloat1622float2(h[e]);
+              h[e] = __floats2bfloat162_rn(x.x * zc, x.y * zc);
+            }
+            *reinterpret_cast<uint4*>(oz + j) = sc;
+          }
+        } else {
+          for (int e = j; e < a.d_in; ++e) {
+            o[e] = q[e];
+            if (oz) oz[e] = __float2bfloat16_rn(__bfloat162float(q[e]) * zc);
+          }
+        }
       }
     } else {
-      for (int j = lane; j < a.d_in; j += 32) o[j] = __float2bfloat16_rn(0.f);
+      for (int j = lane; j < a.d_in; j += 32) {
+        o[j] = __float2bfloat16_rn(0.f);
+        if (oz) oz[j] = __float2bfloat16_rn(0.f);
+      }
     }
   } else {
     const int i = t - a.r;

@@ -1800,14 +1800,17 @@ int flop_active_ranks_gather(const flop_active_gather_t* pr, int n, int dt, void
       if (a.r <= 0 || a.d_in <= 0 || a.d_out <= 0 || a.r > INT32_MAX / 2 || a.d_in > INT32_MAX || a.d_out > INT32_MAX / 2)
         return FLOP_ERR_INVALID_ARG;
       if (!a.z || !a.P || !a.Q || !a.idx || !a.pos || !a.k_dev || !a.z_c || !a.P_c || !a.Q_c || a.ldp < a.r || a.ldq < a.d_in ||
-          a.ldpc < a.r || a.ldqc < a.d_in || (a.dz_dla_c && !a.dz_dla))
+          a.ldpc < a.r || a.ldqc < a.d_in || (a.dz_dla_c && !a.dz_dla) || (a.Qz_c && a.ldqzc < a.d_in))
         return FLOP_ERR_INVALID_ARG;
-      if (!bf16_ok(a.P, a.ldp) || !bf16_ok(a.Q, a.ldq) || !bf16_ok(a.P_c, a.ldpc) || !bf16_ok(a.Q_c, a.ldqc)) return FLOP_ERR_UNSUPPORTED;
+      if (!bf16_ok(a.P, a.ldp) || !bf16_ok(a.Q, a.ldq) || !bf16_ok(a.P_c, a.ldpc) || !bf16_ok(a.Q_c, a.ldqc) ||
+          (a.Qz_c && !bf16_ok(a.Qz_c, a.ldqzc)))
+        return FLOP_ERR_UNSUPPORTED;
       if ((size_t)a.r * 2 * kActiveWarps > (size_t)kSmemBudget) return FLOP_ERR_UNSUPPORTED;
       ActiveGather& o = g.a[g.n];
       o.z = a.z; o.dz_dla = a.dz_dla; o.P = (const bf16*)a.P; o.ldp = a.ldp; o.Q = (const bf16*)a.Q; o.ldq = a.ldq;
       o.r = (int)a.r; o.d_in = (int)a.d_in; o.d_out = (int)a.d_out; o.idx = a.idx; o.pos = a.pos; o.k_dev = a.k_dev;
       o.z_c = a.z_c; o.dz_dla_c = a.dz_dla_c; o.P_c = (bf16*)a.P_c; o.ldpc = a.ldpc; o.Q_c = (bf16*)a.Q_c; o.ldqc = a.ldqc;
+      o.Qz_c = (bf16*)a.Qz_c; o.ldqzc = a.ldqzc;
       max_blocks = std::max(max_blocks, o.r + o.d_out);
       max_r = std::max(max_r, o.r);
     }

@@ -20,7 +20,7 @@ def b():
     return binding
 
 
-def _run(b, w: I.Workload, seed, alpha_shift=0.0, wdt=torch.bfloat16, accumulate=False, chained=False):
+def _run(b, w: I.Workload, seed, alpha_shift=0.0, wdt=torch.bfloat16, accumulate=False, chained=False, per_step=False):
     bf = torch.bfloat16
     es, gat, fwd, bwd, sca = [], [], [], [], []
     for i, m in enumerate(w.matrices):
@@ -45,11 +45,12 @@ def _run(b, w: I.Workload, seed, alpha_shift=0.0, wdt=torch.bfloat16, accumulate
         e["dla"] = torch.full((m.r,), init, device="cuda")
         e["ws"] = b.alloc_workspace(b.workspace_bytes(b.OP_BWD, T, m.d_in, m.d_out, m.r, b.BF16))
         e["ws"].fill_(0xFF)
+        e["Qzc"] = empty_dev(m.r, m.d_in, bf) if per_step else None
         gat.append(b.active_gather_problem(e["z"], e["dzd"], e["P"], e["Q"], e["idx"], e["pos"], e["k"], e["zc"], e["dzc"],
-                                           e["Pc"], e["Qc"]))
+                                           e["Pc"], e["Qc"], Qz_c=e["Qzc"] if per_step == "gather" else None))
         fwd.append(b.fwd_problem(e["X"], e["Qc"], e["Pc"], e["zc"], e["Y"], e["Hc"], r_dev=e["k"]))
         bwd.append(b.bwd_problem(e["dY"], e["X"], e["Qc"], e["Pc"], e["zc"], e["dzc"], e["Hc"], e["dX"], e["dPc"], e["dQc"],
-                                 e["dlac"], e["ws"], r_dev=e["k"]))
+                                 e["dlac"], e["ws"], r_dev=e["k"], Qz=e["Qzc"], defer_dlog_alpha=bool(per_step)))
         sca.append(b.active_scatter_problem(e["idx"], e["pos"], e["k"], m.d_in, m.d_out, m.r, e["dPc"], e["dQc"], e["dlac"],
                                             e["dP"], e["dQ"], e["dla"]))
         es.append(e)
@@ -60,6 +61,19 @@ def _run(b, w: I.Workload, seed, alpha_shift=0.0, wdt=torch.bfloat16, accumulate
         b.gated_lowrank_fwd_chained(fwd, sync)
         b.gated_lowrank_bwd_chained(bwd, sync, wgrad_dt=wd)
         assert int(sync.view(torch.int32).abs().sum().item()) == 0
+    elif per_step:
+        # the per-step form: diag(z_c) Q_c formed once for all matrices, dlog_alpha_c finished once after all backward calls
+        if per_step == "gather":     # diag(z_c) Q_c came out of the gather launch
+            for e in es:
+                k = int(e["k"].item())
+                sel = np.nonzero(e["mask"])[0]
+                want = I.round_to_bf16(e["prob"]["Q"][sel].astype(np.float32) * e["z_np"][sel, None])
+                assert np.array_equal(host(e["Qzc"])[:k], want.astype(np.float64))
+        else:
+            b.scale_rows_grouped([b.scale_rows_problem(e["Qc"], e["zc"], e["Qzc"]) for e in es])
+        b.gated_lowrank_fwd_grouped(fwd)
+        b.gated_lowrank_bwd_grouped(bwd, wgrad_dt=wd)
+        b.dlog_alpha_finish_grouped(bwd)
     else:
         b.gated_lowrank_fwd_grouped(fwd)
         b.gated_lowrank_bwd_grouped(bwd, wgrad_dt=wd)
@@ -119,3 +133,15 @@ def test_active_ranks_through_the_chained_calls(b):
     w = I.WORKLOADS["bert"]
     es = _run(b, I.Workload("a", "bf16", 1024, 1, w.matrices, w.alpha, w.target), 4, chained=True)
     assert all(0 < int(e["k"].item()) < e["m"].r for e in es)
+
+
+@pytest.mark.parametrize("wdt", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("qz_from", ["gather", "scale_rows"])
+def test_active_ranks_per_step_side_work(b, wdt, qz_from):
+    """diag(z_c) Q_c from the gather launch (or one grouped scaling launch) and dlog_alpha_c from one deferred finish,
+    with the rank read on the device."""
+    w = I.WORKLOADS["bert"]
+    es = _run(b, I.Workload("a", "bf16", 1024, 1, w.matrices, w.alpha, w.target), 5, wdt=wdt, per_step=qz_from)
+    assert all(0 < int(e["k"].item()) < e["m"].r for e in es)
+    w2 = I.Workload("a", "bf16", 700, 1, I.WORKLOADS["txl"].matrices, ("normal", 0.5, 1.0), 0.35)
+    _run(b, w2, 6, wdt=wdt, per_step=qz_from)
