@@ -477,6 +477,14 @@ __device__ __forceinline__ void stage_chunk(const Params& p, const uint32_t (&v)
 // direct global stores would touch 32 different rows per instruction (32 partial sectors), which
 // measured ~7000 cycles per block against the ~400 of the staged store; the tensor map also clips
 // the ragged edges.  Otherwise (fp32 outputs, accumulate, split-K slices) each thread stores its row.
+// Arrival on a barrier that may live in the other CTA of the pair.  CTA-scope release: the tensor-memory loads this
+// arrival hands back are complete (tcgen05.wait::ld) and fenced (tcgen05.fence::before_thread_sync) when it is
+// issued, and the thread publishes no ordinary memory with it.  A cluster-scope release here made the thread wait for
+// all its outstanding stores to be acknowledged, 1000-1500 cycles per tile under load.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
 template <int EPI, bool kClusterArrive>
 __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap* tmap_out, uint32_t store_buf, uint32_t t_acc,
                                              int row0, int n_base, int n_limit, int split, int tn, int warp, int lane,
@@ -504,7 +512,7 @@ __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap*
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) {
-        if (kClusterArrive) asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(release_bar) : "memory");
+        if (kClusterArrive) mbar_arrive_remote(release_bar);
         else mbar_arrive(release_bar);
       }
       released = true;
@@ -531,7 +539,7 @@ __device__ __forceinline__ void run_epilogue(const Params& p, const CUtensorMap*
     tcgen05_fence_before();
     __syncwarp();
     if (lane == 0) {
-      if (kClusterArrive) asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(release_bar) : "memory");
+      if (kClusterArrive) mbar_arrive_remote(release_bar);
       else mbar_arrive(release_bar);
     }
   }
