@@ -436,8 +436,24 @@ __device__ __forceinline__ void qdot_chunk(const Params& p, const uint32_t (&v)[
 template <int EPI>
 __device__ __forceinline__ void stage_chunk(const Params& p, const uint32_t (&v)[32], int row, int n0, uint32_t buf,
                                             int piece0, int lane) {
+  const uint32_t row_addr = buf + (uint32_t)lane * 128u;
+  const bool col_gate = EPI == EPI_STORE && p.col_scale;
+  const bool row_gate = EPI == EPI_WGRAD && p.row_scale;
+  if (!col_gate && !row_gate) {      // plain conversion
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * j]), __uint_as_float(v[8 * i + 2 * j + 1]));
+        pk[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      st_shared_v4(row_addr + (uint32_t)(((piece0 + i) ^ (lane & 7)) << 4), pk[0], pk[1], pk[2], pk[3]);
+    }
+    return;
+  }
   float sc[32];
-  if (EPI == EPI_STORE && p.col_scale) {
+  if (col_gate) {
     if (n0 + 32 <= p.N && (reinterpret_cast<uintptr_t>(p.col_scale + n0) & 15) == 0) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -449,11 +465,10 @@ __device__ __forceinline__ void stage_chunk(const Params& p, const uint32_t (&v)
       for (int i = 0; i < 32; ++i) sc[i] = n0 + i < p.N ? __ldg(p.col_scale + n0 + i) : 0.f;
     }
   } else {
-    const float rs = (EPI == EPI_WGRAD && p.row_scale && row < p.M) ? __ldg(p.row_scale + row) : 1.f;
+    const float rs = row < p.M ? __ldg(p.row_scale + row) : 1.f;
 #pragma unroll
     for (int i = 0; i < 32; ++i) sc[i] = rs;
   }
-  const uint32_t row_addr = buf + (uint32_t)lane * 128u;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     uint32_t pk[4];

@@ -3,8 +3,8 @@
 // measures that matter at BERT / Transformer-XL sizes: several tiles per CTA, so that pipeline
 // fill and epilogue drain overlap the next tile's main loop, and half a B tile per SM, so that the
 // bytes an SM has to pull from L2 per MMA drop by about 40 % (that fill rate, ~50 B/clk/SM, is what
-// bounds the one-CTA 128 x 192 x 768 tile; the pair's main loop runs at 84 % of the tensor pipe and
-// no longer responds to the bytes loaded).  Problem table, work list and epilogues are
+// bounds the one-CTA 128 x 192 x 768 tile; the pair's main loop runs at 87-89 % of the tensor pipe and
+// hardly responds to the bytes loaded).  Problem table, work list and epilogues are
 // those of gemm_group_kernel; pair protocol and bounded waits are described in gemm_tc2.cuh.
 #pragma once
 #include "gemm_tc2.cuh"
