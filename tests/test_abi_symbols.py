@@ -63,3 +63,42 @@ def test_workspace_query_and_argument_checks(lib):
                                       None, 0, None) == b.OK                              # T = 0
     assert lib.flop_compact_ranks(None, 2, good, 8, None, 0, None, 0, 0, 0, 0, None, None, None, None, 0, None, 0,
                                   None, 0, None) == b.ERR_INVALID_ARG
+
+
+def test_struct_layouts_match_the_header(tmp_path):
+    """Every argument struct of include/flop.h, compiled as plain C, has the size and the field offsets of its
+    ctypes mirror in the binding (a field added on one side only would shift every pointer after it)."""
+    import shutil
+    import subprocess
+    from paper_1910_04732_b200 import binding as b
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    pairs = {"flop_hc_params_t": b.HcParams, "flop_fwd_problem_t": b.FwdProblem, "flop_bwd_problem_t": b.BwdProblem,
+             "flop_scale_rows_t": b.ScaleRows, "flop_active_gather_t": b.ActiveGather,
+             "flop_active_scatter_t": b.ActiveScatter}
+    text = open(os.path.join(ROOT, "include", "flop.h")).read()
+    structs = set(re.findall(r"}\s*(flop_[a-z0-9_]+_t)\s*;", re.sub(r"/\*.*?\*/", "", text, flags=re.S)))
+    structs -= {"flop_status_t", "flop_op_t", "flop_dtype_t"}      # enums
+    assert structs == set(pairs), structs ^ set(pairs)
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "flop.h"', 'int main(void) {']
+    for cname, cls in pairs.items():
+        lines.append(f'  printf("{cname} size %zu\\n", sizeof({cname}));')
+        for fname, _ in cls._fields_:
+            lines.append(f'  printf("{cname} {fname} %zu\\n", offsetof({cname}, {fname}));')
+    lines += ['  return 0;', '}']
+    src, exe = tmp_path / "layout.c", tmp_path / "layout"
+    src.write_text("\n".join(lines))
+    subprocess.check_call(["gcc", "-std=c99", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)])
+    out = subprocess.check_output([str(exe)], text=True).split("\n")
+    want = {}
+    for ln in out:
+        if ln.strip():
+            c, f, v = ln.split()
+            want[(c, f)] = int(v)
+    for cname, cls in pairs.items():
+        assert ctypes.sizeof(cls) == want[(cname, "size")], cname
+        for fname, _ in cls._fields_:
+            assert getattr(cls, fname).offset == want[(cname, fname)], (cname, fname)
+        # and no field of the C struct is missing from the mirror: the sizes agree and the last field ends the struct
+        last = cls._fields_[-1][0]
+        assert getattr(cls, last).offset + getattr(cls, last).size <= ctypes.sizeof(cls)
