@@ -420,6 +420,12 @@ int add_problem(tc::GroupParams& gp, const TcJob& j, std::vector<double>& item_c
   p.M = (int)j.M; p.N = (int)j.N; p.K = (int)j.K;
   p.bn = j.pl.bn; p.stages = 0; p.tiles_m = j.pl.tiles_m; p.tiles_n = j.pl.tiles_n;
   p.splits = j.pl.splits; p.kb_per_split = j.pl.kb_per_split; p.num_kb = j.pl.num_kb;
+  {
+    const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n, items = tiles * std::max(p.splits, 1);
+    p.div_fast = items < 65536 ? 1 : 0;
+    p.magic_tn = p.tiles_n > 1 ? (uint32_t)(0x100000000ull / (uint64_t)p.tiles_n) + 1u : 0u;
+    p.magic_tiles = (p.div_fast && tiles > 1) ? (uint32_t)(0x100000000ull / (uint64_t)tiles) + 1u : 0u;
+  }
   p.out = j.ep.out; p.ldo = j.ep.ldo; p.col_scale = j.ep.col_scale;
   p.slices = j.ep.slices; p.slice_elems = j.ep.slice_elems; p.ld_slice = j.ep.ld_slice;
   p.qdot = j.ep.qdot; p.ldq = j.ep.ldq; p.dz_part = j.ep.dz_part; p.dz_stride = j.ep.dz_stride; p.dz_meta = j.ep.dz_meta;
@@ -488,6 +494,16 @@ int launch_tc_group(const std::vector<TcJob>& jobs, cudaStream_t st) {
       } else {
         const double lpt = tc::build_schedule(item_cost, units, &gp.sched, &rr);
         if (lpt < 0.0 || lpt > 0.97 * rr) gp.sched.n_units = 0;
+        if (gp.sched.n_units) {     // every entry also names its problem, so that no role has to search for it
+          static_assert(tc::kMaxSched <= (1 << tc::kSchedProblemShift) && tc::kMaxGroup <= (1 << (16 - tc::kSchedProblemShift)), "entry bits");
+          for (int i = 0; i < gp.total_work; ++i) {
+            const int w = gp.sched.item[i];
+            int g = 0;
+            for (int k = 1; k < gp.n; ++k)
+              if (w >= gp.prob[k].work_begin) g = k;
+            gp.sched.item[i] = (uint16_t)((g << tc::kSchedProblemShift) | w);
+          }
+        }
       }
     }
     const bool a_mn = first.A.mn_major, b_mn = first.B.mn_major;

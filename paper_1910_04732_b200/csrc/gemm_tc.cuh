@@ -65,6 +65,9 @@ struct Params {
   int bn;                 // N per tile: 64, 128, 192, 208 (CTA pairs, K-major B) or 256
   int stages;
   int tiles_m, tiles_n, splits, kb_per_split, num_kb;
+  // floor(2^32 / d) + 1 for d = tiles_n and d = tiles_m * tiles_n: n / d == __umulhi(n, magic) for n, d < 65536
+  // (div_fast = 1 when the problem has fewer than 65536 work items); saves the two integer divisions per tile decode
+  uint32_t magic_tn, magic_tiles; int div_fast;
   // EPI_STORE: out[m*ldo + n] = acc * col_scale[n]  (bf16)
   __nv_bfloat16* out; int64_t ldo;
   const float* col_scale;               // nullable
@@ -212,10 +215,17 @@ struct WorkItem { int tm, tn, split, kb0, kb1; };
 __device__ __forceinline__ WorkItem decode(const Params& p, int w) {
   WorkItem it;
   const int tiles = p.tiles_m * p.tiles_n;
-  it.split = w / tiles;
-  const int t = w - it.split * tiles;
-  it.tm = t / p.tiles_n;
-  it.tn = t - it.tm * p.tiles_n;
+  if (p.div_fast) {
+    it.split = tiles == 1 ? w : (int)__umulhi((uint32_t)w, p.magic_tiles);
+    const int t = w - it.split * tiles;
+    it.tm = p.tiles_n == 1 ? t : (int)__umulhi((uint32_t)t, p.magic_tn);
+    it.tn = t - it.tm * p.tiles_n;
+  } else {
+    it.split = w / tiles;
+    const int t = w - it.split * tiles;
+    it.tm = t / p.tiles_n;
+    it.tn = t - it.tm * p.tiles_n;
+  }
   it.kb0 = it.split * p.kb_per_split;
   it.kb1 = min(it.kb0 + p.kb_per_split, p.num_kb);
   return it;

@@ -134,7 +134,7 @@ gemm2_dual_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t phase = 0;
       bool ok = true;
       for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-        const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
+        const GroupItem it = work_item(gp, wi, BM2);
         if (!it.active) continue;
         if (gp.prob[it.g].p.kind == 0) ok = pair_produce_item<A0, B0>(gp, it, rank, smem_base, sbytes, bars, stage, phase, abort_flag);
         else                           ok = pair_produce_item<A1, B1>(gp, it, rank, smem_base, sbytes, bars, stage, phase, abort_flag);
@@ -155,7 +155,7 @@ gemm2_dual_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-        const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
+        const GroupItem it = work_item(gp, wi, BM2);
         if (!it.active) continue;
         if (gp.prob[it.g].p.kind == 0)
           ok = pair_mma_item<A0, B0>(gp, it, smem_base, sbytes, bars, tmem_base, stage, phase, acc, acc_phase, abort_flag);
@@ -169,7 +169,7 @@ gemm2_dual_kernel(const __grid_constant__ GroupParams gp) {
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-      const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
+      const GroupItem it = work_item(gp, wi, BM2);
       if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
       if (!mbar_wait2(bars.tfull(acc), acc_phase, abort_flag)) { ok = false; }

@@ -64,7 +64,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t phase = 0;
       bool ok = true;
       for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-        const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
+        const GroupItem it = work_item(gp, wi, BM2);
         if (!it.active) continue;
         const GroupProblem& pr = gp.prob[it.g];
         const int half_n = pr.p.bn >> 1;
@@ -108,7 +108,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-        const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
+        const GroupItem it = work_item(gp, wi, BM2);
         if (!it.active) continue;
         const uint32_t idesc = instr_desc2(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait2(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -138,7 +138,7 @@ gemm2_group_kernel(const __grid_constant__ GroupParams gp) {
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-      const GroupItem it = decode_group(gp, work_at(gp, wi), BM2);
+      const GroupItem it = work_item(gp, wi, BM2);
         if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
       if (!mbar_wait2(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }

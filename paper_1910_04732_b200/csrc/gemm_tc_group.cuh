@@ -52,7 +52,7 @@ __device__ __forceinline__ WorkRange work_range(const GroupParams& gp, int unit,
   if (gp.sched.n_units) return WorkRange{(int)gp.sched.begin[unit], (int)gp.sched.begin[unit + 1], 1};
   return WorkRange{unit, gp.total_work, nunits};
 }
-__device__ __forceinline__ int work_at(const GroupParams& gp, int i) { return gp.sched.n_units ? (int)gp.sched.item[i] : i; }
+__device__ __forceinline__ int work_at(const GroupParams& gp, int i) { return gp.sched.n_units ? (int)gp.sched.item[i] : i; }   // chained launches: plain indices
 
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -65,11 +65,7 @@ struct GroupItem { int g, tm, tn, split, kb0, kb1, n_limit; bool active; };
 // Work item w of the group; bm = rows of D per tile (128, or 256 for a CTA pair).  When a problem
 // carries device-side sizes the item may lie outside the effective extent (active = false: every
 // role skips it, so stage and accumulator phases stay in step) or have a shorter K loop.
-__device__ __forceinline__ GroupItem decode_group(const GroupParams& gp, int w, int bm) {
-  int g = 0;
-#pragma unroll
-  for (int i = 1; i < kMaxGroup; ++i)
-    if (i < gp.n && w >= gp.prob[i].work_begin) g = i;
+__device__ __forceinline__ GroupItem decode_problem_item(const GroupParams& gp, int g, int w, int bm) {
   const Params& p = gp.prob[g].p;
   const WorkItem it = decode(p, w - gp.prob[g].work_begin);
   GroupItem o{g, it.tm, it.tn, it.split, it.kb0, it.kb1, p.N, true};
@@ -82,6 +78,21 @@ __device__ __forceinline__ GroupItem decode_group(const GroupParams& gp, int w, 
     o.active = o.tm * bm < m_eff && o.tn * p.bn < n_eff && o.kb0 < o.kb1;
   }
   return o;
+}
+__device__ __forceinline__ GroupItem decode_group(const GroupParams& gp, int w, int bm) {
+  int g = 0;
+  for (int i = 1; i < gp.n && w >= gp.prob[i].work_begin; ++i) g = i;   // work_begin ascends; a group of one needs no step
+  return decode_problem_item(gp, g, w, bm);
+}
+// Entry i of a unit's list.  A schedule table built by the grouped launches carries the problem index in the upper
+// five bits of its 16-bit entries (kSchedProblemShift), which saves the walk over the problem table once per tile and
+// role; without a table the entry is the work-list index itself.
+__device__ __forceinline__ GroupItem work_item(const GroupParams& gp, int i, int bm) {
+  if (gp.sched.n_units) {
+    const int e = (int)gp.sched.item[i];
+    return decode_problem_item(gp, e >> kSchedProblemShift, e & ((1 << kSchedProblemShift) - 1), bm);
+  }
+  return decode_group(gp, i, bm);
 }
 
 template <bool A_MN, bool B_MN, int EPI>
@@ -131,7 +142,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       int armed = 0;
       bool ok = true;
       for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-        const GroupItem it = decode_group(gp, work_at(gp, wi), BM);
+        const GroupItem it = work_item(gp, wi, BM);
         if (!it.active) continue;
         const GroupProblem& pr = gp.prob[it.g];
         const int bn = pr.p.bn;
@@ -178,7 +189,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-        const GroupItem it = decode_group(gp, work_at(gp, wi), BM);
+        const GroupItem it = work_item(gp, wi, BM);
         if (!it.active) continue;
         const uint32_t idesc = instr_desc(A_MN, B_MN, gp.prob[it.g].p.bn);
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -208,7 +219,7 @@ gemm_group_kernel(const __grid_constant__ GroupParams gp) {
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int wi = wr.first; wi < wr.last && ok; wi += wr.step) {
-      const GroupItem it = decode_group(gp, work_at(gp, wi), BM);
+      const GroupItem it = work_item(gp, wi, BM);
         if (!it.active) continue;
       const Params& p = gp.prob[it.g].p;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; }

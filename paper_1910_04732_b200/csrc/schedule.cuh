@@ -26,6 +26,7 @@ namespace flop {
 namespace tc {
 
 constexpr int kMaxSched = 2048;   // work items a table can hold
+constexpr int kSchedProblemShift = 11;   // grouped launches: entry = (problem index << 11) | work-list index
 constexpr int kMaxUnits = 148;    // persistent CTAs (one-CTA kernel) or pairs (two-CTA kernel)
 
 struct Schedule {
